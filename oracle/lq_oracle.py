@@ -1,0 +1,288 @@
+"""CPU oracle for the LoRaQ fully quantized linear layer.  TEST INFRASTRUCTURE ONLY.
+
+This file is a plain, slow, obviously-correct numpy statement of what the hot
+path computes.  It is imported only by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg; the product (the CUDA library and its binding)
+never imports it and shares no code, table or constant generator with it.
+
+What it follows
+---------------
+* Quantization error / upper bound: Section 3.1 (Eq. "error_upper_bound").
+* Error absorption, idempotence of Q, the calibration objective
+  ``min_{L,R} || Q(W + L R) - W - L R ||_F`` (MSE form): Section 3.2
+  (Eq. "quantization-error", Eq. "low-rank-optimization").
+* SVD initialisation ``L = -L0, R = R0``: Section 3.2, last paragraph.
+* Gradients with dQ/d. = 0 almost everywhere: Appendix B.2
+  (Eq. "low-rank-gradients", "low-rank-gradients-update", "...-R").
+* Adam, 1000 steps, learning rate 1e-4 for integer formats: Appendix A.1/A.2 "Optimization".
+* Two quantizers Q1 (residual branch) and Q2 (low-rank branch), residual
+  ``P = W - Q2(L)Q2(R)``: Section 3.3 (Eq. "quantization-lr") and the Figure 1 caption.
+* Decomposed forward ``Y = Q(X) Q1(P) + Q(X) Q2(L) Q2(R)`` with the activations of
+  both branches quantized: Figure 1 caption and Appendix A.2 "Quantization".
+* SINT4 format (signed int4, blocks of 64 values, one FP16 scale per block,
+  round-to-nearest): Appendix A.3 "Blockwise Formats".
+
+Readings taken where the paper is silent (each is listed in the design notes):
+symmetric range [-7, 7] with scale = absmax / 7 rounded to fp16; ties to even;
+scale floor 2^-24; groups run along the contraction axis K; a short last group
+when K is not a multiple of 64; the branch quantizers (W8A8 / W6A6 / W4A8) are
+symmetric integers with one fp32 scale per token (activations, and the rank-r
+intermediate) or per output column (the two factors); the intermediate
+``T = Q(X) Q(L1)`` is re-quantized per token; Q2 is applied after the Adam loop
+and P is recomputed from the quantized factors; Sigma is split evenly between
+L0 and R0; the loss is the mean over K*N entries; Adam uses (0.9, 0.999, 1e-8)
+with bias correction; the best iterate seen is returned.
+
+Parity unpinned (the paper prints no number for them): the Adam trajectory, the
+split of Sigma between L0 and R0.
+
+Arithmetic conventions: every "fl32" operation is IEEE binary32, round to nearest
+even, true division, no fused multiply-add (numpy float32 scalars/arrays obey
+this).  Integer products are exact (carried in float64, whose 53-bit significand
+holds every sum that occurs).  Final sums are float64.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+GROUP = 64                      # SINT4 block (Appendix A.3)
+QMAX4 = 7                       # symmetric signed int4: codes in [-7, 7]
+SCALE_FLOOR = np.float16(2.0 ** -24)   # smallest positive fp16
+
+# branch format -> (weight bits, activation bits); None = fp16 (the W16A16 reference)
+BRANCH_BITS = {"w8a8": (8, 8), "w6a6": (6, 6), "w4a8": (4, 8), "w16a16": (None, None), "none": (0, 0)}
+
+
+def qmax(bits: int) -> int:
+    return (1 << (bits - 1)) - 1
+
+
+# --------------------------------------------------------------------------------------
+# Quantizers (Appendix A.3; Section 3.2 for idempotence)
+# --------------------------------------------------------------------------------------
+def qgrp(v, group: int = GROUP):
+    """SINT4 quantizer along the last axis of a 2-D array.
+
+    v[i, :] is cut into consecutive groups of `group` values (the last may be
+    short).  Per group: a = max|v| in fl32; s = fp16(a /fl32 7), floored at 2^-24;
+    q = clamp(rint_even(v /fl32 s), -7, 7).
+    Returns (codes int8 [R, L], scales fp16 [R, ceil(L/group)]).
+    """
+    v = np.asarray(v, dtype=np.float32)
+    R, L = v.shape
+    G = -(-L // group)
+    codes = np.zeros((R, L), dtype=np.int8)
+    scales = np.zeros((R, G), dtype=np.float16)
+    for g in range(G):
+        blk = v[:, g * group:(g + 1) * group]
+        a = np.max(np.abs(blk), axis=1).astype(np.float32)
+        s = (a / np.float32(QMAX4)).astype(np.float16)
+        s = np.maximum(s, SCALE_FLOOR)
+        q = np.rint(blk / s.astype(np.float32)[:, None])
+        codes[:, g * group:(g + 1) * group] = np.clip(q, -QMAX4, QMAX4).astype(np.int8)
+        scales[:, g] = s
+    return codes, scales
+
+
+def deq_grp(codes, scales, group: int = GROUP):
+    """float64 values s * q of a qgrp() result."""
+    R, L = codes.shape
+    s = np.repeat(scales.astype(np.float64), group, axis=1)[:, :L]
+    return s * codes.astype(np.float64)
+
+
+def qtok(v, bits: int):
+    """Symmetric integer quantizer with ONE fp32 scale per row of a 2-D array.
+
+    a = max|row| in fl32; s = a /fl32 qmax(bits), s = 1 when a == 0;
+    q = clamp(rint_even(v /fl32 s), -qmax, qmax).  Returns (codes int8, scales fp32 [R]).
+    """
+    v = np.asarray(v, dtype=np.float32)
+    qm = qmax(bits)
+    a = np.max(np.abs(v), axis=1).astype(np.float32) if v.shape[1] else np.zeros(v.shape[0], np.float32)
+    s = (a / np.float32(qm)).astype(np.float32)
+    s = np.where(a == 0, np.float32(1.0), s).astype(np.float32)
+    q = np.rint(v / s[:, None])
+    return np.clip(q, -qm, qm).astype(np.int8), s
+
+
+def deq_tok(codes, scales):
+    return scales.astype(np.float64)[:, None] * codes.astype(np.float64)
+
+
+def q_weight_main(P):
+    """Q1 on the residual weight P [K, N]: SINT4 groups along K for each output column n.
+    Returns (Wq int8 [K, N], sw fp16 [G, N])."""
+    c, s = qgrp(np.asarray(P, dtype=np.float32).T.copy())
+    return c.T.copy(), s.T.copy()
+
+
+def deq_weight_main(Wq, sw):
+    return deq_grp(Wq.T.copy(), sw.T.copy()).T.copy()
+
+
+def q_factor(F, bits):
+    """Q2 on a branch factor, one scale per COLUMN (L1: per column j over K; L2: per column n over r).
+    bits None = fp16 cast (W16A16).  Returns (codes-or-fp16 array, scales fp32 or None)."""
+    if bits is None:
+        return np.asarray(F, dtype=np.float32).astype(np.float16), None
+    c, s = qtok(np.asarray(F, dtype=np.float32).T.copy(), bits)
+    return c.T.copy(), s
+
+
+def deq_factor(Fq, s):
+    if s is None:
+        return Fq.astype(np.float64)
+    return Fq.astype(np.float64) * s.astype(np.float64)[None, :]
+
+
+# --------------------------------------------------------------------------------------
+# Forward of the decomposed layer (Figure 1; Appendix A.2)
+# --------------------------------------------------------------------------------------
+def forward(X16, layer, group: int = GROUP):
+    """All intermediates and the float64 output of one quantized linear layer.
+
+    layer: dict with Wq int8 [K,N], sw fp16 [G,N], branch (str), rank, and for integer
+    branches L1q int8 [K,r], sL1 f32 [r], L2q int8 [r,N], sL2 f32 [N]; for "w16a16"
+    L1h fp16 [K,r], L2h fp16 [r,N]; optional bias fp16 [N].
+    Steps: (1) qx,sx = SINT4 per token and group; (2) qb,sXb = per-token branch codes;
+    (3) I1 = qb L1q exact; (4) t = fl32(fl32(I1) * fl32(sXb * sL1)); (5) tq,sT = per-token;
+    (6) P_g = qx_g Wq_g exact; (7) U = tq L2q exact;
+    (8) Y = sum_g sx sw P_g + sT sL2 U (+ bias), float64.
+    """
+    X16 = np.asarray(X16, dtype=np.float16)
+    M, K = X16.shape
+    Wq, sw = layer["Wq"], layer["sw"]
+    N = Wq.shape[1]
+    G = -(-K // group)
+    branch, r = layer["branch"], int(layer["rank"])
+    out = {}
+    Xf = X16.astype(np.float32)
+
+    qx, sx = qgrp(Xf, group)                                   # (1)
+    out["qx"], out["sx"] = qx, sx
+
+    Y = np.zeros((M, N), dtype=np.float64)
+    Wq64 = Wq.astype(np.float64)
+    qx64 = qx.astype(np.float64)
+    for g in range(G):                                          # (6) + main part of (8)
+        k0, k1 = g * group, min(K, (g + 1) * group)
+        Pg = qx64[:, k0:k1] @ Wq64[k0:k1, :]                    # exact integers
+        Y += (sx[:, g].astype(np.float64)[:, None] * sw[g, :].astype(np.float64)[None, :]) * Pg
+
+    if branch != "none" and r > 0:
+        if branch == "w16a16":
+            # reference branch: fp16 operands, T rounded once to fp16, no scales
+            T = (X16.astype(np.float64) @ layer["L1h"].astype(np.float64)).astype(np.float16)
+            out["T16"] = T
+            Y += T.astype(np.float64) @ layer["L2h"].astype(np.float64)
+        else:
+            bw, ba = BRANCH_BITS[branch]
+            qb, sXb = qtok(Xf, ba)                              # (2)
+            I1 = qb.astype(np.float64) @ layer["L1q"].astype(np.float64)   # (3) exact
+            sc = (sXb[:, None] * layer["sL1"].astype(np.float32)[None, :]).astype(np.float32)
+            t = (I1.astype(np.float32) * sc).astype(np.float32)            # (4)
+            tq, sT = qtok(t, ba)                                # (5)
+            U = tq.astype(np.float64) @ layer["L2q"].astype(np.float64)    # (7) exact
+            Y += (sT.astype(np.float64)[:, None] * layer["sL2"].astype(np.float64)[None, :]) * U
+            out.update(qb=qb, sXb=sXb, I1=I1, t=t, tq=tq, sT=sT)
+    if layer.get("bias") is not None:
+        Y += layer["bias"].astype(np.float64)[None, :]
+    out["Y"] = Y
+    return out
+
+
+# --------------------------------------------------------------------------------------
+# Data-free calibration (Sections 3.2, 3.3; Appendix A, B.2)
+# --------------------------------------------------------------------------------------
+def svd_init(W, r: int):
+    """Best rank-r approximation M = L0 R0 of W (Eckart-Young), Sigma split evenly."""
+    U, s, Vt = np.linalg.svd(np.asarray(W, dtype=np.float64), full_matrices=False)
+    rs = np.sqrt(s[:r])
+    return U[:, :r] * rs[None, :], rs[:, None] * Vt[:r, :]
+
+
+def q1_dequant(A):
+    """Q1(A) as real numbers: SINT4 along K (axis 0) per output column, input rounded to fl32."""
+    c, s = q_weight_main(A)
+    return deq_weight_main(c, s)
+
+
+def residual_error(W, L, R):
+    """E = Q1(W + L R) - W - L R  (Eq. "low-rank-optimization")."""
+    D = L @ R
+    return q1_dequant(W + D) - W - D
+
+
+def objective(W, L, R) -> float:
+    """MSE form of the calibration objective: mean over K*N entries of E^2."""
+    E = residual_error(W, L, R)
+    return float(np.mean(E * E))
+
+
+def gradients(W, L, R):
+    """(loss, dL, dR) with the quantizer's derivative taken as zero (Appendix B.2):
+    d/d(LR) = -2 E / (K N),  dL = d(LR) R^T,  dR = L^T d(LR)."""
+    E = residual_error(W, L, R)
+    c = -2.0 / E.size
+    return float(np.mean(E * E)), c * (E @ R.T), c * (L.T @ E)
+
+
+def calibrate(W16, rank: int, branch: str = "w8a8", steps: int = 1000, lr: float = 1e-4,
+              beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, bias=None):
+    """Data-free calibration of one weight.  Returns (layer dict, trace [steps+1] of the
+    objective at every iterate visited, iterate 0 = the SVD initialisation)."""
+    W = np.asarray(W16, dtype=np.float16).astype(np.float64)
+    K, N = W.shape
+    layer = {"branch": branch, "rank": int(rank), "K": K, "N": N,
+             "bias": None if bias is None else np.asarray(bias, dtype=np.float16)}
+    if branch == "none" or rank == 0:
+        layer["branch"], layer["rank"] = "none", 0
+        layer["Wq"], layer["sw"] = q_weight_main(W)
+        E = q1_dequant(W) - W
+        return layer, np.array([float(np.mean(E * E))])
+
+    L0, R0 = svd_init(W, rank)
+    L, R = -L0, R0
+    mL = np.zeros_like(L); vL = np.zeros_like(L)
+    mR = np.zeros_like(R); vR = np.zeros_like(R)
+    trace = np.zeros(steps + 1)
+    best = (np.inf, None, None)
+    for t in range(steps + 1):
+        loss, gL, gR = gradients(W, L, R)
+        trace[t] = loss
+        if loss < best[0]:
+            best = (loss, L.copy(), R.copy())
+        if t == steps:
+            break
+        k = t + 1
+        mL = beta1 * mL + (1 - beta1) * gL; vL = beta2 * vL + (1 - beta2) * gL * gL
+        mR = beta1 * mR + (1 - beta1) * gR; vR = beta2 * vR + (1 - beta2) * gR * gR
+        c1, c2 = 1 - beta1 ** k, 1 - beta2 ** k
+        L = L - lr * (mL / c1) / (np.sqrt(vL / c2) + eps)
+        R = R - lr * (mR / c1) / (np.sqrt(vR / c2) + eps)
+
+    # Figure 1 sign: W ~ P + L1 L2 with L1 = -L*, L2 = R*
+    L1, L2 = -best[1], best[2]
+    bw, _ = BRANCH_BITS[branch]
+    if branch == "w16a16":
+        layer["L1h"], _ = q_factor(L1, None)
+        layer["L2h"], _ = q_factor(L2, None)
+        D = layer["L1h"].astype(np.float64) @ layer["L2h"].astype(np.float64)
+    else:
+        layer["L1q"], layer["sL1"] = q_factor(L1, bw)
+        layer["L2q"], layer["sL2"] = q_factor(L2, bw)
+        D = deq_factor(layer["L1q"], layer["sL1"]) @ deq_factor(layer["L2q"], layer["sL2"])
+    layer["Wq"], layer["sw"] = q_weight_main(W - D)       # P = W - Q2(L1) Q2(L2), then Q1
+    return layer, trace
+
+
+def effective_weight(layer):
+    """float64 [K, N]: deq(Q1(P)) + deq(Q2(L1)) deq(Q2(L2)) - what the layer multiplies by
+    when activations are exact."""
+    Wd = deq_weight_main(layer["Wq"], layer["sw"])
+    if layer["branch"] == "none" or layer["rank"] == 0:
+        return Wd
+    if layer["branch"] == "w16a16":
+        return Wd + layer["L1h"].astype(np.float64) @ layer["L2h"].astype(np.float64)
+    return Wd + deq_factor(layer["L1q"], layer["sL1"]) @ deq_factor(layer["L2q"], layer["sL2"])
