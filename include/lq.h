@@ -1,0 +1,163 @@
+/*
+ * lq.h - C ABI of the B200 (sm_100a) implementation of the LoRaQ fully quantized linear layer
+ *
+ *     Y = deq( Q4(X) * Q4(W - L1 L2) )  +  deq( Qb( Qb(X) * Qb(L1) ) * Qb(L2) )
+ *
+ * Notation follows the paper (Section 3.1): X in R^{m x d} activations, W in R^{d x n} weights,
+ * Y = X W.  Here M = m rows (tokens x batch), K = d input features, N = n output features,
+ * r = the rank of the low-rank branch, G = ceil(K / 64) groups.
+ *
+ * Every function returns an lq_status; nothing throws, aborts or prints.  "host" / "device"
+ * in a parameter comment says which address space the pointer lives in.  Device pointers and
+ * the stream belong to the caller (e.g. a torch tensor's data_ptr() and a torch stream's
+ * cuda_stream); everything behind lq_layer* / lq_act* is allocated and owned by the library
+ * and released by the matching _free call.  Calls that take a stream are asynchronous on it.
+ * There is no CPU fallback: without a CUDA device the device-side calls return LQ_ERR_CUDA.
+ */
+#ifndef LQ_H_
+#define LQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LQ_OK = 0,
+  LQ_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, handle/shape mismatch          */
+  LQ_ERR_UNSUPPORTED = 2, /* a size or format outside what the kernels are built for         */
+  LQ_ERR_ALLOC = 3,       /* host or device allocation failed                                 */
+  LQ_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed (or no device)                 */
+  LQ_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (see lq_get_device_status)    */
+  LQ_ERR_NUMERIC = 6      /* non-finite value met where the method needs finite ones          */
+} lq_status;
+
+/* Precision of the low-rank branch: bits of the two factors (W) and of the activations that
+ * enter it, incl. the rank-r intermediate (A).  Section 3.3 quantizes the branch with an
+ * operator Q2; the integer per-token / per-channel variants are this build's configurations. */
+typedef enum {
+  LQ_BRANCH_NONE = 0,   /* rank 0: plain W4A4                                  */
+  LQ_BRANCH_W16A16 = 1, /* fp16 factors, fp16 activations (reference variant)  */
+  LQ_BRANCH_W8A8 = 2,
+  LQ_BRANCH_W6A6 = 3,
+  LQ_BRANCH_W4A8 = 4
+} lq_branch_fmt;
+
+typedef enum { LQ_OUT_F16 = 0, LQ_OUT_F32 = 1 } lq_out_dtype;
+
+/* One layer's shape and calibration settings. */
+typedef struct {
+  int32_t K, N, rank; /* d, n and rho of Sections 3.1-3.2; rank in [0, 128], N even, K <= 8192    */
+  int32_t group;      /* 64: the SINT4 block of Appendix A.3 (the only supported value)           */
+  int32_t branch;     /* an lq_branch_fmt                                                         */
+  int32_t steps;      /* Adam steps on (L, R); 1000 in Appendix A "Optimization"                  */
+  float lr;           /* 1e-4 for integer formats (Appendix A)                                    */
+  float beta1, beta2, eps; /* Adam moments / epsilon; the paper is silent: 0.9, 0.999, 1e-8       */
+  int32_t rot_steps;  /* rotation steps of Section 3.3; must be 0 (rotation is not built)         */
+  float rot_lr;
+  uint64_t seed;      /* start vectors of the host SVD iteration                                  */
+} lq_config;
+
+typedef struct lq_layer lq_layer; /* opaque: Q1(P) codes+scales, Q2(L1), Q2(L2), bias (Figure 1)  */
+typedef struct lq_act lq_act;     /* opaque: device buffers holding one batch of quantized
+                                     activations for one layer shape (qx, sx, qb, sXb, tq, sT)   */
+
+/* Fill *cfg with the defaults above for the given shape. */
+lq_status lq_config_default(lq_config* cfg, int32_t K, int32_t N, int32_t rank, int32_t branch);
+
+/* Data-free calibration of one weight, entirely on the host (Sections 3.2-3.3, Appendix A,
+ * Appendix B.2): SVD initialisation L = -L0, R = R0; Adam on
+ * mean((Q1(W + L R) - W - L R)^2) with the quantizer's derivative taken as zero; the best
+ * iterate is kept; the factors are quantized with Q2; P = W - Q2(L1) Q2(L2) is quantized
+ * with Q1 (SINT4, groups of 64 along K per output column).
+ *   W_f16_host     [K][N] row-major IEEE half bits (the paper's d x n orientation), host
+ *   bias_f16_host  [N] half bits or NULL, host
+ *   out            receives a new layer (host copy only; see lq_layer_to_device)
+ *   objective_trace[steps + 1] doubles or NULL, host: objective at every iterate, [0] = init
+ * Errors: INVALID_ARG (null / bad shape), UNSUPPORTED (rot_steps != 0, group != 64, ...),
+ * NUMERIC (non-finite W), ALLOC. */
+lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W_f16_host,
+                       const uint16_t* bias_f16_host, lq_layer** out, double* objective_trace);
+
+/* Build a layer from already quantized parts (all host pointers, copied):
+ *   Wq_packed [K][N/2] bytes: codes in [-7,7] as two's-complement nibbles, column 2j in the
+ *             low nibble, column 2j+1 in the high nibble
+ *   sw        [G][N] half bits: SINT4 scale of group g of output column n
+ *   L1, L2    integer branches: int8 codes [K][rank] and [rank][N]; W16A16: half bits, same shapes
+ *   sL1, sL2  fp32 per-column scales [rank] and [N]; NULL for W16A16
+ *   bias      [N] half bits or NULL
+ * With rank == 0 or LQ_BRANCH_NONE the branch pointers are ignored. */
+lq_status lq_layer_import(const lq_config* cfg, const uint8_t* Wq_packed, const uint16_t* sw,
+                          const void* L1, const float* sL1, const void* L2, const float* sL2,
+                          const uint16_t* bias, lq_layer** out);
+
+/* Copy a layer's parts out into caller-sized host buffers (same layouts as lq_layer_import;
+ * any pointer may be NULL to skip that part). */
+lq_status lq_layer_export(const lq_layer* layer, uint8_t* Wq_packed, uint16_t* sw, void* L1,
+                          float* sL1, void* L2, float* sL2, uint16_t* bias);
+
+/* Shape of a layer handle. */
+lq_status lq_layer_info(const lq_layer* layer, lq_config* cfg_out);
+
+/* Upload the layer to `device` in the kernels' operand layout (allocates device memory;
+ * synchronous).  Must precede lq_act_create / lq_quantize_act / lq_linear_forward. */
+lq_status lq_layer_to_device(lq_layer* layer, int device);
+
+lq_status lq_layer_free(lq_layer* layer);
+
+/* Allocate the activation record for up to M_max rows of `layer`'s shape on `device`. */
+lq_status lq_act_create(const lq_layer* layer, int32_t M_max, int device, lq_act** out);
+lq_status lq_act_free(lq_act* act);
+
+/* Dynamic activation quantization fused with the branch's down-projection (Figure 1;
+ * Appendix A.2 "Quantization": the activations forwarded to both branches are quantized).
+ * One read of X produces
+ *   qx, sx   SINT4 codes / fp16 scales per token and group of 64 along K (Appendix A.3)
+ *   qb, sXb  per-token branch codes / fp32 scale
+ *   tq, sT   per-token codes / scale of the rank-r intermediate T = deq(qb) deq(L1)
+ *   X_f16_dev  [M][K] row-major half, device, 16-byte aligned
+ *   M          1 <= M <= M_max of `out`
+ * Asynchronous on `cuda_stream` (a cudaStream_t). */
+lq_status lq_quantize_act(const lq_layer* layer, const void* X_f16_dev, int32_t M, lq_act* out,
+                          void* cuda_stream);
+
+/* Y = sum_g sx sw (qx_g Wq_g) + sT sL2 (tq L2q) + bias: the 4-bit main product per group on
+ * the tensor cores, per-group scales and the branch's up-projection applied in one epilogue
+ * (Figure 1; Section 3.3).
+ *   act    result of lq_quantize_act for this layer
+ *   Y_dev  [M][N] row-major, half or float per `dtype`, device, 16-byte aligned
+ * Asynchronous on `cuda_stream`. */
+lq_status lq_linear_forward(const lq_layer* layer, const lq_act* act, void* Y_dev,
+                            lq_out_dtype dtype, void* cuda_stream);
+
+/* Whole path from host memory: copies X to the device, runs lq_quantize_act and
+ * lq_linear_forward, copies Y back and waits for it.  X_f16_host [M][K], Y_host [M][N];
+ * pinned host memory makes the copies asynchronous but is not required.  Staging buffers
+ * inside `act` are allocated on the first call. */
+lq_status lq_linear_forward_host(const lq_layer* layer, lq_act* act, const void* X_f16_host,
+                                 int32_t M, void* Y_host, lq_out_dtype dtype, void* cuda_stream);
+
+/* Decode the activation record of the last lq_quantize_act into plain host arrays (for
+ * parity checks); NULL skips a part.  qx int8 [M][K], sx half bits [M][G], qb int8 [M][K],
+ * sXb float [M], tq int8 [M][rank] (W16A16: half bits [M][rank]), sT float [M].
+ * Synchronises `cuda_stream`. */
+lq_status lq_act_export(const lq_act* act, int8_t* qx, uint16_t* sx, int8_t* qb, float* sXb,
+                        void* tq, float* sT, void* cuda_stream);
+
+/* Status word the kernels write when a bounded wait expires: code is an lq_status
+ * (LQ_OK if none), stage identifies the waiting role.  Reading clears it.  Synchronises
+ * the device. */
+lq_status lq_get_device_status(int device, int32_t* code, int32_t* stage);
+
+/* Tuning knobs for experiments, e.g. "main_kind" (0 = int8 operands, 1 = E4M3-carried
+ * codes).  Returns INVALID_ARG for an unknown name.  Affects layers uploaded afterwards. */
+lq_status lq_set_option(const char* name, int32_t value);
+
+const char* lq_status_string(lq_status s);
+int lq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LQ_H_ */

@@ -1,0 +1,460 @@
+// Handles, import/export, device upload and the host-side plumbing of the C ABI.
+#include <cuda_fp16.h>
+#include <math.h>
+#include <string.h>
+
+#include <mutex>
+#include <new>
+
+#include "lq_internal.h"
+
+int g_lq_main_kind = LQ_KIND_E4M3;
+int g_lq_gemm_ctas = 0;
+
+#define CUDA_OK(expr)                         \
+  do {                                        \
+    cudaError_t e__ = (expr);                 \
+    if (e__ != cudaSuccess) return LQ_ERR_CUDA; \
+  } while (0)
+
+static inline float h2f(uint16_t h) {
+  __half_raw r; r.x = h;
+  return __half2float(__half(r));
+}
+
+extern "C" const char* lq_status_string(lq_status s) {
+  switch (s) {
+    case LQ_OK: return "ok";
+    case LQ_ERR_INVALID_ARG: return "invalid argument";
+    case LQ_ERR_UNSUPPORTED: return "unsupported size or format";
+    case LQ_ERR_ALLOC: return "allocation failed";
+    case LQ_ERR_CUDA: return "CUDA call failed";
+    case LQ_ERR_TIMEOUT: return "bounded device wait expired";
+    case LQ_ERR_NUMERIC: return "non-finite value";
+  }
+  return "unknown status";
+}
+
+extern "C" int lq_version(void) { return 100; }
+
+extern "C" lq_status lq_set_option(const char* name, int32_t value) {
+  if (!name) return LQ_ERR_INVALID_ARG;
+  if (!strcmp(name, "main_kind")) {
+    if (value != LQ_KIND_I8 && value != LQ_KIND_E4M3) return LQ_ERR_INVALID_ARG;
+    g_lq_main_kind = value;
+    return LQ_OK;
+  }
+  if (!strcmp(name, "gemm_ctas")) {
+    if (value < 0) return LQ_ERR_INVALID_ARG;
+    g_lq_gemm_ctas = value;
+    return LQ_OK;
+  }
+  return LQ_ERR_INVALID_ARG;
+}
+
+extern "C" lq_status lq_config_default(lq_config* cfg, int32_t K, int32_t N, int32_t rank, int32_t branch) {
+  if (!cfg) return LQ_ERR_INVALID_ARG;
+  memset(cfg, 0, sizeof(*cfg));
+  cfg->K = K; cfg->N = N; cfg->rank = rank; cfg->group = LQ_GROUP; cfg->branch = branch;
+  cfg->steps = 1000; cfg->lr = 1e-4f; cfg->beta1 = 0.9f; cfg->beta2 = 0.999f; cfg->eps = 1e-8f;
+  cfg->rot_steps = 0; cfg->rot_lr = 0.5f; cfg->seed = 0;
+  return LQ_OK;
+}
+
+static lq_status check_config(const lq_config* c) {
+  if (!c) return LQ_ERR_INVALID_ARG;
+  if (c->K <= 0 || c->N <= 0 || c->rank < 0) return LQ_ERR_INVALID_ARG;
+  if (c->branch < LQ_BRANCH_NONE || c->branch > LQ_BRANCH_W4A8) return LQ_ERR_INVALID_ARG;
+  if (c->group != LQ_GROUP) return LQ_ERR_UNSUPPORTED;
+  if (c->K > LQ_MAX_K || (c->K % 8) != 0) return LQ_ERR_UNSUPPORTED;
+  if ((c->N % 8) != 0) return LQ_ERR_UNSUPPORTED;
+  if (c->rank > LQ_MAX_RANK) return LQ_ERR_UNSUPPORTED;
+  if (c->branch == LQ_BRANCH_W16A16 && c->rank > 64) return LQ_ERR_UNSUPPORTED;
+  if (c->rot_steps != 0) return LQ_ERR_UNSUPPORTED;
+  return LQ_OK;
+}
+
+// Shared by lq_layer_import and lq_calibrate: an empty layer with sizes filled in.
+lq_layer* lq_layer_new(const lq_config* cfg) {
+  lq_layer* L = new (std::nothrow) lq_layer();
+  if (!L) return nullptr;
+  L->cfg = *cfg;
+  L->K = cfg->K; L->N = cfg->N;
+  L->r = (cfg->branch == LQ_BRANCH_NONE) ? 0 : cfg->rank;
+  if (L->r == 0) L->cfg.branch = LQ_BRANCH_NONE;
+  L->cfg.rank = L->r;
+  L->G = lq_ceil_div(L->K, LQ_GROUP);
+  L->Kpad = lq_round_up(L->K, LQ_KSTAGE);
+  L->Gpad = L->Kpad / LQ_GROUP;
+  L->Npad = lq_round_up(L->N, LQ_BN);
+  L->integer_branch = L->r > 0 && L->cfg.branch != LQ_BRANCH_W16A16;
+  L->f16_branch = L->r > 0 && L->cfg.branch == LQ_BRANCH_W16A16;
+  L->has_bias = false;
+  L->device = -1;
+  L->main_kind = g_lq_main_kind;
+  L->d_Wq8 = nullptr; L->d_sw = nullptr; L->d_L1t = nullptr; L->d_L1h = nullptr; L->d_sL1 = nullptr;
+  L->d_L2c = nullptr; L->d_sL2 = nullptr; L->d_bias = nullptr;
+  return L;
+}
+
+extern "C" lq_status lq_layer_import(const lq_config* cfg, const uint8_t* Wq_packed, const uint16_t* sw,
+                                     const void* L1, const float* sL1, const void* L2, const float* sL2,
+                                     const uint16_t* bias, lq_layer** out) {
+  lq_status st = check_config(cfg);
+  if (st != LQ_OK) return st;
+  if (!Wq_packed || !sw || !out) return LQ_ERR_INVALID_ARG;
+  lq_layer* L = lq_layer_new(cfg);
+  if (!L) return LQ_ERR_ALLOC;
+  const int K = L->K, N = L->N, r = L->r, G = L->G;
+  if (r > 0 && (!L1 || !L2)) { delete L; return LQ_ERR_INVALID_ARG; }
+  if (L->integer_branch && (!sL1 || !sL2)) { delete L; return LQ_ERR_INVALID_ARG; }
+  try {
+    L->Wq.resize((size_t)K * N);
+    for (int k = 0; k < K; ++k)
+      for (int j = 0; j < N / 2; ++j) {
+        uint8_t b = Wq_packed[(size_t)k * (N / 2) + j];
+        int lo = (int)(b & 0xF), hi = (int)(b >> 4);
+        lo = lo >= 8 ? lo - 16 : lo; hi = hi >= 8 ? hi - 16 : hi;
+        if (lo < -7 || hi < -7) { delete L; return LQ_ERR_INVALID_ARG; }
+        L->Wq[(size_t)k * N + 2 * j] = (int8_t)lo;
+        L->Wq[(size_t)k * N + 2 * j + 1] = (int8_t)hi;
+      }
+    L->sw.assign(sw, sw + (size_t)G * N);
+    for (size_t i = 0; i < L->sw.size(); ++i)
+      if (!isfinite(h2f(L->sw[i]))) { delete L; return LQ_ERR_NUMERIC; }
+    if (L->integer_branch) {
+      const int qm = (1 << (lq_branch_wbits(L->cfg.branch) - 1)) - 1;
+      const int8_t* a = (const int8_t*)L1; const int8_t* b = (const int8_t*)L2;
+      L->L1q.assign(a, a + (size_t)K * r);
+      L->L2q.assign(b, b + (size_t)r * N);
+      for (int8_t v : L->L1q) if (v > qm || v < -qm) { delete L; return LQ_ERR_INVALID_ARG; }
+      for (int8_t v : L->L2q) if (v > qm || v < -qm) { delete L; return LQ_ERR_INVALID_ARG; }
+      L->sL1.assign(sL1, sL1 + r);
+      L->sL2.assign(sL2, sL2 + N);
+      for (float v : L->sL1) if (!isfinite(v)) { delete L; return LQ_ERR_NUMERIC; }
+      for (float v : L->sL2) if (!isfinite(v)) { delete L; return LQ_ERR_NUMERIC; }
+    } else if (L->f16_branch) {
+      const uint16_t* a = (const uint16_t*)L1; const uint16_t* b = (const uint16_t*)L2;
+      L->L1h.assign(a, a + (size_t)K * r);
+      L->L2h.assign(b, b + (size_t)r * N);
+    }
+    if (bias) { L->bias.assign(bias, bias + N); L->has_bias = true; }
+  } catch (const std::bad_alloc&) { delete L; return LQ_ERR_ALLOC; }
+  *out = L;
+  return LQ_OK;
+}
+
+extern "C" lq_status lq_layer_export(const lq_layer* L, uint8_t* Wq_packed, uint16_t* sw, void* L1,
+                                     float* sL1, void* L2, float* sL2, uint16_t* bias) {
+  if (!L) return LQ_ERR_INVALID_ARG;
+  const int K = L->K, N = L->N, r = L->r;
+  if (Wq_packed)
+    for (int k = 0; k < K; ++k)
+      for (int j = 0; j < N / 2; ++j) {
+        int lo = L->Wq[(size_t)k * N + 2 * j], hi = L->Wq[(size_t)k * N + 2 * j + 1];
+        Wq_packed[(size_t)k * (N / 2) + j] = (uint8_t)((lo & 0xF) | ((hi & 0xF) << 4));
+      }
+  if (sw) memcpy(sw, L->sw.data(), L->sw.size() * sizeof(uint16_t));
+  if (L->integer_branch) {
+    if (L1) memcpy(L1, L->L1q.data(), (size_t)K * r);
+    if (L2) memcpy(L2, L->L2q.data(), (size_t)r * N);
+    if (sL1) memcpy(sL1, L->sL1.data(), r * sizeof(float));
+    if (sL2) memcpy(sL2, L->sL2.data(), N * sizeof(float));
+  } else if (L->f16_branch) {
+    if (L1) memcpy(L1, L->L1h.data(), (size_t)K * r * 2);
+    if (L2) memcpy(L2, L->L2h.data(), (size_t)r * N * 2);
+  }
+  if (bias && L->has_bias) memcpy(bias, L->bias.data(), N * sizeof(uint16_t));
+  return LQ_OK;
+}
+
+extern "C" lq_status lq_layer_info(const lq_layer* L, lq_config* cfg_out) {
+  if (!L || !cfg_out) return LQ_ERR_INVALID_ARG;
+  *cfg_out = L->cfg;
+  return LQ_OK;
+}
+
+// ---- TMA descriptors ---------------------------------------------------------------------
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static encode_tiled_fn get_encode_fn() {
+  static encode_tiled_fn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (encode_tiled_fn)p;
+  });
+  return fn;
+}
+
+// 2-D byte tensor [rows][row_bytes], box [box_rows][128 bytes], 128-byte swizzle.
+static lq_status make_tmap_bytes(CUtensorMap* tm, void* base, uint64_t rows, uint64_t row_bytes, uint32_t box_rows) {
+  encode_tiled_fn fn = get_encode_fn();
+  if (!fn) return LQ_ERR_CUDA;
+  cuuint64_t dims[2] = {row_bytes, rows};
+  cuuint64_t strides[1] = {row_bytes};
+  cuuint32_t box[2] = {128, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? LQ_OK : LQ_ERR_CUDA;
+}
+
+// ---- device status word ------------------------------------------------------------------
+static int32_t* g_status[64] = {nullptr};
+static std::mutex g_status_mu;
+
+int32_t* lq_device_status_ptr(int device) {
+  if (device < 0 || device >= 64) return nullptr;
+  std::lock_guard<std::mutex> lk(g_status_mu);
+  if (!g_status[device]) {
+    int prev = 0;
+    cudaGetDevice(&prev);
+    if (cudaSetDevice(device) != cudaSuccess) return nullptr;
+    int32_t* p = nullptr;
+    if (cudaMalloc(&p, 2 * sizeof(int32_t)) != cudaSuccess) { cudaSetDevice(prev); return nullptr; }
+    cudaMemset(p, 0, 2 * sizeof(int32_t));
+    g_status[device] = p;
+    cudaSetDevice(prev);
+  }
+  return g_status[device];
+}
+
+extern "C" lq_status lq_get_device_status(int device, int32_t* code, int32_t* stage) {
+  int32_t* p = lq_device_status_ptr(device);
+  if (!p) return LQ_ERR_CUDA;
+  int32_t h[2] = {0, 0};
+  CUDA_OK(cudaSetDevice(device));
+  CUDA_OK(cudaDeviceSynchronize());
+  CUDA_OK(cudaMemcpy(h, p, sizeof(h), cudaMemcpyDeviceToHost));
+  CUDA_OK(cudaMemset(p, 0, sizeof(h)));
+  if (code) *code = h[0];
+  if (stage) *stage = h[1];
+  return LQ_OK;
+}
+
+// ---- upload ------------------------------------------------------------------------------
+static void layer_free_device(lq_layer* L) {
+  if (L->device < 0) return;
+  cudaSetDevice(L->device);
+  cudaFree(L->d_Wq8); cudaFree(L->d_sw); cudaFree(L->d_L1t); cudaFree(L->d_L1h); cudaFree(L->d_sL1);
+  cudaFree(L->d_L2c); cudaFree(L->d_sL2); cudaFree(L->d_bias);
+  L->d_Wq8 = nullptr; L->d_sw = nullptr; L->d_L1t = nullptr; L->d_L1h = nullptr; L->d_sL1 = nullptr;
+  L->d_L2c = nullptr; L->d_sL2 = nullptr; L->d_bias = nullptr;
+  L->device = -1;
+}
+
+template <typename T>
+static lq_status upload(T** dptr, const std::vector<T>& h) {
+  if (cudaMalloc((void**)dptr, h.size() * sizeof(T)) != cudaSuccess) return LQ_ERR_ALLOC;
+  CUDA_OK(cudaMemcpy(*dptr, h.data(), h.size() * sizeof(T), cudaMemcpyHostToDevice));
+  return LQ_OK;
+}
+
+extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
+  if (!L) return LQ_ERR_INVALID_ARG;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) return LQ_ERR_CUDA;
+  layer_free_device(L);
+  CUDA_OK(cudaSetDevice(device));
+  L->device = device;
+  L->main_kind = g_lq_main_kind;
+  const int K = L->K, N = L->N, r = L->r, G = L->G, Kpad = L->Kpad, Npad = L->Npad, Gpad = L->Gpad;
+  lq_status st;
+  try {
+    std::vector<uint8_t> w8((size_t)Npad * Kpad, lq_encode_code_host(0, L->main_kind));
+    for (int k = 0; k < K; ++k)
+      for (int n = 0; n < N; ++n) w8[(size_t)n * Kpad + k] = lq_encode_code_host(L->Wq[(size_t)k * N + n], L->main_kind);
+    if ((st = upload(&L->d_Wq8, w8)) != LQ_OK) return st;
+    std::vector<float> swf((size_t)Gpad * Npad, 0.f);
+    for (int g = 0; g < G; ++g)
+      for (int n = 0; n < N; ++n) swf[(size_t)g * Npad + n] = h2f(L->sw[(size_t)g * N + n]);
+    if ((st = upload(&L->d_sw, swf)) != LQ_OK) return st;
+    std::vector<float> bias((size_t)Npad, 0.f);
+    if (L->has_bias) for (int n = 0; n < N; ++n) bias[n] = h2f(L->bias[n]);
+    if ((st = upload(&L->d_bias, bias)) != LQ_OK) return st;
+    std::vector<float> s1(LQ_MAX_RANK, 1.f), s2((size_t)Npad, 1.f);
+    std::vector<uint8_t> l2c((size_t)Npad * LQ_RCONT, 0);
+    if (L->integer_branch) {
+      std::vector<int8_t> l1t((size_t)r * Kpad, 0);
+      for (int k = 0; k < K; ++k)
+        for (int j = 0; j < r; ++j) l1t[(size_t)j * Kpad + k] = L->L1q[(size_t)k * r + j];
+      if ((st = upload(&L->d_L1t, l1t)) != LQ_OK) return st;
+      for (int j = 0; j < r; ++j) s1[j] = L->sL1[j];
+      for (int n = 0; n < N; ++n) s2[n] = L->sL2[n];
+      for (int j = 0; j < r; ++j)
+        for (int n = 0; n < N; ++n) l2c[(size_t)n * LQ_RCONT + j] = (uint8_t)L->L2q[(size_t)j * N + n];
+    } else if (L->f16_branch) {
+      std::vector<uint16_t> l1t((size_t)r * Kpad, 0);
+      for (int k = 0; k < K; ++k)
+        for (int j = 0; j < r; ++j) l1t[(size_t)j * Kpad + k] = L->L1h[(size_t)k * r + j];
+      if ((st = upload(&L->d_L1h, l1t)) != LQ_OK) return st;
+      uint16_t* c16 = (uint16_t*)l2c.data();
+      for (int j = 0; j < r; ++j)
+        for (int n = 0; n < N; ++n) c16[(size_t)n * (LQ_RCONT / 2) + j] = L->L2h[(size_t)j * N + n];
+    }
+    if ((st = upload(&L->d_sL1, s1)) != LQ_OK) return st;
+    if ((st = upload(&L->d_sL2, s2)) != LQ_OK) return st;
+    if ((st = upload(&L->d_L2c, l2c)) != LQ_OK) return st;
+  } catch (const std::bad_alloc&) { return LQ_ERR_ALLOC; }
+  if ((st = make_tmap_bytes(&L->tmB, L->d_Wq8, Npad, Kpad, LQ_BN)) != LQ_OK) return st;
+  if ((st = make_tmap_bytes(&L->tmL2, L->d_L2c, Npad, LQ_RCONT, LQ_BN)) != LQ_OK) return st;
+  if (!lq_device_status_ptr(device)) return LQ_ERR_CUDA;
+  if ((st = lq_gemm_prepare(device)) != LQ_OK) return st;
+  return LQ_OK;
+}
+
+extern "C" lq_status lq_layer_free(lq_layer* L) {
+  if (!L) return LQ_ERR_INVALID_ARG;
+  layer_free_device(L);
+  delete L;
+  return LQ_OK;
+}
+
+// ---- activation record -------------------------------------------------------------------
+extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device, lq_act** out) {
+  if (!L || !out || M_max <= 0) return LQ_ERR_INVALID_ARG;
+  if (L->device != device) return LQ_ERR_INVALID_ARG;
+  lq_act* A = new (std::nothrow) lq_act();
+  if (!A) return LQ_ERR_ALLOC;
+  memset(A, 0, sizeof(*A));
+  A->K = L->K; A->N = L->N; A->r = L->r; A->G = L->G; A->Kpad = L->Kpad; A->Gpad = L->Gpad;
+  A->branch = L->cfg.branch; A->M_max = M_max; A->Mpad = lq_round_up(M_max, LQ_BM);
+  A->device = device; A->main_kind = L->main_kind; A->M = 0;
+  if (cudaSetDevice(device) != cudaSuccess) { delete A; return LQ_ERR_CUDA; }
+  const size_t Mp = A->Mpad, Kp = A->Kpad;
+  bool ok = cudaMalloc((void**)&A->d_qx8, Mp * Kp) == cudaSuccess &&
+            cudaMalloc((void**)&A->d_sx, (size_t)A->Gpad * Mp * sizeof(float)) == cudaSuccess &&
+            cudaMalloc((void**)&A->d_qb, Mp * Kp) == cudaSuccess &&
+            cudaMalloc((void**)&A->d_sXb, Mp * sizeof(float)) == cudaSuccess &&
+            cudaMalloc((void**)&A->d_tq, Mp * LQ_RCONT) == cudaSuccess &&
+            cudaMalloc((void**)&A->d_sT, Mp * sizeof(float)) == cudaSuccess;
+  if (!ok) { lq_act_free(A); return LQ_ERR_ALLOC; }
+  // padding rows/columns are read by the GEMM's tiles: start from defined contents
+  cudaMemset(A->d_qx8, 0, Mp * Kp);
+  cudaMemset(A->d_sx, 0, (size_t)A->Gpad * Mp * sizeof(float));
+  cudaMemset(A->d_qb, 0, Mp * Kp);
+  cudaMemset(A->d_sXb, 0, Mp * sizeof(float));
+  cudaMemset(A->d_tq, 0, Mp * LQ_RCONT);
+  cudaMemset(A->d_sT, 0, Mp * sizeof(float));
+  lq_status st;
+  if ((st = make_tmap_bytes(&A->tmA, A->d_qx8, Mp, Kp, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
+  if ((st = make_tmap_bytes(&A->tmT, A->d_tq, Mp, LQ_RCONT, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
+  if (cudaDeviceSynchronize() != cudaSuccess) { lq_act_free(A); return LQ_ERR_CUDA; }
+  *out = A;
+  return LQ_OK;
+}
+
+extern "C" lq_status lq_act_free(lq_act* A) {
+  if (!A) return LQ_ERR_INVALID_ARG;
+  cudaSetDevice(A->device);
+  cudaFree(A->d_qx8); cudaFree(A->d_sx); cudaFree(A->d_qb); cudaFree(A->d_sXb); cudaFree(A->d_tq); cudaFree(A->d_sT);
+  cudaFree(A->d_Xstage); cudaFree(A->d_Ystage);
+  delete A;
+  return LQ_OK;
+}
+
+static bool act_matches(const lq_layer* L, const lq_act* A) {
+  return L && A && L->device == A->device && L->device >= 0 && L->K == A->K && L->N == A->N && L->r == A->r &&
+         L->cfg.branch == A->branch && L->main_kind == A->main_kind;
+}
+
+extern "C" lq_status lq_quantize_act(const lq_layer* L, const void* X, int32_t M, lq_act* A, void* stream) {
+  if (!L || !A || !X) return LQ_ERR_INVALID_ARG;
+  if (!act_matches(L, A)) return LQ_ERR_INVALID_ARG;
+  if (M <= 0 || M > A->M_max) return LQ_ERR_INVALID_ARG;
+  if (((uintptr_t)X & 15) != 0) return LQ_ERR_INVALID_ARG;
+  A->M = M;
+  return lq_launch_quantize(L, X, M, A, (cudaStream_t)stream);
+}
+
+extern "C" lq_status lq_linear_forward(const lq_layer* L, const lq_act* A, void* Y, lq_out_dtype dt, void* stream) {
+  if (!L || !A || !Y) return LQ_ERR_INVALID_ARG;
+  if (!act_matches(L, A)) return LQ_ERR_INVALID_ARG;
+  if (A->M <= 0) return LQ_ERR_INVALID_ARG;
+  if (dt != LQ_OUT_F16 && dt != LQ_OUT_F32) return LQ_ERR_INVALID_ARG;
+  if (((uintptr_t)Y & 15) != 0) return LQ_ERR_INVALID_ARG;
+  return lq_launch_gemm(L, A, Y, dt, (cudaStream_t)stream);
+}
+
+extern "C" lq_status lq_linear_forward_host(const lq_layer* L, lq_act* A, const void* Xh, int32_t M, void* Yh,
+                                            lq_out_dtype dt, void* stream) {
+  if (!L || !A || !Xh || !Yh) return LQ_ERR_INVALID_ARG;
+  if (!act_matches(L, A)) return LQ_ERR_INVALID_ARG;
+  if (M <= 0 || M > A->M_max) return LQ_ERR_INVALID_ARG;
+  if (dt != LQ_OUT_F16 && dt != LQ_OUT_F32) return LQ_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  CUDA_OK(cudaSetDevice(A->device));
+  if (!A->d_Xstage && cudaMalloc(&A->d_Xstage, (size_t)A->M_max * A->K * 2) != cudaSuccess) return LQ_ERR_ALLOC;
+  const size_t ybytes = (size_t)A->M_max * A->N * (dt == LQ_OUT_F32 ? 4 : 2);
+  if (A->ystage_bytes < ybytes) {
+    cudaFree(A->d_Ystage); A->d_Ystage = nullptr; A->ystage_bytes = 0;
+    if (cudaMalloc(&A->d_Ystage, ybytes) != cudaSuccess) return LQ_ERR_ALLOC;
+    A->ystage_bytes = ybytes;
+  }
+  CUDA_OK(cudaMemcpyAsync(A->d_Xstage, Xh, (size_t)M * A->K * 2, cudaMemcpyHostToDevice, st));
+  lq_status s = lq_quantize_act(L, A->d_Xstage, M, A, stream);
+  if (s != LQ_OK) return s;
+  s = lq_linear_forward(L, A, A->d_Ystage, dt, stream);
+  if (s != LQ_OK) return s;
+  CUDA_OK(cudaMemcpyAsync(Yh, A->d_Ystage, (size_t)M * A->N * (dt == LQ_OUT_F32 ? 4 : 2), cudaMemcpyDeviceToHost, st));
+  CUDA_OK(cudaStreamSynchronize(st));
+  return LQ_OK;
+}
+
+static int decode_code(uint8_t b, int kind) {
+  if (kind == LQ_KIND_I8) return (int)(int8_t)b;
+  int mag = 0;
+  switch (b & 0x7F) {
+    case 0x00: mag = 0; break; case 0x38: mag = 1; break; case 0x40: mag = 2; break; case 0x44: mag = 3; break;
+    case 0x48: mag = 4; break; case 0x4A: mag = 5; break; case 0x4C: mag = 6; break; case 0x4E: mag = 7; break;
+    default: mag = 99; break;   // not a code byte: surfaces as a parity failure
+  }
+  return (b & 0x80) ? -mag : mag;
+}
+
+extern "C" lq_status lq_act_export(const lq_act* A, int8_t* qx, uint16_t* sx, int8_t* qb, float* sXb, void* tq,
+                                   float* sT, void* stream) {
+  if (!A || A->M <= 0) return LQ_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  CUDA_OK(cudaSetDevice(A->device));
+  CUDA_OK(cudaStreamSynchronize(st));
+  const int M = A->M, K = A->K, G = A->G, r = A->r;
+  const size_t Kp = A->Kpad, Mp = A->Mpad;
+  try {
+    if (qx) {
+      std::vector<uint8_t> h((size_t)M * Kp);
+      CUDA_OK(cudaMemcpy(h.data(), A->d_qx8, h.size(), cudaMemcpyDeviceToHost));
+      for (int m = 0; m < M; ++m)
+        for (int k = 0; k < K; ++k) qx[(size_t)m * K + k] = (int8_t)decode_code(h[m * Kp + k], A->main_kind);
+    }
+    if (sx) {
+      std::vector<float> h((size_t)A->Gpad * Mp);
+      CUDA_OK(cudaMemcpy(h.data(), A->d_sx, h.size() * sizeof(float), cudaMemcpyDeviceToHost));
+      for (int m = 0; m < M; ++m)
+        for (int g = 0; g < G; ++g) {
+          __half v = __float2half_rn(h[(size_t)g * Mp + m]);   // exact: the value is an fp16 number
+          sx[(size_t)m * G + g] = __half_raw(v).x;
+        }
+    }
+    if (qb && A->branch != LQ_BRANCH_NONE && A->branch != LQ_BRANCH_W16A16) {
+      std::vector<int8_t> h((size_t)M * Kp);
+      CUDA_OK(cudaMemcpy(h.data(), A->d_qb, h.size(), cudaMemcpyDeviceToHost));
+      for (int m = 0; m < M; ++m) memcpy(qb + (size_t)m * K, h.data() + m * Kp, K);
+    }
+    if (sXb && r > 0) CUDA_OK(cudaMemcpy(sXb, A->d_sXb, M * sizeof(float), cudaMemcpyDeviceToHost));
+    if (tq && r > 0) {
+      std::vector<uint8_t> h((size_t)M * LQ_RCONT);
+      CUDA_OK(cudaMemcpy(h.data(), A->d_tq, h.size(), cudaMemcpyDeviceToHost));
+      const int eb = A->branch == LQ_BRANCH_W16A16 ? 2 : 1;
+      for (int m = 0; m < M; ++m) memcpy((uint8_t*)tq + (size_t)m * r * eb, h.data() + (size_t)m * LQ_RCONT, (size_t)r * eb);
+    }
+    if (sT && r > 0) CUDA_OK(cudaMemcpy(sT, A->d_sT, M * sizeof(float), cudaMemcpyDeviceToHost));
+  } catch (const std::bad_alloc&) { return LQ_ERR_ALLOC; }
+  return LQ_OK;
+}

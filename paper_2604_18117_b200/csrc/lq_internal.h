@@ -1,0 +1,98 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "lq.h"
+
+#define LQ_GROUP 64
+#define LQ_BM 128            // rows per output tile (one tcgen05 MMA, M = 128)
+#define LQ_BN 128            // columns per output tile
+#define LQ_KSTAGE 128        // bytes of K per shared-memory stage row (two groups of 64 codes)
+#define LQ_RCONT 128         // bytes per row of the branch containers (tq, L2q): rank <= 128
+#define LQ_MAX_K 8192
+#define LQ_MAX_RANK 128
+
+// role identifiers reported through the device status word
+enum { LQ_STAGE_NONE = 0, LQ_STAGE_PRODUCER = 1, LQ_STAGE_MMA = 2, LQ_STAGE_DRAIN = 3, LQ_STAGE_TEARDOWN = 4 };
+
+enum { LQ_KIND_I8 = 0, LQ_KIND_E4M3 = 1 };
+
+static inline int lq_ceil_div(int a, int b) { return (a + b - 1) / b; }
+static inline int lq_round_up(int a, int b) { return lq_ceil_div(a, b) * b; }
+
+static inline int lq_branch_wbits(int branch) {
+  return branch == LQ_BRANCH_W8A8 ? 8 : branch == LQ_BRANCH_W6A6 ? 6 : branch == LQ_BRANCH_W4A8 ? 4 : 0;
+}
+static inline int lq_branch_abits(int branch) {
+  return branch == LQ_BRANCH_W8A8 ? 8 : branch == LQ_BRANCH_W6A6 ? 6 : branch == LQ_BRANCH_W4A8 ? 8 : 0;
+}
+
+struct lq_layer {
+  lq_config cfg;
+  int K, N, r, G;          // logical sizes
+  int Kpad, Npad, Gpad;    // Kpad: multiple of 128; Npad: multiple of LQ_BN; Gpad = Kpad / 64
+  bool integer_branch, f16_branch, has_bias;
+  // host copy, canonical layouts
+  std::vector<int8_t> Wq;      // [K][N]
+  std::vector<uint16_t> sw;    // [G][N] half bits
+  std::vector<int8_t> L1q;     // [K][r]
+  std::vector<int8_t> L2q;     // [r][N]
+  std::vector<float> sL1, sL2; // [r], [N]
+  std::vector<uint16_t> L1h;   // [K][r] half bits (W16A16)
+  std::vector<uint16_t> L2h;   // [r][N]
+  std::vector<uint16_t> bias;  // [N]
+  // device copy, operand layouts
+  int device;
+  int main_kind;               // LQ_KIND_*: byte encoding of the 4-bit codes in the MMA operands
+  uint8_t* d_Wq8;              // [Npad][Kpad] bytes, K contiguous (B operand, K-major)
+  float* d_sw;                 // [Gpad][Npad] fp32 (exact images of the fp16 scales)
+  int8_t* d_L1t;               // [r][Kpad] int8, K contiguous   (integer branches)
+  uint16_t* d_L1h;             // [r][Kpad] half, K contiguous   (W16A16)
+  float* d_sL1;                // [LQ_MAX_RANK]
+  uint8_t* d_L2c;              // [Npad][LQ_RCONT] bytes: int8 codes (or up to 64 halves) of column n, r contiguous
+  float* d_sL2;                // [Npad]  (ones for W16A16)
+  float* d_bias;               // [Npad]  (zeros without bias)
+  CUtensorMap tmB;             // over d_Wq8, box [LQ_BN][128B], 128B swizzle
+  CUtensorMap tmL2;            // over d_L2c, box [LQ_BN][128B], 128B swizzle
+};
+
+struct lq_act {
+  int K, N, r, G, Kpad, Gpad, branch;
+  int M_max, Mpad, device, main_kind;
+  int M;                       // rows of the last lq_quantize_act
+  uint8_t* d_qx8;              // [Mpad][Kpad] operand bytes of the 4-bit codes (A operand, K-major)
+  float* d_sx;                 // [Gpad][Mpad] fp32 images of the fp16 scales
+  int8_t* d_qb;                // [Mpad][Kpad] branch activation codes
+  float* d_sXb;                // [Mpad]
+  uint8_t* d_tq;               // [Mpad][LQ_RCONT] bytes: int8 codes (or halves) of T, r contiguous
+  float* d_sT;                 // [Mpad] (ones for W16A16)
+  void* d_Xstage;              // lazily allocated staging for lq_linear_forward_host
+  void* d_Ystage;
+  size_t ystage_bytes;
+  CUtensorMap tmA;             // over d_qx8, box [LQ_BM][128B], 128B swizzle
+  CUtensorMap tmT;             // over d_tq,  box [LQ_BM][128B], 128B swizzle
+};
+
+// device status word (one per device, allocated on first use): {code, stage}
+int32_t* lq_device_status_ptr(int device);
+
+// kernels' host launchers (defined in lq_quant.cu / lq_gemm.cu)
+lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A, cudaStream_t st);
+lq_status lq_launch_gemm(const lq_layer* L, const lq_act* A, void* Y, lq_out_dtype dt, cudaStream_t st);
+lq_status lq_gemm_prepare(int device);   // sets the kernel's shared-memory attribute once per device
+
+// byte an MMA operand carries for a 4-bit code q in [-7, 7]
+static inline uint8_t lq_encode_code_host(int q, int kind) {
+  if (kind == LQ_KIND_I8) return (uint8_t)(int8_t)q;
+  static const uint8_t mag[8] = {0x00, 0x38, 0x40, 0x44, 0x48, 0x4A, 0x4C, 0x4E};  // E4M3 of 0..7
+  int a = q < 0 ? -q : q;
+  return (uint8_t)(mag[a] | (q < 0 ? 0x80 : 0));
+}
+
+extern int g_lq_main_kind;   // option "main_kind"
+extern int g_lq_gemm_ctas;   // option "gemm_ctas" (0 = one per SM)

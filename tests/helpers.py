@@ -1,0 +1,57 @@
+"""Glue used by the GPU parity tests: oracle layer -> library handle, one forward, comparisons."""
+import numpy as np
+
+from paper_2604_18117_b200 import binding as B
+
+
+def import_oracle_layer(layer: dict):
+    """Feeds a layer produced by the CPU oracle to lq_layer_import (the direction data flows in
+    every parity test: oracle -> library, never the reverse)."""
+    cfg = B.lq_config_default(layer["K"], layer["N"], layer["rank"], layer["branch"])
+    if layer["branch"] == "w16a16":
+        L1, L2, s1, s2 = layer["L1h"], layer["L2h"], None, None
+    elif layer["branch"] == "none" or layer["rank"] == 0:
+        L1 = L2 = s1 = s2 = None
+    else:
+        L1, L2, s1, s2 = layer["L1q"], layer["L2q"], layer["sL1"], layer["sL2"]
+    h = B.lq_layer_import(cfg, B.pack_nibbles(layer["Wq"]), layer["sw"], L1, s1, L2, s2, layer.get("bias"))
+    return h, cfg
+
+
+def gpu_forward(layer: dict, X16: np.ndarray, out_f32: bool = True, export: bool = True, device: int = 0):
+    """Runs lq_quantize_act + lq_linear_forward through the C ABI; returns (Y, exported act dict)."""
+    import torch
+    h, cfg = import_oracle_layer(layer)
+    B.lq_layer_to_device(h, device)
+    M = X16.shape[0]
+    act = B.lq_act_create(h, M, device)
+    try:
+        Xd = torch.from_numpy(np.ascontiguousarray(X16)).to(f"cuda:{device}")
+        Yd = torch.full((M, cfg.N), float("nan"), dtype=torch.float32 if out_f32 else torch.float16,
+                        device=f"cuda:{device}")
+        st = torch.cuda.current_stream().cuda_stream
+        B.lq_quantize_act(h, Xd.data_ptr(), M, act, st)
+        B.lq_linear_forward(h, act, Yd.data_ptr(), B.OUT_F32 if out_f32 else B.OUT_F16, st)
+        torch.cuda.synchronize()
+        code, stage = B.lq_get_device_status(device)
+        assert code == 0, f"device status {code} at stage {stage}"
+        ex = B.lq_act_export(act, M, cfg, st) if export else None
+        return Yd.cpu().numpy(), ex
+    finally:
+        B.lq_act_free(act)
+        B.lq_layer_free(h)
+
+
+def rel_fro(Y, Yref) -> float:
+    Y = Y.astype(np.float64)
+    return float(np.linalg.norm(Y - Yref) / max(np.linalg.norm(Yref), 1e-300))
+
+
+def assert_codes_equal(ex: dict, ref: dict, branch: str):
+    assert np.array_equal(ex["qx"], ref["qx"]), "qx differs"
+    assert np.array_equal(ex["sx"].view(np.uint16), ref["sx"].view(np.uint16)), "sx differs"
+    if branch in ("w8a8", "w6a6", "w4a8"):
+        assert np.array_equal(ex["qb"], ref["qb"]), "qb differs"
+        assert np.array_equal(ex["sXb"].view(np.uint32), ref["sXb"].view(np.uint32)), "sXb differs"
+        assert np.array_equal(ex["tq"], ref["tq"]), "tq differs"
+        assert np.array_equal(ex["sT"].view(np.uint32), ref["sT"].view(np.uint32)), "sT differs"

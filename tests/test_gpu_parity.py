@@ -1,0 +1,112 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Codes and scales must match bit for bit; Y within a relative Frobenius error
+of 1e-3 (fp16 output; the fp16 rounding of Y alone is ~3e-4) and 1e-5 with fp32 output
+(accumulation order only)."""
+import numpy as np
+import pytest
+
+from oracle import lq_oracle as O
+from paper_2604_18117_b200 import binding as B
+from paper_2604_18117_b200 import inputs as I
+from tests.helpers import assert_codes_equal, gpu_forward, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+TOL_F16 = 1e-3
+TOL_F32 = 1e-5
+
+
+def _random_layer(rng, K, N, r, branch, bias=True):
+    """A layer with random quantized parts (no calibration needed for forward parity)."""
+    layer = {"branch": branch if r > 0 else "none", "rank": r, "K": K, "N": N,
+             "bias": (rng.standard_normal(N) * 0.05).astype(np.float16) if bias else None}
+    layer["Wq"], layer["sw"] = O.q_weight_main(rng.standard_normal((K, N)) * 0.02)
+    if r == 0:
+        return layer
+    L1 = rng.standard_normal((K, r)) * 0.05
+    L2 = rng.standard_normal((r, N)) * 0.05
+    if branch == "w16a16":
+        layer["L1h"], _ = O.q_factor(L1, None)
+        layer["L2h"], _ = O.q_factor(L2, None)
+    else:
+        bw, _ = O.BRANCH_BITS[branch]
+        layer["L1q"], layer["sL1"] = O.q_factor(L1, bw)
+        layer["L2q"], layer["sL2"] = O.q_factor(L2, bw)
+    return layer
+
+
+def _check(layer, X, tol32=TOL_F32, tol16=TOL_F16):
+    ref = O.forward(X, layer)
+    Y32, ex = gpu_forward(layer, X, out_f32=True)
+    assert np.isfinite(Y32).all()
+    assert_codes_equal(ex, ref, layer["branch"])
+    e32 = rel_fro(Y32, ref["Y"])
+    assert e32 <= tol32, f"fp32 output error {e32}"
+    Y16, _ = gpu_forward(layer, X, out_f32=False, export=False)
+    fits = np.abs(ref["Y"]).max(axis=1) < 6.0e4            # rows whose outputs fit fp16
+    assert np.isfinite(Y16[fits]).all()
+    e16 = rel_fro(Y16[fits], ref["Y"][fits])
+    assert e16 <= tol16, f"fp16 output error {e16}"
+    return e32, e16
+
+
+def test_integer_exact_main_product():
+    """Integer X in [-7,7] with every group maximum 7 and unit weight scales: all scales are 1,
+    codes equal the inputs, and Y must equal the integer matrix product exactly - any inexact
+    accumulation on the tensor cores shows up as a non-integer or wrong value."""
+    rng = np.random.default_rng(0)
+    M, K, N = 256, 1152, 384
+    X = rng.integers(-7, 8, size=(M, K)).astype(np.float16)
+    X[:, ::64] = 7
+    X[0, :] = 7; X[1, :] = -7                               # extreme partial sums (+-3136 per group)
+    Wi = rng.integers(-7, 8, size=(K, N)); Wi[::64, :] = 7
+    Wi[:, 0] = 7; Wi[:, 1] = -7
+    layer = {"branch": "none", "rank": 0, "K": K, "N": N, "bias": None}
+    layer["Wq"], layer["sw"] = O.q_weight_main(Wi.astype(np.float64))
+    assert np.all(layer["sw"] == 1)
+    Y, ex = gpu_forward(layer, X, out_f32=True)
+    assert np.array_equal(ex["qx"], X.astype(np.int8)) and np.all(ex["sx"] == 1)
+    expect = X.astype(np.int64) @ Wi
+    assert np.array_equal(Y.astype(np.int64), expect) and np.array_equal(Y, expect.astype(np.float32))
+
+
+@pytest.mark.parametrize("branch", ["none", "w8a8", "w6a6", "w4a8", "w16a16"])
+def test_small_shapes_all_branches(branch):
+    rng = np.random.default_rng(1)
+    M, K, N, r = 200, 320, 200, 0 if branch == "none" else 32      # ragged M, N; K = 5 groups (odd)
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    X[:, 7] *= 20
+    _check(_random_layer(rng, K, N, r, branch), X)
+
+
+@pytest.mark.parametrize("r", [16, 64, 128])
+def test_rank_sweep(r):
+    rng = np.random.default_rng(2)
+    M, K, N = 384, 1152, 256
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    _check(_random_layer(rng, K, N, r, "w8a8"), X)
+
+
+def test_ragged_k_and_edge_values():
+    """K = 5600 -> 87.5 groups (short last group); rows of zeros, huge and subnormal values,
+    exact ties."""
+    rng = np.random.default_rng(3)
+    M, K, N, r = 130, 5600, 136, 32
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    X[0, :] = 0
+    X[1, :64] = 0
+    X[2, :] = np.float16(65504.0) * np.sign(rng.standard_normal(K)).astype(np.float16)
+    X[3, :] = np.float16(2.0 ** -24)
+    X[4, :] = (rng.integers(-14, 15, size=K) * 0.5).astype(np.float16); X[4, ::64] = 7   # ties k + 1/2
+    X[5, :] = np.float16(6e-5) * rng.standard_normal(K).astype(np.float16)               # subnormal halves
+    _check(_random_layer(rng, K, N, r, "w4a8"), X)
+
+
+def test_config0_full_calibration():
+    """Config 0: 256 x 1152 x 1152, r = 32, W8A8 branch, data-free calibration run by the oracle."""
+    wl = I.workload(0)
+    X, W, _ = I.layer_inputs(wl, wl.layers[0])
+    layer, trace = O.calibrate(W, 32, "w8a8", steps=1000, lr=1e-4)
+    assert min(trace) < trace[0]
+    e32, e16 = _check(layer, X)
+    print(f"config0 rel err fp32 {e32:.3e} fp16 {e16:.3e}")
