@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of the LoRaQ fused quantized-linear hot path on B200.
+
+One "step" = one pass of the whole hot path (activation quantizer + down-projection, then the
+W4A4 tensor-core GEMM with fused per-group scales / up-projection / bias) over every linear of
+one PixArt-class transformer block (qkv, attn-out, fc1, fc2; hidden 1152, MLP 4608) at
+M = 4096 tokens x batch 2 = 8192 rows, rank 32, W8A8 branch - seeded synthetic tensors that
+stand in for the paper's PixArt-Sigma activations and weights.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is TOPS (2MKN + 2Mr(K+N) algorithmic ops per layer) with inputs
+resident in HBM; `e2e` is the same metric through lq_linear_forward_host (pinned host X in,
+host Y out, copies inside the timed region); `roofline` describes the GEMM kernel against the
+8-bit-operand tensor peak (2 x the measured bf16 cuBLAS peak); `cpu_baseline` is the CPU oracle
+timed on a 256-row sample of the same layers.  With N > 1 (torchrun) every rank runs the same
+rows-sharded workload independently (rows are independent: no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "fused_w4a4_loraq_linear_throughput"
+UNIT = "TOPS"
+SAMPLE_ROWS = 256
+
+
+def layer_ops(M, K, N, r):
+    return 2.0 * M * K * N + 2.0 * M * r * (K + N)
+
+
+def gemm_ops(M, K, N, r):
+    return 2.0 * M * K * N + 2.0 * M * r * N
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows, self.proc, self.index = [], None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([t.strip() for t in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def blas_threads() -> int:
+    """Threads numpy's BLAS (the oracle's matmul) runs on; the rest of the oracle is single-threaded."""
+    try:
+        from threadpoolctl import threadpool_info
+        n = [d.get("num_threads", 1) for d in threadpool_info() if d.get("user_api") == "blas"]
+        return int(max(n)) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def build_workload(args):
+    from paper_2604_18117_b200 import inputs as I
+    wl = I.workload(args.config, branch=args.branch, rank=args.rank)
+    return I, wl
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle as it stands, on a bounded row sample of the same layers."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import lq_oracle as O
+    I, wl = build_workload(args)
+    layers = []
+    for spec in wl.layers:
+        X, W, _ = I.layer_inputs(wl, spec, M=SAMPLE_ROWS)
+        layer, _ = O.calibrate(W, wl.rank, wl.branch, steps=args.calib_steps)
+        layers.append((spec, X, layer))
+    ops_sample = sum(layer_ops(SAMPLE_ROWS, s.K, s.N, wl.rank) for s, _, _ in layers)
+    for _ in range(args.warmup):
+        for _, X, layer in layers:
+            O.forward(X, layer)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        for _, X, layer in layers:
+            O.forward(X, layer)
+    dt = time.perf_counter() - t0
+    value = ops_sample * args.steps / dt / 1e12
+    cores = blas_threads()
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "impl": "reference", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(wl, args) | {"rows_per_step": SAMPLE_ROWS},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{SAMPLE_ROWS} seeded rows of each of the {len(layers)} layers per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def workload_config(wl, args):
+    return {"workload": f"config{wl.config}: PixArt-class block linears (qkv 1152->3456, attn-out 1152->1152, "
+                        f"fc1 1152->4608, fc2 4608->1152), M={wl.M} rows (4096 tokens x batch 2), rank {wl.rank}, "
+                        f"main W4A4 SINT4 group 64, branch {wl.branch}" if wl.config in (1, 2) else f"config{wl.config}",
+            "rows": wl.M, "rank": wl.rank, "branch": wl.branch, "layers": [s.name for s in wl.layers],
+            "calibration_steps": args.calib_steps,
+            "l2": "L2 flushed (256 MiB write) before every timed step; layers inside a step run back to back",
+            "parallelism": f"rows sharded x{args.gpus}, no collective"}
+
+
+def cpu_baseline(wl, I, args):
+    """The oracle on this machine's host cores: 256 sampled rows per layer, all layers, repeated
+    until about 10 s have passed."""
+    from oracle import lq_oracle as O
+    layers = []
+    for spec in wl.layers:
+        X, W, _ = I.layer_inputs(wl, spec, M=SAMPLE_ROWS)
+        layer, _ = O.calibrate(W, wl.rank, wl.branch, steps=0)
+        layers.append((spec, X, layer))
+    ops = sum(layer_ops(SAMPLE_ROWS, s.K, s.N, wl.rank) for s, _, _ in layers)
+    for _, X, layer in layers:
+        O.forward(X, layer)
+    n, t0 = 0, time.perf_counter()
+    while True:
+        for _, X, layer in layers:
+            O.forward(X, layer)
+        n += 1
+        dt = time.perf_counter() - t0
+        if dt > 10.0 or n >= 200:
+            break
+    return {"value": ops * n / dt / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": f"{SAMPLE_ROWS} seeded rows of each of the {len(layers)} layers, {n} passes in {dt:.1f} s "
+                      f"(numpy/BLAS threads as configured on the box)"}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2604_18117_b200 import binding as B
+    from paper_2604_18117_b200 import build as BUILD
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    BUILD.build()
+    I, wl = build_workload(args)
+    M, r = wl.M, wl.rank
+    st = torch.cuda.current_stream().cuda_stream
+
+    layers = []
+    for spec in wl.layers:
+        Xh, W, bias = I.layer_inputs(wl, spec, seed=rank, with_bias=True)
+        cfg = B.lq_config_default(spec.K, spec.N, r, wl.branch)
+        cfg.steps = args.calib_steps
+        h, _ = B.lq_calibrate(cfg, W, bias)
+        B.lq_layer_to_device(h, local)
+        act = B.lq_act_create(h, M, local)
+        Xd = torch.from_numpy(Xh).to(dev)
+        Yd = torch.empty((M, spec.N), dtype=torch.float16, device=dev)
+        Xp = torch.from_numpy(Xh).pin_memory()
+        Yp = torch.empty((M, spec.N), dtype=torch.float16).pin_memory()
+        layers.append(dict(spec=spec, h=h, act=act, Xd=Xd, Yd=Yd, Xp=Xp, Yp=Yp))
+    ops_step = sum(layer_ops(M, L["spec"].K, L["spec"].N, r) for L in layers)
+    gops_step = sum(gemm_ops(M, L["spec"].K, L["spec"].N, r) for L in layers)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+
+    def step(timed=None):
+        flush.zero_()
+        if timed is not None:
+            timed["s"].record()
+        for i, L in enumerate(layers):
+            B.lq_quantize_act(L["h"], L["Xd"].data_ptr(), M, L["act"], st)
+            if timed is not None:
+                timed["g0"][i].record()
+            B.lq_linear_forward(L["h"], L["act"], L["Yd"].data_ptr(), B.OUT_F16, st)
+            if timed is not None:
+                timed["g1"][i].record()
+        if timed is not None:
+            timed["e"].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    timers = [dict(s=ev(), e=ev(), g0=[ev() for _ in layers], g1=[ev() for _ in layers]) for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    for t in timers:
+        step(t)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    step_ms = [t["s"].elapsed_time(t["e"]) for t in timers]
+    gemm_ms = [sum(a.elapsed_time(b) for a, b in zip(t["g0"], t["g1"])) for t in timers]
+    quant_ms = [m - g for m, g in zip(step_ms, gemm_ms)]
+    total_ms = float(sum(step_ms))
+    code, stage = B.lq_get_device_status(local)
+    if code != 0:
+        raise SystemExit(f"device status {code} (stage {stage}) after the timed region")
+    tmax = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    total_ms_max = float(tmax.item())
+
+    # end to end: pinned host X -> device -> K1 -> K2 -> pinned host Y, every step
+    def e2e_step():
+        for L in layers:
+            B.lq_linear_forward_host(L["h"], L["act"], L["Xp"].data_ptr(), M, L["Yp"].data_ptr(), B.OUT_F16, st)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e2e_steps = max(3, min(args.steps, 10))
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_s = float(te.item())
+
+    if rank == 0:
+        peaks = measured_peaks()
+        peak_tops = 2.0 * peaks["bf16_tflops"]
+        gemm_avg_ms = float(np.mean(gemm_ms))
+        achieved = gops_step / (gemm_avg_ms * 1e-3) / 1e12
+        # algorithmic bytes per row of the quantizer: X read once (2K); packed 4-bit codes (K/2), 8-bit branch
+        # codes (K), fp16 group scales (2G), the per-token scale (4), r intermediate codes and their scale (4)
+        k1_bytes = sum(M * (2 * L["spec"].K + L["spec"].K // 2 + L["spec"].K + 2 * (-(-L["spec"].K // 64)) + 4 + r + 4)
+                       for L in layers)
+        quant_avg_ms = float(np.mean(quant_ms))
+        line = {
+            "metric": METRIC, "value": world * ops_step * args.steps / (total_ms_max * 1e-3) / 1e12, "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": total_ms_max / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "e4m3/int8 operands, fp32 accumulate", "data": "synthetic",
+            "config": workload_config(wl, args),
+            "tokens_per_s": world * M * args.steps / (total_ms_max * 1e-3),
+            "e2e": {"value": world * ops_step * e2e_steps / e2e_s / 1e12, "unit": UNIT,
+                    "h2d_bytes_per_step": int(sum(M * L["spec"].K * 2 for L in layers)),
+                    "d2h_bytes_per_step": int(sum(M * L["spec"].N * 2 for L in layers)),
+                    "ms_per_step": e2e_s / e2e_steps * 1e3},
+            "gpu_launches": args.steps * len(layers) * 3,
+            "roofline": {"kernel": "lq_gemm_kernel (4 launches per step, one per layer)", "bound": "tensor",
+                         "achieved": achieved, "peak": peak_tops, "unit": "TOP/s", "frac": achieved / peak_tops,
+                         "traffic": None,
+                         "peak_source": f"2 x bf16_tflops ({peaks['bf16_tflops']}) of {peaks['source']}: 8-bit operands, "
+                                        f"nominal ratio 2 to bf16",
+                         "avg_launch_ms_sum": gemm_avg_ms},
+            "roofline_quantizer": {"kernel": "lq_quant_kernel + down-projection", "bound": "hbm",
+                                   "achieved": k1_bytes / (quant_avg_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                                   "unit": "GB/s", "frac": k1_bytes / (quant_avg_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                   "avg_ms_sum": quant_avg_ms},
+            "clocks": clocks,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(wl, I, args)
+        print(json.dumps(line))
+    for L in layers:
+        B.lq_act_free(L["act"])
+        B.lq_layer_free(L["h"])
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--rank", type=int, default=32)
+    ap.add_argument("--branch", default=None)
+    ap.add_argument("--calib-steps", type=int, default=2, dest="calib_steps")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

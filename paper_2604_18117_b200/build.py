@@ -12,7 +12,7 @@ LIB = os.path.join(HERE, "liblq.so")
 SOURCES = ["lq_api.cu", "lq_quant.cu", "lq_gemm.cu", "lq_calibrate.cpp"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC,-O2,-fopenmp", "-cudart", "static",
+    "-Xcompiler", "-fPIC,-O2,-fopenmp,-ffp-contract=off", "-cudart", "static",
     "-I", os.path.join(ROOT, "include"), "-I", CSRC,
 ]
 

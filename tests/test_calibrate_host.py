@@ -1,0 +1,96 @@
+"""lq_calibrate (host-side C++ in the library) checked on the CPU against closed forms and
+against the oracle's statement of the same procedure."""
+import numpy as np
+
+from oracle import lq_oracle as O
+from paper_2604_18117_b200 import binding as B
+from paper_2604_18117_b200 import build as BUILD
+from paper_2604_18117_b200 import inputs as I
+
+BUILD.build()
+
+
+def _export_as_oracle_layer(h):
+    ex = B.lq_layer_export(h)
+    layer = {"branch": ex["branch"], "rank": ex["rank"], "K": ex["K"], "N": ex["N"], "bias": None,
+             "Wq": B.unpack_nibbles(ex["Wq_packed"]), "sw": ex["sw"]}
+    if ex["branch"] == "w16a16":
+        layer["L1h"], layer["L2h"] = ex["L1"], ex["L2"]
+    elif ex["rank"] > 0:
+        layer.update(L1q=ex["L1"], sL1=ex["sL1"], L2q=ex["L2"], sL2=ex["sL2"])
+    return layer
+
+
+def test_svd_init_eckart_young_known_spectrum():
+    """steps = 0 with the fp16 branch exports L1 L2 = L0 R0 (rounded to fp16): its distance to W
+    must equal the closed-form tail energy of a matrix built with a known spectrum."""
+    rng = np.random.default_rng(0)
+    K, N, r = 128, 96, 8
+    U, _ = np.linalg.qr(rng.standard_normal((K, N)))
+    V, _ = np.linalg.qr(rng.standard_normal((N, N)))
+    sig = np.concatenate([np.linspace(4.0, 2.0, r), np.linspace(0.5, 0.05, N - r)])
+    W = ((U * sig[None, :]) @ V.T).astype(np.float16)
+    s_true = np.linalg.svd(W.astype(np.float64), compute_uv=False)
+    cfg = B.lq_config_default(K, N, r, "w16a16"); cfg.steps = 0
+    h, _ = B.lq_calibrate(cfg, W)
+    ex = B.lq_layer_export(h)
+    approx = ex["L1"].astype(np.float64) @ ex["L2"].astype(np.float64)
+    err2 = np.linalg.norm(W.astype(np.float64) - approx) ** 2
+    tail = np.sum(s_true[r:] ** 2)
+    assert abs(err2 - tail) <= 2e-3 * tail + 1e-6 * np.sum(s_true ** 2)
+    # even split of Sigma: column norms of L1 and row norms of L2 are sqrt(sigma_i)
+    assert np.allclose(np.sort(np.linalg.norm(ex["L1"].astype(np.float64), axis=0))[::-1], np.sqrt(s_true[:r]), rtol=2e-3)
+    assert np.allclose(np.sort(np.linalg.norm(ex["L2"].astype(np.float64), axis=1))[::-1], np.sqrt(s_true[:r]), rtol=2e-3)
+    B.lq_layer_free(h)
+
+
+def test_objective_trace_and_result():
+    W = I.make_weight(0, 0, "pin", 256, 192, 2)
+    cfg = B.lq_config_default(256, 192, 8, "w8a8"); cfg.steps = 150
+    h, trace = B.lq_calibrate(cfg, W, want_trace=True)
+    assert trace.shape == (151,)
+    # iterate 0 = SVD initialisation: same objective as the oracle's closed statement of it
+    _, tr_o = O.calibrate(W, 8, "w8a8", steps=0)
+    assert abs(trace[0] - tr_o[0]) <= 1e-4 * tr_o[0]
+    best = np.minimum.accumulate(trace)
+    assert best[-1] < 0.98 * trace[0]
+    layer = _export_as_oracle_layer(h)
+    W64 = W.astype(np.float64)
+    err = np.linalg.norm(O.effective_weight(layer) - W64)
+    rtn = np.linalg.norm(O.q1_dequant(W64) - W64)
+    assert err < rtn
+    assert np.abs(layer["Wq"]).max() == 7 and np.abs(layer["L1q"]).max() == 127 and np.abs(layer["L2q"]).max() == 127
+    # Figure 1: stored residual codes are Q1 of P = W - Q2(L1) Q2(L2)
+    D = O.deq_factor(layer["L1q"], layer["sL1"]) @ O.deq_factor(layer["L2q"], layer["sL2"])
+    Wq, sw = O.q_weight_main(W64 - D)
+    assert np.mean(Wq == layer["Wq"]) > 0.9999 and np.mean(sw == layer["sw"]) > 0.999
+    B.lq_layer_free(h)
+
+
+def test_rank0_and_round_trip_of_import_export():
+    rng = np.random.default_rng(1)
+    Wq = rng.integers(-7, 8, size=(128, 16)); Wq[0] = 7; Wq[64] = -7
+    W = (Wq * 0.03125).astype(np.float16)
+    cfg = B.lq_config_default(128, 16, 0, "none"); cfg.steps = 0
+    h, trace = B.lq_calibrate(cfg, W, want_trace=True)
+    ex = B.lq_layer_export(h)
+    assert trace[0] == 0.0 and np.array_equal(B.unpack_nibbles(ex["Wq_packed"]), Wq)
+    assert np.all(ex["sw"] == np.float16(0.03125))
+    B.lq_layer_free(h)
+    lay, _ = O.calibrate(I.make_weight(0, 0, "rt", 128, 64, 1), 4, "w6a6", steps=2,
+                         bias=(rng.standard_normal(64) * 0.1).astype(np.float16))
+    c2 = B.lq_config_default(128, 64, 4, "w6a6")
+    h2 = B.lq_layer_import(c2, B.pack_nibbles(lay["Wq"]), lay["sw"], lay["L1q"], lay["sL1"], lay["L2q"], lay["sL2"], lay["bias"])
+    ex2 = B.lq_layer_export(h2)
+    assert np.array_equal(B.unpack_nibbles(ex2["Wq_packed"]), lay["Wq"]) and np.array_equal(ex2["sw"], lay["sw"])
+    assert np.array_equal(ex2["L1"], lay["L1q"]) and np.array_equal(ex2["L2"], lay["L2q"])
+    assert np.array_equal(ex2["sL1"], lay["sL1"]) and np.array_equal(ex2["sL2"], lay["sL2"])
+    assert np.array_equal(ex2["bias"], lay["bias"])
+    B.lq_layer_free(h2)
+    # codes outside the branch's range are rejected
+    bad = lay["L1q"].copy(); bad[0, 0] = 100
+    try:
+        B.lq_layer_import(c2, B.pack_nibbles(lay["Wq"]), lay["sw"], bad, lay["sL1"], lay["L2q"], lay["sL2"], None)
+        assert False
+    except B.LqError as e:
+        assert e.code == 1
