@@ -138,6 +138,33 @@ lq_status lq_linear_forward(const lq_layer* layer, const lq_act* act, void* Y_de
 lq_status lq_linear_forward_host(const lq_layer* layer, lq_act* act, const void* X_f16_host,
                                  int32_t M, void* Y_host, lq_out_dtype dtype, void* cuda_stream);
 
+/* (The paper has no counterpart for this entry point; it exists for deployment.)
+ * Same result as lq_quantize_act followed by lq_linear_forward, for callers that may not
+ * allocate device memory when they call: servers whose own pool owns all device memory once
+ * start-up is over, loops with a fixed memory budget, plugins inside a framework that owns the
+ * allocator - a raw allocation there can fail, fragment the pool, and stalls every stream while
+ * it synchronises the device.  This call performs no allocation (no cudaMalloc / cudaFree,
+ * no allocating library routine): the activation record lives in one fixed device array of
+ * LQ_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU that loads the
+ * library holds that much memory until the process exits.  The caller passes only inputs and
+ * outputs:
+ *   layer      uploaded with lq_layer_to_device (that earlier call is where the layer's
+ *              own device memory was allocated)
+ *   X_f16_dev  [M][K] row-major half, device, 16-byte aligned
+ *   Y_dev      [M][N] row-major half or float per `dtype`, device, 16-byte aligned
+ * Limit: with Mp = M rounded up to 128, Kp = K rounded up to 128 and G2 = Kp / 64, the record
+ * needs about 2*Mp*Kp + 4*G2*Mp + 136*Mp bytes (each part rounded up to 256); if that exceeds
+ * LQ_STATIC_SCRATCH_BYTES the call returns LQ_ERR_UNSUPPORTED and launches nothing
+ * (8 MiB holds e.g. M = 256 at any supported K, or M = 1024 at K = 2240).
+ * The first call on each device looks up the array's device address (one-time set-up, done
+ * with that device current); make that first call before starting any stream capture.
+ * All calls share the one array, which keeps the previous call's contents: each call first
+ * clears the part it uses (on `cuda_stream`), and two calls that overlap on the GPU - other
+ * streams, other threads - race on it; serialise them.  Asynchronous on `cuda_stream`. */
+#define LQ_STATIC_SCRATCH_BYTES (8u << 20)
+lq_status lq_linear_forward_static(const lq_layer* layer, const void* X_f16_dev, int32_t M, void* Y_dev,
+                                   lq_out_dtype dtype, void* cuda_stream);
+
 /* Decode the activation record of the last lq_quantize_act into plain host arrays (for
  * parity checks); NULL skips a part.  qx int8 [M][K], sx half bits [M][G], qb int8 [M][K],
  * sXb float [M], tq int8 [M][rank] (W16A16: half bits [M][rank]), sT float [M].

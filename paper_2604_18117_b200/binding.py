@@ -50,6 +50,7 @@ _SIGNATURES = {
     "lq_quantize_act": [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p],
     "lq_linear_forward": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p],
     "lq_linear_forward_host": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_int, C.c_void_p],
+    "lq_linear_forward_static": [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_int, C.c_void_p],
     "lq_act_export": [C.c_void_p] * 8,
     "lq_get_device_status": [C.c_int, C.POINTER(C.c_int32), C.POINTER(C.c_int32)],
     "lq_set_option": [C.c_char_p, C.c_int32],
@@ -178,6 +179,17 @@ def lq_linear_forward(layer, act, Y_dev_ptr: int, dtype: int = OUT_F16, stream: 
 def lq_linear_forward_host(layer, act, X_host_ptr: int, M: int, Y_host_ptr: int, dtype: int = OUT_F16, stream: int = 0):
     _check(lib().lq_linear_forward_host(layer, act, C.c_void_p(X_host_ptr), M, C.c_void_p(Y_host_ptr), dtype,
                                         C.c_void_p(stream)), "lq_linear_forward_host")
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def lq_linear_forward_static(layer, X_dev_ptr: int, M: int, Y_dev_ptr: int, dtype: int = OUT_F16, stream: int = 0):
+    """Whole forward without any allocation at call time: the activation record lives in a fixed
+    device array inside the library (for callers whose memory pool forbids raw allocations).
+    Raises LqError(code 2) when M x K does not fit the array; calls must not overlap on the GPU."""
+    _check(lib().lq_linear_forward_static(layer, C.c_void_p(X_dev_ptr), M, C.c_void_p(Y_dev_ptr), dtype,
+                                          C.c_void_p(stream)), "lq_linear_forward_static")
 
 
 def lq_act_export(act, M: int, cfg: LqConfig, stream: int = 0) -> dict:
