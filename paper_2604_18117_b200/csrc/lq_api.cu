@@ -10,6 +10,7 @@
 
 int g_lq_main_kind = LQ_KIND_E4M3;
 int g_lq_gemm_ctas = 0;
+int g_lq_store_qb = 0;
 
 #define CUDA_OK(expr)                         \
   do {                                        \
@@ -42,6 +43,10 @@ extern "C" lq_status lq_set_option(const char* name, int32_t value) {
   if (!strcmp(name, "main_kind")) {
     if (value != LQ_KIND_I8 && value != LQ_KIND_E4M3) return LQ_ERR_INVALID_ARG;
     g_lq_main_kind = value;
+    return LQ_OK;
+  }
+  if (!strcmp(name, "store_qb")) {
+    g_lq_store_qb = value != 0;
     return LQ_OK;
   }
   if (!strcmp(name, "gemm_ctas")) {
@@ -92,7 +97,7 @@ lq_layer* lq_layer_new(const lq_config* cfg) {
   L->has_bias = false;
   L->device = -1;
   L->main_kind = g_lq_main_kind;
-  L->d_Wq8 = nullptr; L->d_sw = nullptr; L->d_L1t = nullptr; L->d_L1h = nullptr; L->d_sL1 = nullptr;
+  L->d_Wq8 = nullptr; L->d_sw = nullptr; L->d_L1f = nullptr; L->d_L1h = nullptr; L->d_sL1 = nullptr;
   L->d_L2c = nullptr; L->d_sL2 = nullptr; L->d_bias = nullptr;
   return L;
 }
@@ -242,9 +247,9 @@ extern "C" lq_status lq_get_device_status(int device, int32_t* code, int32_t* st
 static void layer_free_device(lq_layer* L) {
   if (L->device < 0) return;
   cudaSetDevice(L->device);
-  cudaFree(L->d_Wq8); cudaFree(L->d_sw); cudaFree(L->d_L1t); cudaFree(L->d_L1h); cudaFree(L->d_sL1);
+  cudaFree(L->d_Wq8); cudaFree(L->d_sw); cudaFree(L->d_L1f); cudaFree(L->d_L1h); cudaFree(L->d_sL1);
   cudaFree(L->d_L2c); cudaFree(L->d_sL2); cudaFree(L->d_bias);
-  L->d_Wq8 = nullptr; L->d_sw = nullptr; L->d_L1t = nullptr; L->d_L1h = nullptr; L->d_sL1 = nullptr;
+  L->d_Wq8 = nullptr; L->d_sw = nullptr; L->d_L1f = nullptr; L->d_L1h = nullptr; L->d_sL1 = nullptr;
   L->d_L2c = nullptr; L->d_sL2 = nullptr; L->d_bias = nullptr;
   L->device = -1;
 }
@@ -281,10 +286,21 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
     std::vector<float> s1(LQ_MAX_RANK, 1.f), s2((size_t)Npad, 1.f);
     std::vector<uint8_t> l2c((size_t)Npad * LQ_RCONT, 0);
     if (L->integer_branch) {
-      std::vector<int8_t> l1t((size_t)r * Kpad, 0);
-      for (int k = 0; k < K; ++k)
-        for (int j = 0; j < r; ++j) l1t[(size_t)j * Kpad + k] = L->L1q[(size_t)k * r + j];
-      if ((st = upload(&L->d_L1t, l1t)) != LQ_OK) return st;
+      // B fragments of mma.sync.m16n8k32 (s8): lane = 4 * (n % 8) + t holds k = 32 ks + 4 t + {0..3} and + 16
+      const int rpad = lq_round_up(r, 8), ksteps = Kpad / 32, ntiles = rpad / 8;
+      std::vector<uint8_t> l1f((size_t)ksteps * ntiles * 32 * 8, 0);
+      for (int ks = 0; ks < ksteps; ++ks)
+        for (int nt = 0; nt < ntiles; ++nt)
+          for (int lane = 0; lane < 32; ++lane) {
+            const int j = nt * 8 + (lane >> 2), kb = ks * 32 + (lane & 3) * 4;
+            uint8_t* dst = &l1f[(((size_t)ks * ntiles + nt) * 32 + lane) * 8];
+            for (int i = 0; i < 4; ++i) {
+              const int k0 = kb + i, k1 = kb + 16 + i;
+              dst[i] = (j < r && k0 < K) ? (uint8_t)L->L1q[(size_t)k0 * r + j] : 0;
+              dst[4 + i] = (j < r && k1 < K) ? (uint8_t)L->L1q[(size_t)k1 * r + j] : 0;
+            }
+          }
+      if ((st = upload(&L->d_L1f, l1f)) != LQ_OK) return st;
       for (int j = 0; j < r; ++j) s1[j] = L->sL1[j];
       for (int n = 0; n < N; ++n) s2[n] = L->sL2[n];
       for (int j = 0; j < r; ++j)

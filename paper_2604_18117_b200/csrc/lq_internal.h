@@ -51,7 +51,7 @@ struct lq_layer {
   int main_kind;               // LQ_KIND_*: byte encoding of the 4-bit codes in the MMA operands
   uint8_t* d_Wq8;              // [Npad][Kpad] bytes, K contiguous (B operand, K-major)
   float* d_sw;                 // [Gpad][Npad] fp32 (exact images of the fp16 scales)
-  int8_t* d_L1t;               // [r][Kpad] int8, K contiguous   (integer branches)
+  uint8_t* d_L1f;              // [Kpad/32][rpad/8][32 lanes][8 bytes]: first factor in mma.sync B-fragment order (integer branches)
   uint16_t* d_L1h;             // [r][Kpad] half, K contiguous   (W16A16)
   float* d_sL1;                // [LQ_MAX_RANK]
   uint8_t* d_L2c;              // [Npad][LQ_RCONT] bytes: int8 codes (or up to 64 halves) of column n, r contiguous
@@ -96,3 +96,4 @@ static inline uint8_t lq_encode_code_host(int q, int kind) {
 
 extern int g_lq_main_kind;   // option "main_kind"
 extern int g_lq_gemm_ctas;   // option "gemm_ctas" (0 = one per SM)
+extern int g_lq_store_qb;    // option "store_qb": also write the branch activation codes to HBM (parity export)

@@ -18,9 +18,13 @@ def import_oracle_layer(layer: dict):
     return h, cfg
 
 
-def gpu_forward(layer: dict, X16: np.ndarray, out_f32: bool = True, export: bool = True, device: int = 0):
-    """Runs lq_quantize_act + lq_linear_forward through the C ABI; returns (Y, exported act dict)."""
+def gpu_forward(layer: dict, X16: np.ndarray, out_f32: bool = True, export: bool = True, device: int = 0,
+                store_qb: bool = True):
+    """Runs lq_quantize_act + lq_linear_forward through the C ABI; returns (Y, exported act dict).
+    store_qb=True also writes the branch activation codes to HBM so that they can be compared
+    (the benchmark configuration leaves them on chip)."""
     import torch
+    B.lq_set_option("store_qb", 1 if store_qb else 0)
     h, cfg = import_oracle_layer(layer)
     B.lq_layer_to_device(h, device)
     M = X16.shape[0]
@@ -38,6 +42,7 @@ def gpu_forward(layer: dict, X16: np.ndarray, out_f32: bool = True, export: bool
         ex = B.lq_act_export(act, M, cfg, st) if export else None
         return Yd.cpu().numpy(), ex
     finally:
+        B.lq_set_option("store_qb", 0)
         B.lq_act_free(act)
         B.lq_layer_free(h)
 
@@ -47,11 +52,12 @@ def rel_fro(Y, Yref) -> float:
     return float(np.linalg.norm(Y - Yref) / max(np.linalg.norm(Yref), 1e-300))
 
 
-def assert_codes_equal(ex: dict, ref: dict, branch: str):
+def assert_codes_equal(ex: dict, ref: dict, branch: str, with_qb: bool = True):
     assert np.array_equal(ex["qx"], ref["qx"]), "qx differs"
     assert np.array_equal(ex["sx"].view(np.uint16), ref["sx"].view(np.uint16)), "sx differs"
     if branch in ("w8a8", "w6a6", "w4a8"):
-        assert np.array_equal(ex["qb"], ref["qb"]), "qb differs"
+        if with_qb:
+            assert np.array_equal(ex["qb"], ref["qb"]), "qb differs"
         assert np.array_equal(ex["sXb"].view(np.uint32), ref["sXb"].view(np.uint32)), "sXb differs"
         assert np.array_equal(ex["tq"], ref["tq"]), "tq differs"
         assert np.array_equal(ex["sT"].view(np.uint32), ref["sT"].view(np.uint32)), "sT differs"

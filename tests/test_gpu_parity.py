@@ -102,6 +102,49 @@ def test_ragged_k_and_edge_values():
     _check(_random_layer(rng, K, N, r, "w4a8"), X)
 
 
+def test_quantizer_random_bit_patterns_and_exact_ties():
+    """Codes only (Y may overflow): every finite fp16 bit pattern can occur, and whole groups / rows sit
+    exactly on rounding ties with non-trivial scales, which the fast path must hand to the exact path."""
+    rng = np.random.default_rng(4)
+    M, K, N, r = 96, 1024, 64, 16
+    bits = rng.integers(0, 1 << 16, size=(M, K), dtype=np.uint16)
+    bits[(bits & 0x7C00) == 0x7C00] &= 0xBFFF                      # no inf / nan
+    X = bits.view(np.float16).copy()
+    # rows 0..31: each group holds s * c / 2 with group maximum 7 s, s = 2^e (1 + j/8): ties at odd c
+    for m in range(32):
+        for g in range(K // 64):
+            s = np.float16(2.0 ** rng.integers(-10, 6) * (1 + rng.integers(0, 8) / 8))
+            c = rng.integers(-14, 15, size=64)
+            c[rng.integers(0, 64)] = 14
+            X[m, g * 64:(g + 1) * 64] = (np.float32(s) * c.astype(np.float32) * np.float32(0.5)).astype(np.float16)
+    # rows 32..47: per-token ties of the 8-bit branch: row maximum 127 * 2^e, entries (k + 1/2) * 2^e
+    for m in range(32, 48):
+        e = 2.0 ** rng.integers(-6, 3)
+        k = rng.integers(-126, 126, size=K)
+        X[m, :] = ((k + 0.5) * e).astype(np.float16)
+        X[m, rng.integers(0, K)] = np.float16(127 * e)
+    X[48, :] = np.float16(2.0 ** -24)                                # smallest subnormal everywhere
+    X[49, :] = (rng.integers(-12, 13, size=K) * 2.0 ** -24).astype(np.float16)   # subnormal scales, quotients > 7
+    for branch in ("w8a8", "w6a6"):
+        layer = _random_layer(rng, K, N, r, branch)
+        ref = O.forward(X, layer)
+        _, ex = gpu_forward(layer, X, out_f32=True)
+        assert_codes_equal(ex, ref, branch)
+
+
+def test_branch_codes_stay_on_chip_by_default():
+    """The benchmark configuration does not write qb to HBM; everything else must be unchanged."""
+    rng = np.random.default_rng(5)
+    M, K, N, r = 300, 1152, 256, 32
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    layer = _random_layer(rng, K, N, r, "w8a8")
+    ref = O.forward(X, layer)
+    Y, ex = gpu_forward(layer, X, out_f32=True, store_qb=False)
+    assert_codes_equal(ex, ref, "w8a8", with_qb=False)
+    assert not ex["qb"].any()
+    assert rel_fro(Y, ref["Y"]) <= TOL_F32
+
+
 def test_config0_full_calibration():
     """Config 0: 256 x 1152 x 1152, r = 32, W8A8 branch, data-free calibration run by the oracle."""
     wl = I.workload(0)
