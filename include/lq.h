@@ -182,6 +182,9 @@ lq_status lq_get_device_status(int device, int32_t* code, int32_t* stage);
 lq_status lq_set_option(const char* name, int32_t value);
 
 const char* lq_status_string(lq_status s);
+/* Text of the last CUDA runtime error this host thread met inside the library ("no error" if none);
+ * what LQ_ERR_CUDA stood for. */
+const char* lq_last_cuda_error(void);
 int lq_version(void);
 
 #ifdef __cplusplus

@@ -31,7 +31,8 @@ class LqConfig(C.Structure):
 class LqError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
-        super().__init__(f"{where}: {lib().lq_status_string(code).decode()} (lq_status {code})")
+        detail = f" [{lib().lq_last_cuda_error().decode()}]" if code == 4 else ""
+        super().__init__(f"{where}: {lib().lq_status_string(code).decode()} (lq_status {code}){detail}")
 
 
 _lib = None
@@ -55,7 +56,7 @@ _SIGNATURES = {
     "lq_get_device_status": [C.c_int, C.POINTER(C.c_int32), C.POINTER(C.c_int32)],
     "lq_set_option": [C.c_char_p, C.c_int32],
 }
-EXPORTED = tuple(_SIGNATURES) + ("lq_status_string", "lq_version")
+EXPORTED = tuple(_SIGNATURES) + ("lq_status_string", "lq_last_cuda_error", "lq_version")
 
 
 def lib() -> C.CDLL:
@@ -71,6 +72,8 @@ def lib() -> C.CDLL:
             fn.restype = C.c_int
         _lib.lq_status_string.argtypes = [C.c_int]
         _lib.lq_status_string.restype = C.c_char_p
+        _lib.lq_last_cuda_error.argtypes = []
+        _lib.lq_last_cuda_error.restype = C.c_char_p
         _lib.lq_version.argtypes = []
         _lib.lq_version.restype = C.c_int
     return _lib

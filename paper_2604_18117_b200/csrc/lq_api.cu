@@ -12,10 +12,18 @@ int g_lq_main_kind = LQ_KIND_E4M3;
 int g_lq_gemm_ctas = 0;
 int g_lq_store_qb = 0;
 
-#define CUDA_OK(expr)                         \
-  do {                                        \
-    cudaError_t e__ = (expr);                 \
-    if (e__ != cudaSuccess) return LQ_ERR_CUDA; \
+static thread_local cudaError_t t_last_cuda_error = cudaSuccess;
+
+cudaError_t lq_note_cuda(cudaError_t e) {
+  if (e != cudaSuccess) t_last_cuda_error = e;
+  return e;
+}
+
+extern "C" const char* lq_last_cuda_error(void) { return cudaGetErrorString(t_last_cuda_error); }
+
+#define CUDA_OK(expr)                                      \
+  do {                                                     \
+    if (lq_note_cuda(expr) != cudaSuccess) return LQ_ERR_CUDA; \
   } while (0)
 
 static inline float h2f(uint16_t h) {

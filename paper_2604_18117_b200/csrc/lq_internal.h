@@ -78,6 +78,9 @@ struct lq_act {
   CUtensorMap tmT;             // over d_tq,  box [LQ_BM][128B], 128B swizzle
 };
 
+// remembers the last failing CUDA runtime code (per host thread) for lq_last_cuda_error(); returns its argument
+cudaError_t lq_note_cuda(cudaError_t e);
+
 // device status word (one per device, allocated on first use): {code, stage}
 int32_t* lq_device_status_ptr(int device);
 
