@@ -17,7 +17,8 @@
 //   warps 2-17  drain: each warp owns 32 rows x a quarter of the tile's columns; tcgen05.ld one
 //               32 x 16 slice at a time, acc += P * (sx * sw) with packed f32x2 arithmetic
 //               in fp32 registers; after the last group: bias, convert, stage the warp's
-//               rows in shared memory and write each row segment with one bulk copy
+//               rows in shared memory, read them back with lanes along the row and store
+//               whole 64/128-byte row segments
 // Work is cut in units of 128 x 128 outputs; every CTA takes a contiguous run of units
 // (balanced to one unit) and walks it as 128 x 256 tiles, with a 128 x 128 tile where the
 // run or the row block ends.
@@ -140,16 +141,6 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
                : "memory");
 }
-
-// shared -> global bulk copy of one row segment (16-byte aligned, size a multiple of 16), tracked per thread
-__device__ __forceinline__ void bulk_store(void* dst, uint32_t src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(reinterpret_cast<uint64_t>(dst)), "r"(src),
-               "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ void bulk_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -385,7 +376,6 @@ lq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int cgi = (warp - FIRST_DRAIN_WARP) >> 2;     // which quarter of the tile's columns
     const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16);
     uint8_t* out_row = out_ptr + (warp - FIRST_DRAIN_WARP) * OUT_WARP_BYTES + lane * OUT_ROW_STRIDE;
-    const uint32_t out_row_s = smem_u32(out_row);
     uint32_t it = 0, slot = 0;
     bool ok = true;
     for (int u = u_begin; u < u_end && ok;) {
@@ -393,11 +383,19 @@ lq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
       const int m0 = mb * LQ_BM, n0 = nu * UNIT;
       const int coff = cgi * width * 32;                // first of this warp's width*32 columns
-      float2 acc[4][8];                                 // [16-column chunk][column pair]
+      float2 acc[4][8];                                 // [16-column chunk][column pair], starts from the bias
 #pragma unroll
-      for (int a = 0; a < 4; ++a)
+      for (int a = 0; a < 4; ++a) {
+        if (a < 2 * width) {
+          const float4* b4 = reinterpret_cast<const float4*>(p.bias + n0 + coff + a * 16);
 #pragma unroll
-        for (int b = 0; b < 8; ++b) acc[a][b] = make_float2(0.f, 0.f);
+          for (int b = 0; b < 4; ++b) {
+            const float4 bv = __ldg(b4 + b);
+            acc[a][2 * b] = make_float2(bv.x, bv.y);
+            acc[a][2 * b + 1] = make_float2(bv.z, bv.w);
+          }
+        }
+      }
       for (int s = 0; s < stages_per_tile && ok; ++s, ++it) {
         const int st = it % NSTAGE;
         ok = mbar_wait(bar_full(st), (it / NSTAGE) & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
@@ -434,8 +432,9 @@ lq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) mbar_arrive(bar_sempty(st));
       }
       if (!ok) break;
-      // epilogue: bias, convert, stage this thread's row segment, one bulk copy per row and pass
-      const int row = m0 + quad * 32 + lane;
+      // epilogue: convert, stage this thread's row segment in the warp's shared-memory rows, read it back
+      // with lanes along the row and store whole 64/128-byte row segments
+      const int rbase = m0 + quad * 32;
       const int col0 = n0 + coff;
       const int esize = p.out_f32 ? 4 : 2;
       const int cols_per_pass = OUT_ROW_BYTES / esize;                  // 64 halves or 32 floats
@@ -443,53 +442,55 @@ lq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
       for (int pass = 0; pass < 2; ++pass) {
         if (pass < npass) {
-          bulk_store_wait_read();                                       // the staging rows are free again
-          const int cpass = col0 + pass * cols_per_pass;
+          __syncwarp();                                                 // previous pass has been read back
           if (p.out_f32) {
 #pragma unroll
             for (int cc = 0; cc < 2; ++cc) {
               const int ch = pass * 2 + cc;
               if (ch < 2 * width) {
-                const float4* b4 = reinterpret_cast<const float4*>(p.bias + col0 + ch * 16);
 #pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                  const float4 b = __ldg(b4 + c4);
+                for (int c4 = 0; c4 < 4; ++c4)
                   *reinterpret_cast<float4*>(out_row + cc * 64 + c4 * 16) =
-                      make_float4(acc[ch][c4 * 2].x + b.x, acc[ch][c4 * 2].y + b.y, acc[ch][c4 * 2 + 1].x + b.z,
-                                  acc[ch][c4 * 2 + 1].y + b.w);
-                }
+                      make_float4(acc[ch][c4 * 2].x, acc[ch][c4 * 2].y, acc[ch][c4 * 2 + 1].x, acc[ch][c4 * 2 + 1].y);
               }
             }
           } else {
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
               if (ch < 2 * width) {
-                const float4* b4 = reinterpret_cast<const float4*>(p.bias + col0 + ch * 16);
 #pragma unroll
                 for (int c8 = 0; c8 < 2; ++c8) {
-                  const float4 b0 = __ldg(b4 + 2 * c8), b1 = __ldg(b4 + 2 * c8 + 1);
                   __half2 h[4];
-                  h[0] = __floats2half2_rn(acc[ch][c8 * 4 + 0].x + b0.x, acc[ch][c8 * 4 + 0].y + b0.y);
-                  h[1] = __floats2half2_rn(acc[ch][c8 * 4 + 1].x + b0.z, acc[ch][c8 * 4 + 1].y + b0.w);
-                  h[2] = __floats2half2_rn(acc[ch][c8 * 4 + 2].x + b1.x, acc[ch][c8 * 4 + 2].y + b1.y);
-                  h[3] = __floats2half2_rn(acc[ch][c8 * 4 + 3].x + b1.z, acc[ch][c8 * 4 + 3].y + b1.w);
+                  h[0] = __floats2half2_rn(acc[ch][c8 * 4 + 0].x, acc[ch][c8 * 4 + 0].y);
+                  h[1] = __floats2half2_rn(acc[ch][c8 * 4 + 1].x, acc[ch][c8 * 4 + 1].y);
+                  h[2] = __floats2half2_rn(acc[ch][c8 * 4 + 2].x, acc[ch][c8 * 4 + 2].y);
+                  h[3] = __floats2half2_rn(acc[ch][c8 * 4 + 3].x, acc[ch][c8 * 4 + 3].y);
                   *reinterpret_cast<uint4*>(out_row + ch * 32 + c8 * 16) = *reinterpret_cast<uint4*>(h);
                 }
               }
             }
           }
-          fence_proxy_async();                                          // generic-proxy writes -> visible to the bulk copy
-          int ncols = width * 32 - pass * cols_per_pass;
+          __syncwarp();
+          int ncols = width * 32 - pass * cols_per_pass;                // columns of this pass
           if (ncols > cols_per_pass) ncols = cols_per_pass;
-          if (ncols > p.N - cpass) ncols = p.N - cpass;
-          if (row < p.M && ncols > 0)
-            bulk_store(reinterpret_cast<uint8_t*>(p.Y) + ((size_t)row * p.N + cpass) * esize, out_row_s, (uint32_t)(ncols * esize));
-          bulk_store_commit();
+          const int lpr = ncols * esize / 16;                           // lanes per row: 4 or 8
+          const int rpi = 32 / lpr;                                     // rows per instruction
+          const int cpl = 16 / esize;                                   // columns per lane
+          const int lcol = col0 + pass * cols_per_pass + (lane % lpr) * cpl;
+          const uint8_t* wbase = out_ptr + (warp - FIRST_DRAIN_WARP) * OUT_WARP_BYTES + (lane % lpr) * 16;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            if (i * rpi < 32) {
+              const int rl = i * rpi + lane / lpr;
+              const uint4 val = *reinterpret_cast<const uint4*>(wbase + rl * OUT_ROW_STRIDE);
+              if (rbase + rl < p.M && lcol < p.N)
+                *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.Y) + ((size_t)(rbase + rl) * p.N + lcol) * esize) = val;
+            }
+          }
         }
       }
       u += width;
     }
-    bulk_store_wait_read();   // shared memory must outlive the copies that read it
   }
 
   // ---------------------------------------------------------------------- teardown
