@@ -5,37 +5,30 @@
 //   a3  down-projection I1 = qb L1q, exact int32, on the tensor cores (mma.sync, s8)
 //   a4  t = fl32(fl32(I1) * fl32(sXb * sL1)), per-token re-quantization of the rank-r row
 //
-// A CTA owns 16 rows (one m16 MMA tile); each of its 8 warps quantizes 2 rows, one after the
-// other, holding the row in registers (16-byte loads, X is read from HBM exactly once), then
-// the CTA multiplies its 16 x K tile of branch codes, staged in shared memory, with L1q.
+// A CTA owns 16 rows (one m16 MMA tile).  A warp holds one row in registers (16-byte loads,
+// X is read from HBM exactly once), finds the row maximum, then walks the row once more and
+// emits both code streams; the CTA then multiplies its 16 x K tile of branch codes, staged in
+// shared memory, with L1q.
 //
 // Exactness contract: codes and scales equal the definition evaluated in IEEE binary32 with
-// round-to-nearest-even and true division.  The fast path replaces the per-element division
-// by a multiplication with the correctly rounded reciprocal plus an exact remainder test:
-//   main    q' = rint(x * (1/s)); e = fma(-q', s, x) is exact (q' has 4 bits, s 11 bits).
+// round-to-nearest-even and true division.  The fast path is division free:
+//   scale   fp16(a / 7) == fp16(a * fl32(1/7)) for every finite fp16 a (checked exhaustively on
+//           the host), because a/7 never comes closer than 2^-15 (relative) to an fp16 midpoint.
+//   main    q' = rint(x * r), r ~ 1/s; e = fma(-q', s, x) is exact (q' has 3 bits, s 11 bits).
 //           x and s are fp16 numbers, so x/s is either exactly k + 1/2 or at least 1e-4 away
-//           from it, while x * (1/s) is within 5e-7 of x/s: q' is the correctly rounded code
-//           unless |e| == s/2 exactly (a true tie) - those elements take the slow path.
-//   branch  same with the fp32 scale; the element takes the slow path (IEEE division) whenever
-//           |e| >= 0.499 s, i.e. whenever the quotient is not safely inside a rounding cell.
+//           from it, while x * r is within 3e-6 of x/s: q' is the correctly rounded code unless
+//           |e| == s/2 exactly (a true tie) - those elements take the exact path.
+//   branch  same with the fp32 per-token scale; an element takes the exact path (IEEE division)
+//           whenever |e| >= 0.4999 s, i.e. whenever the quotient is not safely inside a
+//           rounding cell (the estimate is within 5e-5 of the quotient).
 #include <cuda_fp16.h>
 
 #include "lq_internal.h"
 
 namespace {
 
-constexpr int ROWS = 16;          // rows per CTA
-constexpr int QWARPS = 8;
+constexpr int ROWS = 16;               // rows per CTA
 constexpr float MAGIC = 12582912.0f;   // 1.5 * 2^23: adding it rounds to an integer (ties to even)
-
-__device__ __forceinline__ uint32_t encode_code(int q, int kind) {
-  if (kind == LQ_KIND_I8) return (uint32_t)q & 0xFFu;
-  // E4M3 byte of an integer in [-7, 7]: 0,1,2,3,4,5,6,7 -> 00 38 40 44 48 4A 4C 4E
-  const int a = q < 0 ? -q : q;
-  const uint64_t tab = 0x4E4C4A4844403800ull;
-  uint32_t b = (uint32_t)(tab >> (8 * a)) & 0xFFu;
-  return b | (q < 0 ? 0x80u : 0u);
-}
 
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
@@ -48,6 +41,12 @@ __device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float hi, float lo) {
   uint16_t r;
   asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
   return (uint32_t)r;
+}
+
+__device__ __forceinline__ float rcp_fast(float x) {
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
 }
 
 __device__ __forceinline__ void mma_s8_16832(int (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
@@ -69,14 +68,14 @@ struct QuantParams {
   uint8_t* tq;          // [Mpad][LQ_RCONT]
   float* sT;            // [Mpad]
   int r, rpad;          // rank, rank rounded up to 8
-  int main_kind;
   int branch_qmax;      // 0: no integer branch
 };
 
 // Shared memory: qb tile [ROWS][Kpad + 16] bytes | sx tile [Gpad][ROWS] floats | I1 [ROWS][rpad] ints | sXb [ROWS]
-template <int NCHUNK>
-__global__ void __launch_bounds__(QWARPS * 32) lq_quant_kernel(const QuantParams p) {
+template <int NCHUNK, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams p) {
   extern __shared__ __align__(16) uint8_t qsm[];
+  constexpr int RPW = ROWS / WARPS;    // rows per warp
   const int qb_stride = p.Kpad + 16;
   const int Gpad = p.Kpad / LQ_GROUP;
   uint8_t* qb_s = qsm;
@@ -86,13 +85,13 @@ __global__ void __launch_bounds__(QWARPS * 32) lq_quant_kernel(const QuantParams
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * ROWS;
-  const bool e4m3 = p.main_kind == LQ_KIND_E4M3;
   const float qm = (float)p.branch_qmax;
 
-  for (int i = threadIdx.x; i < ROWS * p.rpad; i += QWARPS * 32) I1_s[i] = 0;
+  for (int i = threadIdx.x; i < ROWS * p.rpad; i += WARPS * 32) I1_s[i] = 0;
 
-  for (int rr = 0; rr < 2; ++rr) {
-    const int rl = warp * 2 + rr;
+#pragma unroll 1
+  for (int rr = 0; rr < RPW; ++rr) {
+    const int rl = warp * RPW + rr;
     const int m = m0 + rl;
     if (m >= p.M) {   // tail rows: zero codes so the MMA tile is defined
       if (p.branch_qmax > 0)
@@ -106,104 +105,84 @@ __global__ void __launch_bounds__(QWARPS * 32) lq_quant_kernel(const QuantParams
       const int k0 = c * 256 + lane * 8;
       v[c] = (k0 < p.K) ? __ldg(xrow + (k0 >> 3)) : make_uint4(0, 0, 0, 0);
     }
-    float rowmax = 0.f;
-    // ---------------------------------------------------------------- a1: SINT4 codes
+    // ---- pass A: this lane's maximum per chunk (exact in fp16) and the row maximum
+    __half hm[NCHUNK];
+    __half hrow = __ushort_as_half((unsigned short)0);
+#pragma unroll
+    for (int c = 0; c < NCHUNK; ++c) {
+      const __half2* h2 = reinterpret_cast<const __half2*>(&v[c]);
+      const __half2 m2 = __hmax2(__hmax2(__habs2(h2[0]), __habs2(h2[1])), __hmax2(__habs2(h2[2]), __habs2(h2[3])));
+      hm[c] = __hmax(__low2half(m2), __high2half(m2));
+      hrow = __hmax(hrow, hm[c]);
+    }
+    float sb = 1.0f, invb = 1.0f, thr = 0.f;
+    if (p.branch_qmax > 0) {
+      const float rowmax = warp_max(__half2float(hrow));
+      sb = (rowmax == 0.f) ? 1.0f : __fdiv_rn(rowmax, qm);
+      invb = __frcp_rn(sb);
+      thr = 0.4999f * sb;
+      if (lane == 0) { sXb_s[rl] = sb; p.sXb[m] = sb; }
+    }
+    // ---- pass B: group scales, 4-bit codes (a1) and branch codes (a2)
 #pragma unroll
     for (int c = 0; c < NCHUNK; ++c) {
       const int k0 = c * 256 + lane * 8;
-      const __half2* h2 = reinterpret_cast<const __half2*>(&v[c]);
-      const __half2 m2 = __hmax2(__hmax2(__habs2(h2[0]), __habs2(h2[1])), __hmax2(__habs2(h2[2]), __habs2(h2[3])));
-      float a = fmaxf(__low2float(m2), __high2float(m2));
-      rowmax = fmaxf(rowmax, a);
+      float a = __half2float(hm[c]);
       a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
       a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
       a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 4));
-      __half s16 = __float2half_rn(__fdiv_rn(a, 7.0f));
-      const unsigned short sbits = __half_as_ushort(s16);
-      if (sbits == 0) s16 = __ushort_as_half((unsigned short)1);   // floor 2^-24
-      const float s = __half2float(s16);
-      if (k0 < p.K) {
-        float x[8], q[8];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float2 f = __half22float2(h2[i]);
-          x[2 * i] = f.x; x[2 * i + 1] = f.y;
-        }
-        bool slow = sbits < 0x0400;          // subnormal scale: quotient may exceed 7, use the plain definition
-        if (!slow) {
-          const float inv = __frcp_rn(s), hs = 0.5f * s;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            q[i] = __fadd_rn(__fmaf_rn(x[i], inv, MAGIC), -MAGIC);
-            const float e = __fmaf_rn(-q[i], s, x[i]);
-            slow |= (fabsf(e) == hs);
-          }
-        }
-        if (slow) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) q[i] = fminf(fmaxf(rintf(__fdiv_rn(x[i], s)), -7.f), 7.f);
-        }
-        uint32_t w0, w1;
-        if (e4m3) {
-          w0 = f32x2_to_e4m3x2(q[1], q[0]) | (f32x2_to_e4m3x2(q[3], q[2]) << 16);
-          w1 = f32x2_to_e4m3x2(q[5], q[4]) | (f32x2_to_e4m3x2(q[7], q[6]) << 16);
-        } else {
-          w0 = ((uint32_t)(int)q[0] & 0xFFu) | (((uint32_t)(int)q[1] & 0xFFu) << 8) | (((uint32_t)(int)q[2] & 0xFFu) << 16) |
-               (((uint32_t)(int)q[3] & 0xFFu) << 24);
-          w1 = ((uint32_t)(int)q[4] & 0xFFu) | (((uint32_t)(int)q[5] & 0xFFu) << 8) | (((uint32_t)(int)q[6] & 0xFFu) << 16) |
-               (((uint32_t)(int)q[7] & 0xFFu) << 24);
-        }
-        *reinterpret_cast<uint2*>(p.qx8 + (size_t)m * p.Kpad + k0) = make_uint2(w0, w1);
-        if ((lane & 7) == 0) sx_s[(k0 >> 6) * ROWS + rl] = s;
-      }
-    }
-    if (p.branch_qmax <= 0) continue;
-    // ---------------------------------------------------------------- a2: per-token branch codes
-    rowmax = warp_max(rowmax);
-    const float sb = (rowmax == 0.f) ? 1.0f : __fdiv_rn(rowmax, qm);
-    if (lane == 0) { sXb_s[rl] = sb; p.sXb[m] = sb; }
-    const float inv = __frcp_rn(sb), thr = 0.499f * sb;
-#pragma unroll
-    for (int c = 0; c < NCHUNK; ++c) {
-      const int k0 = c * 256 + lane * 8;
       if (k0 < p.Kpad) {
-        uint32_t w0 = 0, w1 = 0;
+        uint32_t w0 = 0, w1 = 0, b0 = 0, b1 = 0;
         if (k0 < p.K) {
+          __half s16 = __float2half_rn(__fmul_rn(a, 0.142857149243354797f));   // fl32(1/7)
+          const unsigned short sbits = __half_as_ushort(s16);
+          if (sbits == 0) s16 = __ushort_as_half((unsigned short)1);             // floor 2^-24
+          const float s = __half2float(s16);
           const __half2* h2 = reinterpret_cast<const __half2*>(&v[c]);
-          float x[8], t[8];
+          float x[8], q[8], t[8];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const float2 f = __half22float2(h2[i]);
             x[2 * i] = f.x; x[2 * i + 1] = f.y;
           }
-          bool slow = false;
+          const float inv = rcp_fast(s), hs = 0.5f * s;
+          bool exact = sbits < 0x0400;          // subnormal scale: quotient may exceed 7, use the plain definition
+          bool near = false;
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            t[i] = __fmaf_rn(x[i], inv, MAGIC);                    // low byte of the bit pattern = code
-            const float e = __fmaf_rn(-__fadd_rn(t[i], -MAGIC), sb, x[i]);
-            slow |= !(fabsf(e) < thr);
+            q[i] = __fadd_rn(__fmaf_rn(x[i], inv, MAGIC), -MAGIC);
+            const float e = __fmaf_rn(-q[i], s, x[i]);
+            exact |= (fabsf(e) == hs);
+            t[i] = __fmaf_rn(x[i], invb, MAGIC);                    // low byte of the bit pattern = branch code
+            const float eb = __fmaf_rn(-__fadd_rn(t[i], -MAGIC), sb, x[i]);
+            near |= !(fabsf(eb) < thr);
           }
-          if (slow) {
+          if (exact) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const float qf = fminf(fmaxf(rintf(__fdiv_rn(x[i], sb)), -qm), qm);
-              t[i] = __fadd_rn(qf, MAGIC);
-            }
+            for (int i = 0; i < 8; ++i) q[i] = fminf(fmaxf(rintf(__fdiv_rn(x[i], s)), -7.f), 7.f);
           }
-          w0 = __byte_perm(__byte_perm(__float_as_uint(t[0]), __float_as_uint(t[1]), 0x0040),
+          if (near) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) t[i] = __fadd_rn(fminf(fmaxf(rintf(__fdiv_rn(x[i], sb)), -qm), qm), MAGIC);
+          }
+          w0 = f32x2_to_e4m3x2(q[1], q[0]) | (f32x2_to_e4m3x2(q[3], q[2]) << 16);
+          w1 = f32x2_to_e4m3x2(q[5], q[4]) | (f32x2_to_e4m3x2(q[7], q[6]) << 16);
+          b0 = __byte_perm(__byte_perm(__float_as_uint(t[0]), __float_as_uint(t[1]), 0x0040),
                            __byte_perm(__float_as_uint(t[2]), __float_as_uint(t[3]), 0x0040), 0x5410);
-          w1 = __byte_perm(__byte_perm(__float_as_uint(t[4]), __float_as_uint(t[5]), 0x0040),
+          b1 = __byte_perm(__byte_perm(__float_as_uint(t[4]), __float_as_uint(t[5]), 0x0040),
                            __byte_perm(__float_as_uint(t[6]), __float_as_uint(t[7]), 0x0040), 0x5410);
+          *reinterpret_cast<uint2*>(p.qx8 + (size_t)m * p.Kpad + k0) = make_uint2(w0, w1);
+          if ((lane & 7) == 0) sx_s[(k0 >> 6) * ROWS + rl] = s;
+          if (p.qb != nullptr && p.branch_qmax > 0) *reinterpret_cast<uint2*>(p.qb + (size_t)m * p.Kpad + k0) = make_uint2(b0, b1);
         }
-        *reinterpret_cast<uint2*>(qb_s + rl * qb_stride + k0) = make_uint2(w0, w1);
-        if (p.qb != nullptr && k0 < p.K) *reinterpret_cast<uint2*>(p.qb + (size_t)m * p.Kpad + k0) = make_uint2(w0, w1);
+        if (p.branch_qmax > 0) *reinterpret_cast<uint2*>(qb_s + rl * qb_stride + k0) = make_uint2(b0, b1);
       }
     }
   }
   __syncthreads();
 
   // group scales, transposed: [g][m0 .. m0+15] are 64-byte segments
-  for (int i = threadIdx.x; i < p.G * ROWS; i += QWARPS * 32) {
+  for (int i = threadIdx.x; i < p.G * ROWS; i += WARPS * 32) {
     const int g = i / ROWS, rl = i % ROWS;
     if (m0 + rl < p.M) p.sx[(size_t)g * p.Mpad + m0 + rl] = sx_s[g * ROWS + rl];
   }
@@ -218,7 +197,7 @@ __global__ void __launch_bounds__(QWARPS * 32) lq_quant_kernel(const QuantParams
     for (int a = 0; a < 4; ++a)
 #pragma unroll
       for (int b = 0; b < 4; ++b) acc[a][b] = 0;
-    for (int ks = warp; ks < ksteps; ks += QWARPS) {
+    for (int ks = warp; ks < ksteps; ks += WARPS) {
       uint32_t a[4];
       const uint8_t* ab = qb_s + ks * 32 + tig * 4;
       a[0] = *reinterpret_cast<const uint32_t*>(ab + gid * qb_stride);
@@ -247,8 +226,8 @@ __global__ void __launch_bounds__(QWARPS * 32) lq_quant_kernel(const QuantParams
   __syncthreads();
 
   // ------------------------------------------------------------------ a4: re-quantize the rank-r row
-  for (int rr = 0; rr < 2; ++rr) {
-    const int rl = warp * 2 + rr, m = m0 + rl;
+  for (int rr = 0; rr < RPW; ++rr) {
+    const int rl = warp * RPW + rr, m = m0 + rl;
     if (m >= p.M) continue;
     const float sb = sXb_s[rl];
     float t[4], amax = 0.f;
@@ -293,17 +272,17 @@ __global__ void __launch_bounds__(256) lq_down_f16_kernel(const __half* __restri
   if (lane == 0) sT[m] = 1.0f;
 }
 
-template <int NCHUNK>
+template <int NCHUNK, int WARPS>
 cudaError_t launch_quant(const QuantParams& p, size_t smem, cudaStream_t st) {
   static bool attr_set[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
   if (smem > 48 * 1024 && !attr_set[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(lq_quant_kernel<NCHUNK>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(lq_quant_kernel<NCHUNK, WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
     attr_set[dev & 63] = true;
   }
-  lq_quant_kernel<NCHUNK><<<lq_ceil_div(p.M, ROWS), QWARPS * 32, smem, st>>>(p);
+  lq_quant_kernel<NCHUNK, WARPS><<<lq_ceil_div(p.M, ROWS), WARPS * 32, smem, st>>>(p);
   return cudaGetLastError();
 }
 
@@ -322,21 +301,21 @@ lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A,
   p.L1f = reinterpret_cast<const uint2*>(L->d_L1f);
   p.sL1 = L->d_sL1; p.tq = A->d_tq; p.sT = A->d_sT;
   p.r = L->r; p.rpad = lq_round_up(L->r > 0 ? L->r : 8, 8);
-  p.main_kind = A->main_kind;
   p.branch_qmax = (L->integer_branch && abits > 0) ? ((1 << (abits - 1)) - 1) : 0;
   const size_t smem = (p.branch_qmax > 0 ? (size_t)ROWS * (Kpad + 16) : 0) + (size_t)(Kpad / LQ_GROUP) * ROWS * 4 +
                       (size_t)ROWS * p.rpad * 4 + ROWS * 4;
   const int nchunk = lq_ceil_div(Kpad, 256);
   cudaError_t e;
-  if (nchunk <= 2) e = launch_quant<2>(p, smem, st);
-  else if (nchunk <= 5) e = launch_quant<5>(p, smem, st);
-  else if (nchunk <= 9) e = launch_quant<9>(p, smem, st);
-  else if (nchunk <= 12) e = launch_quant<12>(p, smem, st);
-  else if (nchunk <= 18) e = launch_quant<18>(p, smem, st);
-  else if (nchunk <= 22) e = launch_quant<22>(p, smem, st);
-  else if (nchunk <= 32) e = launch_quant<32>(p, smem, st);
+  if (A->main_kind != LQ_KIND_E4M3) return LQ_ERR_UNSUPPORTED;
+  if (nchunk <= 2) e = launch_quant<2, 16>(p, smem, st);        // one row per warp while the row fits 128 registers
+  else if (nchunk <= 5) e = launch_quant<5, 16>(p, smem, st);
+  else if (nchunk <= 9) e = launch_quant<9, 16>(p, smem, st);
+  else if (nchunk <= 12) e = launch_quant<12, 8>(p, smem, st);
+  else if (nchunk <= 18) e = launch_quant<18, 8>(p, smem, st);
+  else if (nchunk <= 22) e = launch_quant<22, 8>(p, smem, st);
+  else if (nchunk <= 32) e = launch_quant<32, 8>(p, smem, st);
   else return LQ_ERR_UNSUPPORTED;
-  if (e != cudaSuccess) return LQ_ERR_CUDA;
+  if (lq_note_cuda(e) != cudaSuccess) return LQ_ERR_CUDA;
   if (L->f16_branch) {
     lq_down_f16_kernel<<<lq_ceil_div(M, 8), 256, 0, st>>>(reinterpret_cast<const __half*>(X),
                                                           reinterpret_cast<const __half*>(L->d_L1h), M, K, Kpad, L->r,
