@@ -53,6 +53,21 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def gemm_traffic_bytes():
+    """DRAM bytes of one step's GEMM launches as measured by ncu (profiles/gemm_dram_traffic.json),
+    or None when the GEMM source differs from the one that was profiled."""
+    import hashlib
+    rec = os.path.join(ROOT, "profiles", "gemm_dram_traffic.json")
+    src = os.path.join(ROOT, "paper_2604_18117_b200", "csrc", "lq_gemm.cu")
+    try:
+        d = json.load(open(rec))
+        if hashlib.sha256(open(src, "rb").read()).hexdigest() != d["lq_gemm_cu_sha256"]:
+            return None
+        return int(d["dram_bytes_per_step"])
+    except (OSError, KeyError, ValueError):
+        return None
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks / throttle reasons while the timed region runs."""
 
@@ -227,6 +242,8 @@ def run_ours(args):
         if timed is not None:
             timed["s"].record()
         for i, L in enumerate(layers):
+            if timed is not None:
+                timed["q0"][i].record()
             B.lq_quantize_act(L["h"], L["Xd"].data_ptr(), M, L["act"], st)
             if timed is not None:
                 timed["g0"][i].record()
@@ -244,7 +261,8 @@ def run_ours(args):
     for _ in range(max(args.warmup, 3)):
         step()
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    timers = [dict(s=ev(), e=ev(), g0=[ev() for _ in layers], g1=[ev() for _ in layers]) for _ in range(args.steps)]
+    timers = [dict(s=ev(), e=ev(), q0=[ev() for _ in layers], g0=[ev() for _ in layers], g1=[ev() for _ in layers])
+              for _ in range(args.steps)]
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -255,7 +273,15 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     step_ms = [t["s"].elapsed_time(t["e"]) for t in timers]
     gemm_ms = [sum(a.elapsed_time(b) for a, b in zip(t["g0"], t["g1"])) for t in timers]
-    quant_ms = [m - g for m, g in zip(step_ms, gemm_ms)]
+    quant_ms = [sum(a.elapsed_time(b) for a, b in zip(t["q0"], t["g0"])) for t in timers]
+    per_layer = []
+    for i, L in enumerate(layers):
+        q = float(np.mean([t["q0"][i].elapsed_time(t["g0"][i]) for t in timers]))
+        g = float(np.mean([t["g0"][i].elapsed_time(t["g1"][i]) for t in timers]))
+        sp = L["spec"]
+        per_layer.append({"layer": sp.name, "K": sp.K, "N": sp.N, "quantize_us": q * 1e3, "gemm_us": g * 1e3,
+                          "gemm_tops": gemm_ops(M, sp.K, sp.N, r) / (g * 1e-3) / 1e12,
+                          "pair_tops": layer_ops(M, sp.K, sp.N, r) / ((q + g) * 1e-3) / 1e12})
     total_ms = float(sum(step_ms))
     code, stage = B.lq_get_device_status(local)
     if code != 0:
@@ -298,17 +324,18 @@ def run_ours(args):
             "metric": METRIC, "value": world * ops_step * args.steps / (total_ms_max * 1e-3) / 1e12, "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": total_ms_max / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "e4m3/int8 operands, fp32 accumulate", "data": "synthetic",
+            "vs_baseline": None, "dtype": "e4m3 (exact int4 codes) / int8 operands, fp32 accumulate", "data": "synthetic",
             "config": workload_config(wl, args),
             "tokens_per_s": world * M * args.steps / (total_ms_max * 1e-3),
             "e2e": {"value": world * ops_step * e2e_steps / e2e_s / 1e12, "unit": UNIT,
                     "h2d_bytes_per_step": int(sum(M * L["spec"].K * 2 for L in layers)),
                     "d2h_bytes_per_step": int(sum(M * L["spec"].N * 2 for L in layers)),
                     "ms_per_step": e2e_s / e2e_steps * 1e3},
-            "gpu_launches": args.steps * len(layers) * 3,
+            "gpu_launches": args.steps * len(layers) * (3 if wl.branch == "w16a16" else 2),
             "roofline": {"kernel": "lq_gemm_kernel (4 launches per step, one per layer)", "bound": "tensor",
                          "achieved": achieved, "peak": peak_tops, "unit": "TOP/s", "frac": achieved / peak_tops,
-                         "traffic": None,
+                         "traffic": gemm_traffic_bytes(), "traffic_note": "DRAM read + write bytes of the four GEMM "
+                         "launches of one step from one ncu capture; null when the kernel source changed since",
                          "peak_source": f"2 x bf16_tflops ({peaks['bf16_tflops']}) of {peaks['source']}: 8-bit operands, "
                                         f"nominal ratio 2 to bf16",
                          "avg_launch_ms_sum": gemm_avg_ms},
@@ -316,6 +343,7 @@ def run_ours(args):
                                    "achieved": k1_bytes / (quant_avg_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                                    "unit": "GB/s", "frac": k1_bytes / (quant_avg_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                    "avg_ms_sum": quant_avg_ms},
+            "layers": per_layer,
             "clocks": clocks,
         }
         if not args.no_cpu_baseline and world == 1:

@@ -72,7 +72,10 @@ struct QuantParams {
 };
 
 // Shared memory: qb tile [ROWS][Kpad + 16] bytes | sx tile [Gpad][ROWS] floats | I1 [ROWS][rpad] ints | sXb [ROWS]
-template <int NCHUNK, int WARPS>
+// RELOAD: rows too long for the register file are read twice, chunk by chunk - once for the row maximum,
+// once to quantize; the second read is served by the L2 (the row was touched microseconds earlier), so DRAM
+// still sees X once, and the kernel keeps 64 registers per thread and full occupancy.
+template <int NCHUNK, int WARPS, bool RELOAD>
 __global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams p) {
   extern __shared__ __align__(16) uint8_t qsm[];
   constexpr int RPW = ROWS / WARPS;    // rows per warp
@@ -99,21 +102,34 @@ __global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams 
       continue;
     }
     const uint4* xrow = p.X + (size_t)m * (p.K / 8);
-    uint4 v[NCHUNK];
-#pragma unroll
-    for (int c = 0; c < NCHUNK; ++c) {
-      const int k0 = c * 256 + lane * 8;
-      v[c] = (k0 < p.K) ? __ldg(xrow + (k0 >> 3)) : make_uint4(0, 0, 0, 0);
-    }
-    // ---- pass A: this lane's maximum per chunk (exact in fp16) and the row maximum
-    __half hm[NCHUNK];
+    constexpr int NKEEP = RELOAD ? 1 : NCHUNK;
+    uint4 v[NKEEP];
+    __half hm[NKEEP];
     __half hrow = __ushort_as_half((unsigned short)0);
-#pragma unroll
-    for (int c = 0; c < NCHUNK; ++c) {
-      const __half2* h2 = reinterpret_cast<const __half2*>(&v[c]);
+    // ---- pass A: this lane's maximum per chunk (exact in fp16) and the row maximum
+    auto lane_max = [](const uint4& w) {
+      const __half2* h2 = reinterpret_cast<const __half2*>(&w);
       const __half2 m2 = __hmax2(__hmax2(__habs2(h2[0]), __habs2(h2[1])), __hmax2(__habs2(h2[2]), __habs2(h2[3])));
-      hm[c] = __hmax(__low2half(m2), __high2half(m2));
-      hrow = __hmax(hrow, hm[c]);
+      return __hmax(__low2half(m2), __high2half(m2));
+    };
+    if constexpr (RELOAD) {
+#pragma unroll 6
+      for (int c = 0; c < NCHUNK; ++c) {
+        const int k0 = c * 256 + lane * 8;
+        const uint4 w = (k0 < p.K) ? __ldg(xrow + (k0 >> 3)) : make_uint4(0, 0, 0, 0);
+        hrow = __hmax(hrow, lane_max(w));
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < NCHUNK; ++c) {
+        const int k0 = c * 256 + lane * 8;
+        v[c] = (k0 < p.K) ? __ldg(xrow + (k0 >> 3)) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int c = 0; c < NCHUNK; ++c) {
+        hm[c] = lane_max(v[c]);
+        hrow = __hmax(hrow, hm[c]);
+      }
     }
     float sb = 1.0f, invb = 1.0f, thr = 0.f;
     if (p.branch_qmax > 0) {
@@ -124,10 +140,18 @@ __global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams 
       if (lane == 0) { sXb_s[rl] = sb; p.sXb[m] = sb; }
     }
     // ---- pass B: group scales, 4-bit codes (a1) and branch codes (a2)
-#pragma unroll
+#pragma unroll(RELOAD ? 3 : NCHUNK)
     for (int c = 0; c < NCHUNK; ++c) {
       const int k0 = c * 256 + lane * 8;
-      float a = __half2float(hm[c]);
+      uint4 vc;
+      float a;
+      if constexpr (RELOAD) {
+        vc = (k0 < p.K) ? __ldg(xrow + (k0 >> 3)) : make_uint4(0, 0, 0, 0);
+        a = __half2float(lane_max(vc));
+      } else {
+        vc = v[c];
+        a = __half2float(hm[c]);
+      }
       a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
       a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
       a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 4));
@@ -138,7 +162,7 @@ __global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams 
           const unsigned short sbits = __half_as_ushort(s16);
           if (sbits == 0) s16 = __ushort_as_half((unsigned short)1);             // floor 2^-24
           const float s = __half2float(s16);
-          const __half2* h2 = reinterpret_cast<const __half2*>(&v[c]);
+          const __half2* h2 = reinterpret_cast<const __half2*>(&vc);
           float x[8], q[8], t[8];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
@@ -272,17 +296,17 @@ __global__ void __launch_bounds__(256) lq_down_f16_kernel(const __half* __restri
   if (lane == 0) sT[m] = 1.0f;
 }
 
-template <int NCHUNK, int WARPS>
+template <int NCHUNK, int WARPS, bool RELOAD>
 cudaError_t launch_quant(const QuantParams& p, size_t smem, cudaStream_t st) {
   static bool attr_set[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
   if (smem > 48 * 1024 && !attr_set[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(lq_quant_kernel<NCHUNK, WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(lq_quant_kernel<NCHUNK, WARPS, RELOAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
     attr_set[dev & 63] = true;
   }
-  lq_quant_kernel<NCHUNK, WARPS><<<lq_ceil_div(p.M, ROWS), WARPS * 32, smem, st>>>(p);
+  lq_quant_kernel<NCHUNK, WARPS, RELOAD><<<lq_ceil_div(p.M, ROWS), WARPS * 32, smem, st>>>(p);
   return cudaGetLastError();
 }
 
@@ -307,13 +331,13 @@ lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A,
   const int nchunk = lq_ceil_div(Kpad, 256);
   cudaError_t e;
   if (A->main_kind != LQ_KIND_E4M3) return LQ_ERR_UNSUPPORTED;
-  if (nchunk <= 2) e = launch_quant<2, 16>(p, smem, st);        // one row per warp while the row fits 128 registers
-  else if (nchunk <= 5) e = launch_quant<5, 16>(p, smem, st);
-  else if (nchunk <= 9) e = launch_quant<9, 16>(p, smem, st);
-  else if (nchunk <= 12) e = launch_quant<12, 8>(p, smem, st);
-  else if (nchunk <= 18) e = launch_quant<18, 8>(p, smem, st);
-  else if (nchunk <= 22) e = launch_quant<22, 8>(p, smem, st);
-  else if (nchunk <= 32) e = launch_quant<32, 8>(p, smem, st);
+  if (nchunk <= 2) e = launch_quant<2, 16, false>(p, smem, st);        // the row stays in registers (one warp per row)
+  else if (nchunk <= 5) e = launch_quant<5, 16, false>(p, smem, st);
+  else if (nchunk <= 9) e = launch_quant<9, 16, true>(p, smem, st);     // longer rows: read twice, second time from the L2
+  else if (nchunk <= 12) e = launch_quant<12, 16, true>(p, smem, st);
+  else if (nchunk <= 18) e = launch_quant<18, 16, true>(p, smem, st);
+  else if (nchunk <= 22) e = launch_quant<22, 16, true>(p, smem, st);
+  else if (nchunk <= 32) e = launch_quant<32, 16, true>(p, smem, st);
   else return LQ_ERR_UNSUPPORTED;
   if (lq_note_cuda(e) != cudaSuccess) return LQ_ERR_CUDA;
   if (L->f16_branch) {
