@@ -171,7 +171,9 @@ def workload_config(wl, args):
                         f"main W4A4 SINT4 group 64, branch {wl.branch}" if wl.config in (1, 2) else f"config{wl.config}",
             "rows": wl.M, "rank": wl.rank, "branch": wl.branch, "layers": [s.name for s in wl.layers],
             "calibration_steps": args.calib_steps,
-            "l2": "L2 flushed (256 MiB write) before every timed step; layers inside a step run back to back",
+            "l2": ("L2 flushed (256 MiB write) before every timed step; layers inside a step run back to back"
+                   if args.l2 == "flush" else
+                   "no explicit flush: one step reads 132 MB of X and writes 170 MB of Y plus 66 MB of codes, the L2 holds 126 MB"),
             "parallelism": f"rows sharded x{args.gpus}, no collective"}
 
 
@@ -238,7 +240,8 @@ def run_ours(args):
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
 
     def step(timed=None):
-        flush.zero_()
+        if args.l2 == "flush":
+            flush.zero_()
         if timed is not None:
             timed["s"].record()
         for i, L in enumerate(layers):
@@ -367,6 +370,8 @@ def main():
     ap.add_argument("--branch", default=None)
     ap.add_argument("--calib-steps", type=int, default=2, dest="calib_steps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--l2", default="flush", choices=["flush", "working-set"],
+                    help="flush: write 256 MiB before every step; working-set: rely on one step touching more than the L2 holds")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
