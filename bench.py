@@ -269,11 +269,31 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+        t_wait = time.perf_counter()          # nvidia-smi needs a moment before its first line: keep the GPU busy meanwhile
+        while not sampler.rows and time.perf_counter() - t_wait < 3.0:
+            step()
+            torch.cuda.synchronize()
     barrier()
+    n_before = len(sampler.rows)
+    t_timed = time.perf_counter()
     for t in timers:
         step(t)
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    timed_wall = time.perf_counter() - t_timed
+    clocks = None
+    if rank == 0:
+        # The timed region of a short run is over before nvidia-smi (one line per 100 ms) reports: repeat the same
+        # steps, untimed, until at least 1.5 s of this load have been sampled.
+        extended = False
+        while time.perf_counter() - t_timed < 1.5:
+            extended = True
+            step()
+            torch.cuda.synchronize()
+        sampler.rows = sampler.rows[n_before:]
+        clocks = sampler.stop()
+        clocks["window"] = (f"timed region of {timed_wall * 1e3:.0f} ms" +
+                            (" plus untimed repeats of the same steps up to 1.5 s" if extended else ""))
+    barrier()
     step_ms = [t["s"].elapsed_time(t["e"]) for t in timers]
     gemm_ms = [sum(a.elapsed_time(b) for a, b in zip(t["g0"], t["g1"])) for t in timers]
     quant_ms = [sum(a.elapsed_time(b) for a, b in zip(t["q0"], t["g0"])) for t in timers]
