@@ -132,9 +132,12 @@ lq_status lq_linear_forward(const lq_layer* layer, const lq_act* act, void* Y_de
                             lq_out_dtype dtype, void* cuda_stream);
 
 /* Whole path from host memory: copies X to the device, runs lq_quantize_act and
- * lq_linear_forward, copies Y back and waits for it.  X_f16_host [M][K], Y_host [M][N];
- * pinned host memory makes the copies asynchronous but is not required.  Staging buffers
- * inside `act` are allocated on the first call. */
+ * lq_linear_forward, copies Y back and waits for it.  X_f16_host [M][K], Y_host [M][N].
+ * Rows are independent, so for M >= 1024 the call is pipelined over four row chunks: one chunk
+ * is computed on `cuda_stream` while the next travels host -> device and the previous one
+ * device -> host on two internal copy streams (this needs pinned host memory to overlap;
+ * pageable memory works but serialises).  Staging buffers, streams and events inside `act`
+ * are created on the first call.  Afterwards `act` holds the codes of all M rows. */
 lq_status lq_linear_forward_host(const lq_layer* layer, lq_act* act, const void* X_f16_host,
                                  int32_t M, void* Y_host, lq_out_dtype dtype, void* cuda_stream);
 

@@ -379,6 +379,11 @@ extern "C" lq_status lq_act_free(lq_act* A) {
   cudaSetDevice(A->device);
   cudaFree(A->d_qx8); cudaFree(A->d_sx); cudaFree(A->d_qb); cudaFree(A->d_sXb); cudaFree(A->d_tq); cudaFree(A->d_sT);
   cudaFree(A->d_Xstage); cudaFree(A->d_Ystage);
+  if (A->pipe_ready) {
+    cudaStreamDestroy(A->s_h2d); cudaStreamDestroy(A->s_d2h);
+    for (int c = 0; c < LQ_HOST_CHUNKS; ++c) { cudaEventDestroy(A->ev_x[c]); cudaEventDestroy(A->ev_y[c]); }
+    cudaEventDestroy(A->ev_begin); cudaEventDestroy(A->ev_end);
+  }
   delete A;
   return LQ_OK;
 }
@@ -421,12 +426,56 @@ extern "C" lq_status lq_linear_forward_host(const lq_layer* L, lq_act* A, const 
     if (cudaMalloc(&A->d_Ystage, ybytes) != cudaSuccess) return LQ_ERR_ALLOC;
     A->ystage_bytes = ybytes;
   }
-  CUDA_OK(cudaMemcpyAsync(A->d_Xstage, Xh, (size_t)M * A->K * 2, cudaMemcpyHostToDevice, st));
-  lq_status s = lq_quantize_act(L, A->d_Xstage, M, A, stream);
-  if (s != LQ_OK) return s;
-  s = lq_linear_forward(L, A, A->d_Ystage, dt, stream);
-  if (s != LQ_OK) return s;
-  CUDA_OK(cudaMemcpyAsync(Yh, A->d_Ystage, (size_t)M * A->N * (dt == LQ_OUT_F32 ? 4 : 2), cudaMemcpyDeviceToHost, st));
+  // Rows are independent, so the call is pipelined over row chunks: while chunk c is computed on the caller's
+  // stream, chunk c+1 travels host -> device and chunk c-1 device -> host on two copy streams.
+  if (!A->pipe_ready) {
+    CUDA_OK(cudaStreamCreateWithFlags(&A->s_h2d, cudaStreamNonBlocking));
+    CUDA_OK(cudaStreamCreateWithFlags(&A->s_d2h, cudaStreamNonBlocking));
+    for (int c = 0; c < LQ_HOST_CHUNKS; ++c) {
+      CUDA_OK(cudaEventCreateWithFlags(&A->ev_x[c], cudaEventDisableTiming));
+      CUDA_OK(cudaEventCreateWithFlags(&A->ev_y[c], cudaEventDisableTiming));
+    }
+    CUDA_OK(cudaEventCreateWithFlags(&A->ev_begin, cudaEventDisableTiming));
+    CUDA_OK(cudaEventCreateWithFlags(&A->ev_end, cudaEventDisableTiming));
+    A->pipe_ready = true;
+  }
+  const int nchunk = M >= LQ_HOST_CHUNKS * 2 * LQ_BM ? LQ_HOST_CHUNKS : 1;
+  const int rows_per = lq_round_up(lq_ceil_div(M, nchunk), LQ_BM);
+  const size_t esz = dt == LQ_OUT_F32 ? 4 : 2;
+  CUDA_OK(cudaEventRecord(A->ev_begin, st));                  // copies start after what the caller queued before
+  CUDA_OK(cudaStreamWaitEvent(A->s_h2d, A->ev_begin, 0));
+  CUDA_OK(cudaStreamWaitEvent(A->s_d2h, A->ev_begin, 0));
+  for (int c = 0; c < nchunk; ++c) {
+    const int m0 = c * rows_per;
+    if (m0 >= M) break;
+    const int Mc = M - m0 < rows_per ? M - m0 : rows_per;
+    const uint8_t* xh = (const uint8_t*)Xh + (size_t)m0 * A->K * 2;
+    uint8_t* xd = (uint8_t*)A->d_Xstage + (size_t)m0 * A->K * 2;
+    uint8_t* yd = (uint8_t*)A->d_Ystage + (size_t)m0 * A->N * esz;
+    CUDA_OK(cudaMemcpyAsync(xd, xh, (size_t)Mc * A->K * 2, cudaMemcpyHostToDevice, A->s_h2d));
+    CUDA_OK(cudaEventRecord(A->ev_x[c], A->s_h2d));
+    CUDA_OK(cudaStreamWaitEvent(st, A->ev_x[c], 0));
+    // a view of the activation record that starts at row m0 (m0 is a multiple of the row tile)
+    lq_act V = *A;
+    V.M = Mc; V.M_max = Mc;
+    V.d_qx8 = A->d_qx8 + (size_t)m0 * A->Kpad;
+    V.d_qb = A->d_qb + (size_t)m0 * A->Kpad;
+    V.d_sx = A->d_sx + m0;                                     // [Gpad][Mpad]: the row stride stays Mpad
+    V.d_sXb = A->d_sXb + m0;
+    V.d_tq = A->d_tq + (size_t)m0 * LQ_RCONT;
+    V.d_sT = A->d_sT + m0;
+    lq_status s;
+    if ((s = make_tmap_bytes(&V.tmA, V.d_qx8, (uint64_t)(A->Mpad - m0), A->Kpad, LQ_BM)) != LQ_OK) return s;
+    if ((s = make_tmap_bytes(&V.tmT, V.d_tq, (uint64_t)(A->Mpad - m0), LQ_RCONT, LQ_BM)) != LQ_OK) return s;
+    if ((s = lq_launch_quantize(L, xd, Mc, &V, st)) != LQ_OK) return s;
+    if ((s = lq_launch_gemm(L, &V, yd, dt, st)) != LQ_OK) return s;
+    CUDA_OK(cudaEventRecord(A->ev_y[c], st));
+    CUDA_OK(cudaStreamWaitEvent(A->s_d2h, A->ev_y[c], 0));
+    CUDA_OK(cudaMemcpyAsync((uint8_t*)Yh + (size_t)m0 * A->N * esz, yd, (size_t)Mc * A->N * esz, cudaMemcpyDeviceToHost, A->s_d2h));
+  }
+  A->M = M;
+  CUDA_OK(cudaEventRecord(A->ev_end, A->s_d2h));
+  CUDA_OK(cudaStreamWaitEvent(st, A->ev_end, 0));
   CUDA_OK(cudaStreamSynchronize(st));
   return LQ_OK;
 }

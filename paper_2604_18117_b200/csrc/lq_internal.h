@@ -16,6 +16,7 @@
 #define LQ_RCONT 128         // bytes per row of the branch containers (tq, L2q): rank <= 128
 #define LQ_MAX_K 8192
 #define LQ_MAX_RANK 128
+#define LQ_HOST_CHUNKS 4       // row chunks lq_linear_forward_host overlaps (copy in / compute / copy out)
 
 // role identifiers reported through the device status word
 enum { LQ_STAGE_NONE = 0, LQ_STAGE_PRODUCER = 1, LQ_STAGE_MMA = 2, LQ_STAGE_DRAIN = 3, LQ_STAGE_TEARDOWN = 4 };
@@ -74,6 +75,9 @@ struct lq_act {
   void* d_Xstage;              // lazily allocated staging for lq_linear_forward_host
   void* d_Ystage;
   size_t ystage_bytes;
+  cudaStream_t s_h2d, s_d2h;   // copy streams of lq_linear_forward_host's row-chunk pipeline (created on first use)
+  cudaEvent_t ev_x[LQ_HOST_CHUNKS], ev_y[LQ_HOST_CHUNKS], ev_begin, ev_end;
+  bool pipe_ready;
   CUtensorMap tmA;             // over d_qx8, box [LQ_BM][128B], 128B swizzle
   CUtensorMap tmT;             // over d_tq,  box [LQ_BM][128B], 128B swizzle
 };

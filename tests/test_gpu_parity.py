@@ -153,3 +153,40 @@ def test_config0_full_calibration():
     assert min(trace) < trace[0]
     e32, e16 = _check(layer, X)
     print(f"config0 rel err fp32 {e32:.3e} fp16 {e16:.3e}")
+
+
+def test_host_entry_point_pipelines_row_chunks():
+    """lq_linear_forward_host overlaps copy-in, compute and copy-out over row chunks; the result must be the
+    same as one lq_quantize_act + lq_linear_forward over all rows (bit for bit: rows are independent), and the
+    activation record must hold every chunk's codes."""
+    import torch
+    from tests.helpers import import_oracle_layer
+    rng = np.random.default_rng(6)
+    M, K, N, r = 1300, 1152, 392, 32                       # four chunks, the last one ragged; N not a multiple of 128
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    layer = _random_layer(rng, K, N, r, "w8a8")
+    ref = O.forward(X, layer)
+    h, cfg = import_oracle_layer(layer)
+    B.lq_layer_to_device(h, 0)
+    act = B.lq_act_create(h, M, 0)
+    try:
+        st = torch.cuda.current_stream().cuda_stream
+        Xp = torch.from_numpy(X).pin_memory()
+        for dtype, tdt, tol in ((B.OUT_F32, torch.float32, TOL_F32), (B.OUT_F16, torch.float16, TOL_F16)):
+            Yp = torch.full((M, N), float("nan"), dtype=tdt).pin_memory()
+            B.lq_linear_forward_host(h, act, Xp.data_ptr(), M, Yp.data_ptr(), dtype, st)
+            assert B.lq_get_device_status(0)[0] == 0
+            Yh = Yp.numpy().copy()
+            Xd = torch.from_numpy(X).cuda()
+            Yd = torch.full((M, N), float("nan"), dtype=tdt, device="cuda")
+            B.lq_quantize_act(h, Xd.data_ptr(), M, act, st)
+            B.lq_linear_forward(h, act, Yd.data_ptr(), dtype, st)
+            torch.cuda.synchronize()
+            assert np.array_equal(Yh, Yd.cpu().numpy())
+            assert rel_fro(Yh, ref["Y"]) <= tol
+        B.lq_linear_forward_host(h, act, Xp.data_ptr(), M, Yp.data_ptr(), B.OUT_F16, st)
+        ex = B.lq_act_export(act, M, cfg, st)
+        assert_codes_equal(ex, ref, "w8a8", with_qb=False)
+    finally:
+        B.lq_act_free(act)
+        B.lq_layer_free(h)
