@@ -208,9 +208,8 @@ def run_ours(args):
     from paper_2604_18117_b200 import binding as B
     from paper_2604_18117_b200 import build as BUILD
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2604_18117_b200 import dist_util as D
+    world, rank, local = D.env_ranks()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local)
@@ -224,7 +223,7 @@ def run_ours(args):
 
     layers = []
     for spec in wl.layers:
-        Xh, W, bias = I.layer_inputs(wl, spec, seed=rank, with_bias=True)
+        Xh, W, bias = I.layer_inputs(wl, spec, seed=D.shard_seed(0, rank), with_bias=True)
         cfg = B.lq_config_default(spec.K, spec.N, r, wl.branch)
         cfg.steps = args.calib_steps
         h, _ = B.lq_calibrate(cfg, W, bias)
@@ -309,10 +308,7 @@ def run_ours(args):
     code, stage = B.lq_get_device_status(local)
     if code != 0:
         raise SystemExit(f"device status {code} (stage {stage}) after the timed region")
-    tmax = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-    total_ms_max = float(tmax.item())
+    total_ms_max = D.max_over_ranks(total_ms, world, dev)
 
     # end to end: pinned host X -> device -> K1 -> K2 -> pinned host Y, every step
     def e2e_step():
@@ -328,10 +324,7 @@ def run_ours(args):
         e2e_step()
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_s = float(te.item())
+    e2e_s = D.max_over_ranks(e2e_s, world, dev)
 
     if rank == 0:
         peaks = measured_peaks()
@@ -344,13 +337,13 @@ def run_ours(args):
                        for L in layers)
         quant_avg_ms = float(np.mean(quant_ms))
         line = {
-            "metric": METRIC, "value": world * ops_step * args.steps / (total_ms_max * 1e-3) / 1e12, "unit": UNIT,
+            "metric": METRIC, "value": D.job_throughput(ops_step, args.steps, total_ms_max, world) / 1e12, "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": total_ms_max / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "e4m3 (exact int4 codes) / int8 operands, fp32 accumulate", "data": "synthetic",
             "config": workload_config(wl, args),
-            "tokens_per_s": world * M * args.steps / (total_ms_max * 1e-3),
-            "e2e": {"value": world * ops_step * e2e_steps / e2e_s / 1e12, "unit": UNIT,
+            "tokens_per_s": D.job_throughput(M, args.steps, total_ms_max, world),
+            "e2e": {"value": D.job_throughput(ops_step, e2e_steps, e2e_s * 1e3, world) / 1e12, "unit": UNIT,
                     "h2d_bytes_per_step": int(sum(M * L["spec"].K * 2 for L in layers)),
                     "d2h_bytes_per_step": int(sum(M * L["spec"].N * 2 for L in layers)),
                     "ms_per_step": e2e_s / e2e_steps * 1e3},

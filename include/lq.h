@@ -180,6 +180,14 @@ lq_status lq_act_export(const lq_act* act, int8_t* qx, uint16_t* sx, int8_t* qb,
  * the device. */
 lq_status lq_get_device_status(int device, int32_t* code, int32_t* stage);
 
+/* Self-test of the kernels' failure detection (the paper has no counterpart).  Every wait inside the
+ * kernels is bounded: a role that waits longer than its limit records LQ_ERR_TIMEOUT and its
+ * stage in the status word, and the kernel returns instead of hanging.  This call launches a
+ * one-warp kernel that waits, with a limit of about 0.1 s, on a barrier that nothing ever arrives
+ * on; afterwards lq_get_device_status must report {LQ_ERR_TIMEOUT, 4} and the device stays usable.
+ * Asynchronous on `cuda_stream`. */
+lq_status lq_selftest_wait_timeout(int device, void* cuda_stream);
+
 /* Tuning knobs for experiments, e.g. "main_kind" (0 = int8 operands, 1 = E4M3-carried
  * codes).  Returns INVALID_ARG for an unknown name.  Affects layers uploaded afterwards. */
 lq_status lq_set_option(const char* name, int32_t value);

@@ -55,6 +55,7 @@ _SIGNATURES = {
     "lq_act_export": [C.c_void_p] * 8,
     "lq_get_device_status": [C.c_int, C.POINTER(C.c_int32), C.POINTER(C.c_int32)],
     "lq_set_option": [C.c_char_p, C.c_int32],
+    "lq_selftest_wait_timeout": [C.c_int, C.c_void_p],
 }
 EXPORTED = tuple(_SIGNATURES) + ("lq_status_string", "lq_last_cuda_error", "lq_version")
 
@@ -215,6 +216,10 @@ def lq_get_device_status(device: int = 0):
     code, stage = C.c_int32(), C.c_int32()
     _check(lib().lq_get_device_status(device, C.byref(code), C.byref(stage)), "lq_get_device_status")
     return code.value, stage.value
+
+
+def lq_selftest_wait_timeout(device: int = 0, stream: int = 0):
+    _check(lib().lq_selftest_wait_timeout(device, C.c_void_p(stream)), "lq_selftest_wait_timeout")
 
 
 def lq_set_option(name: str, value: int):

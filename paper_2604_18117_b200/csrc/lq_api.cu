@@ -251,6 +251,10 @@ extern "C" lq_status lq_get_device_status(int device, int32_t* code, int32_t* st
   return LQ_OK;
 }
 
+extern "C" lq_status lq_selftest_wait_timeout(int device, void* stream) {
+  return lq_launch_wait_probe(device, (cudaStream_t)stream);
+}
+
 // ---- upload ------------------------------------------------------------------------------
 static void layer_free_device(lq_layer* L) {
   if (L->device < 0) return;

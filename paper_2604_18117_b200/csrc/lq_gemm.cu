@@ -97,13 +97,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false when the CTA is aborting or the deadline passed (then it
 // raises the abort flag and records who gave up).
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                            int role) {
+                                            int role, long long limit = WAIT_LIMIT_CYCLES) {
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 0xFF) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      if (clock64() - t0 > limit) {
         *abort_flag = 1;
         if (atomicCAS(status, 0, (int)LQ_ERR_TIMEOUT) == 0) status[1] = role;
         return false;
@@ -502,7 +502,29 @@ lq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier that nothing ever arrives on.
+__global__ void lq_wait_probe_kernel(int32_t* status, long long limit) {
+  __shared__ uint64_t barrier_word;
+  __shared__ int abort_word;
+  const uint32_t bar = smem_u32(&barrier_word);
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    abort_word = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  mbar_wait_slow(bar, 0, &abort_word, status, LQ_STAGE_TEARDOWN, limit);
+}
+
 }  // namespace
+
+lq_status lq_launch_wait_probe(int device, cudaStream_t st) {
+  if (cudaSetDevice(device) != cudaSuccess) return LQ_ERR_CUDA;
+  int32_t* status = lq_device_status_ptr(device);
+  if (!status) return LQ_ERR_CUDA;
+  lq_wait_probe_kernel<<<1, 32, 0, st>>>(status, 200000000ll);   // ~0.1 s
+  return lq_note_cuda(cudaGetLastError()) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
+}
 
 lq_status lq_gemm_prepare(int device) {
   if (cudaSetDevice(device) != cudaSuccess) return LQ_ERR_CUDA;

@@ -91,7 +91,8 @@ int32_t* lq_device_status_ptr(int device);
 // kernels' host launchers (defined in lq_quant.cu / lq_gemm.cu)
 lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A, cudaStream_t st);
 lq_status lq_launch_gemm(const lq_layer* L, const lq_act* A, void* Y, lq_out_dtype dt, cudaStream_t st);
-lq_status lq_gemm_prepare(int device);   // sets the kernel's shared-memory attribute once per device
+lq_status lq_gemm_prepare(int device);
+lq_status lq_launch_wait_probe(int device, cudaStream_t st);   // bounded-wait self-test kernel   // sets the kernel's shared-memory attribute once per device
 
 // byte an MMA operand carries for a 4-bit code q in [-7, 7]
 static inline uint8_t lq_encode_code_host(int q, int kind) {

@@ -190,3 +190,18 @@ def test_host_entry_point_pipelines_row_chunks():
     finally:
         B.lq_act_free(act)
         B.lq_layer_free(h)
+
+
+def test_bounded_wait_reports_timeout_and_device_stays_usable():
+    """Failure detection without a fault: a wait that nothing satisfies runs into its limit, the kernel records
+    LQ_ERR_TIMEOUT (5) with the waiting stage in the status word and returns; the next forward is unaffected."""
+    import torch
+    st = torch.cuda.current_stream().cuda_stream
+    assert B.lq_get_device_status(0)[0] == 0
+    B.lq_selftest_wait_timeout(0, st)
+    code, stage = B.lq_get_device_status(0)                 # synchronises; reading clears the word
+    assert (code, stage) == (5, 4)
+    assert B.lq_get_device_status(0) == (0, 0)
+    rng = np.random.default_rng(7)
+    X = rng.standard_normal((130, 320)).astype(np.float16)
+    _check(_random_layer(rng, 320, 72, 16, "w8a8"), X)
