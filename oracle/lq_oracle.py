@@ -21,6 +21,8 @@ What it follows
   both branches quantized: Figure 1 caption and Appendix A.2 "Quantization".
 * SINT4 format (signed int4, blocks of 64 values, one FP16 scale per block,
   round-to-nearest): Appendix A.3 "Blockwise Formats".
+* MXINT4 format (signed int4, blocks of 32 values, one E8M0 power-of-two scale per
+  block, round-to-nearest): Appendix A.3; used for the residual branch in Table 2.
 
 Readings taken where the paper is silent (each is listed in the design notes):
 symmetric range [-7, 7] with scale = absmax / 7 rounded to fp16; ties to even;
@@ -32,6 +34,10 @@ intermediate) or per output column (the two factors); the intermediate
 and P is recomputed from the quantized factors; Sigma is split evenly between
 L0 and R0; the loss is the mean over K*N entries; Adam uses (0.9, 0.999, 1e-8)
 with bias correction; the best iterate seen is returned.
+
+MXINT4 reading (the paper gives neither range nor exponent rule): codes in [-7, 7],
+scale 2^e with e the smallest integer such that 7 * 2^e >= absmax of the block (no
+clipping), e limited to the E8M0 range [-127, 127], e = -127 for an all-zero block.
 
 Parity unpinned (the paper prints no number for them): the Adam trajectory, the
 split of Sigma between L0 and R0.
@@ -82,6 +88,51 @@ def qgrp(v, group: int = GROUP):
         codes[:, g * group:(g + 1) * group] = np.clip(q, -QMAX4, QMAX4).astype(np.int8)
         scales[:, g] = s
     return codes, scales
+
+
+MX_BLOCK = 32                   # MXINT4 block (Appendix A.3)
+
+
+def qmx(v, block: int = MX_BLOCK):
+    """MXINT4 quantizer along the last axis of a 2-D array.
+
+    Per block of `block` consecutive values (the last may be short): a = max|v|;
+    e = the smallest integer with 7 * 2^e >= a, clamped to [-127, 127] (-127 when a == 0);
+    q = clamp(rint_even(v / 2^e), -7, 7) - the division by a power of two is exact.
+    Returns (codes int8 [R, L], exponents int16 [R, ceil(L/block)]); the scale is 2.0**e.
+    """
+    v = np.asarray(v, dtype=np.float64)
+    R, L = v.shape
+    G = -(-L // block)
+    codes = np.zeros((R, L), dtype=np.int8)
+    exps = np.zeros((R, G), dtype=np.int16)
+    for g in range(G):
+        blk = v[:, g * block:(g + 1) * block]
+        a = np.max(np.abs(blk), axis=1)
+        e = np.full(R, -127, dtype=np.int64)
+        nz = a > 0
+        # frexp: a = m * 2^x with m in [0.5, 1); 7 * 2^e >= a  <=>  e >= x + log2(m / 7)
+        m, x = np.frexp(a[nz])
+        e[nz] = np.where(m <= 7.0 / 8.0, x - 3, x - 2)          # 7 * 2^(x-3) = (7/8) 2^x >= m 2^x  iff  m <= 7/8
+        e = np.clip(e, -127, 127)
+        q = np.rint(blk / np.exp2(e.astype(np.float64))[:, None])
+        codes[:, g * block:(g + 1) * block] = np.clip(q, -QMAX4, QMAX4).astype(np.int8)
+        exps[:, g] = e
+    return codes, exps
+
+
+def deq_mx(codes, exps, block: int = MX_BLOCK):
+    """float64 values q * 2^e of a qmx() result."""
+    R, L = codes.shape
+    s = np.repeat(np.exp2(exps.astype(np.float64)), block, axis=1)[:, :L]
+    return s * codes.astype(np.float64)
+
+
+def q_weight_main_mx(P):
+    """MXINT4 on the residual weight P [K, N]: blocks of 32 along K for each output column n.
+    Returns (Wq int8 [K, N], ew int16 [K/32 blocks, N])."""
+    c, e = qmx(np.asarray(P, dtype=np.float64).T.copy())
+    return c.T.copy(), e.T.copy()
 
 
 def deq_grp(codes, scales, group: int = GROUP):
@@ -152,23 +203,33 @@ def forward(X16, layer, group: int = GROUP):
     """
     X16 = np.asarray(X16, dtype=np.float16)
     M, K = X16.shape
-    Wq, sw = layer["Wq"], layer["sw"]
+    Wq, sw = layer["Wq"], layer.get("sw")
     N = Wq.shape[1]
     G = -(-K // group)
     branch, r = layer["branch"], int(layer["rank"])
     out = {}
     Xf = X16.astype(np.float32)
 
-    qx, sx = qgrp(Xf, group)                                   # (1)
-    out["qx"], out["sx"] = qx, sx
-
     Y = np.zeros((M, N), dtype=np.float64)
     Wq64 = Wq.astype(np.float64)
-    qx64 = qx.astype(np.float64)
-    for g in range(G):                                          # (6) + main part of (8)
-        k0, k1 = g * group, min(K, (g + 1) * group)
-        Pg = qx64[:, k0:k1] @ Wq64[k0:k1, :]                    # exact integers
-        Y += (sx[:, g].astype(np.float64)[:, None] * sw[g, :].astype(np.float64)[None, :]) * Pg
+    if layer.get("main", "sint4") == "mxint4":
+        # MXINT4 main branch: blocks of 32, power-of-two scales 2^ex (activations) and 2^ew (weights)
+        qx, ex = qmx(Xf)                                        # (1)
+        out["qx"], out["ex"] = qx, ex
+        qx64 = qx.astype(np.float64)
+        ew = layer["ew"]
+        for g in range(-(-K // MX_BLOCK)):                      # (6) + main part of (8)
+            k0, k1 = g * MX_BLOCK, min(K, (g + 1) * MX_BLOCK)
+            Pg = qx64[:, k0:k1] @ Wq64[k0:k1, :]                # exact integers
+            Y += np.exp2(ex[:, g].astype(np.float64))[:, None] * np.exp2(ew[g, :].astype(np.float64))[None, :] * Pg
+    else:
+        qx, sx = qgrp(Xf, group)                                # (1)
+        out["qx"], out["sx"] = qx, sx
+        qx64 = qx.astype(np.float64)
+        for g in range(G):                                      # (6) + main part of (8)
+            k0, k1 = g * group, min(K, (g + 1) * group)
+            Pg = qx64[:, k0:k1] @ Wq64[k0:k1, :]                # exact integers
+            Y += (sx[:, g].astype(np.float64)[:, None] * sw[g, :].astype(np.float64)[None, :]) * Pg
 
     if branch != "none" and r > 0:
         if branch == "w16a16":

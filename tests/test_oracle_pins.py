@@ -430,3 +430,110 @@ def test_inputs_are_reproducible_and_shaped():
     assert np.sum(chmax > 25) == 8                               # eight outlier channels
     s3 = I.workload(3)
     assert s3.n_act_outliers(2240) == 22 and s3.n_w_outliers(5600) == 56
+
+
+# --------------------------------------------------------------------------------------
+# MXINT4 (Appendix A.3: signed int4, blocks of 32, E8M0 scale; Table 2 uses it for the residual branch)
+# --------------------------------------------------------------------------------------
+def test_mxint4_hand_examples(golden_dir):
+    cases, cur = [], {}
+    for line in open(os.path.join(golden_dir, "mxint4_hand_examples.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        key, vals = line.split(":")
+        cur[key] = [float(t) for t in vals.split()]
+        if key == "q":
+            cases.append(cur); cur = {}
+    assert len(cases) == 5
+    for c in cases:
+        v = np.zeros((1, 32)); v[0, :len(c["v"])] = c["v"]
+        q, e = O.qmx(v)
+        assert e[0, 0] == int(c["e"][0]), c
+        assert list(q[0, :len(c["q"])]) == [int(t) for t in c["q"]], c
+        assert not q[0, len(c["q"]):].any()
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_mxint4_properties(seed):
+    """Minimal power-of-two scale without clipping, range, half-step error, idempotence (Section 3.2), sign symmetry,
+    blocks independent; the exponent rule is re-derived with exact rational arithmetic."""
+    from fractions import Fraction
+    rng = np.random.default_rng(seed)
+    v = (rng.standard_normal((40, 32 * 5 + 7)) * np.exp2(rng.integers(-12, 8, size=(40, 1)))).astype(np.float16).astype(np.float64)
+    q, e = O.qmx(v)
+    assert q.min() >= -7 and q.max() <= 7
+    s = np.repeat(np.exp2(e.astype(np.float64)), 32, axis=1)[:, :v.shape[1]]
+    assert np.all(np.abs(v - s * q) <= s / 2)                                  # RTN without clipping
+    for r in range(0, 40, 7):
+        for g in range(e.shape[1]):
+            a = Fraction(float(np.abs(v[r, g * 32:(g + 1) * 32]).max()))
+            if a == 0:
+                assert e[r, g] == -127
+                continue
+            ee = int(e[r, g])
+            assert 7 * Fraction(2) ** ee >= a > 7 * Fraction(2) ** (ee - 1)       # smallest admissible exponent
+            assert np.abs(q[r, g * 32:(g + 1) * 32]).max() >= 4                  # so the top code is at least 4
+    q2, e2 = O.qmx(O.deq_mx(q, e))
+    assert np.array_equal(q2, q) and np.array_equal(e2, e)
+    qn, en = O.qmx(-v)
+    assert np.array_equal(qn, -q) and np.array_equal(en, e)
+    w = v.copy(); w[:, 32:64] *= 16
+    qw, ew = O.qmx(w)
+    assert np.array_equal(np.delete(qw, np.s_[32:64], axis=1), np.delete(q, np.s_[32:64], axis=1))
+    assert np.array_equal(ew[:, 1], np.where(e[:, 1] == -127, -127, e[:, 1] + 4)) and np.array_equal(qw[:, 32:64], q[:, 32:64])
+
+
+def test_mxint4_weight_blocks_run_along_K():
+    rng = np.random.default_rng(3)
+    P = rng.standard_normal((96, 5)) * 0.02
+    Wq, ew = O.q_weight_main_mx(P)
+    assert Wq.shape == (96, 5) and ew.shape == (3, 5)
+    for n in range(5):
+        q, e = O.qmx(P[:, n][None, :])
+        assert np.array_equal(q[0], Wq[:, n]) and np.array_equal(e[0], ew[:, n])
+
+
+@pytest.mark.parametrize("branch", ["none", "w8a8", "w4a8"])
+def test_forward_mxint4_brute_force_tiny(branch):
+    """The MXINT4 forward against Python-scalar loops written from the definition: every block's integer dot product
+    times 2^(ex + ew), plus the integer branch, in exact rational arithmetic."""
+    from fractions import Fraction
+    rng = np.random.default_rng(11)
+    M, K, N, r = 3, 80, 4, (0 if branch == "none" else 3)                      # K = 2.5 blocks: a short last block
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    X[:, 5] *= 20
+    layer = {"main": "mxint4", "branch": branch if r else "none", "rank": r, "K": K, "N": N,
+             "bias": (rng.standard_normal(N) * 0.1).astype(np.float16)}
+    layer["Wq"], layer["ew"] = O.q_weight_main_mx(rng.standard_normal((K, N)) * 0.02)
+    if r:
+        bw, _ = O.BRANCH_BITS[branch]
+        layer["L1q"], layer["sL1"] = O.q_factor(rng.standard_normal((K, r)) * 0.05, bw)
+        layer["L2q"], layer["sL2"] = O.q_factor(rng.standard_normal((r, N)) * 0.05, bw)
+    out = O.forward(X, layer)
+    qx, ex = O.qmx(X.astype(np.float64))
+    assert np.array_equal(out["qx"], qx) and np.array_equal(out["ex"], ex)
+    for m in range(M):
+        for n in range(N):
+            y = Fraction(float(layer["bias"][n]))
+            for g in range(3):
+                dot = sum(int(qx[m, k]) * int(layer["Wq"][k, n]) for k in range(g * 32, min(K, g * 32 + 32)))
+                y += Fraction(2) ** (int(ex[m, g]) + int(layer["ew"][g, n])) * dot
+            if r:
+                u = sum(int(out["tq"][m, j]) * int(layer["L2q"][j, n]) for j in range(r))
+                y += Fraction(float(out["sT"][m])) * Fraction(float(layer["sL2"][n])) * u
+            assert abs(float(y) - out["Y"][m, n]) <= 1e-12 * max(1.0, abs(float(y)))
+
+
+def test_forward_mxint4_exact_integer_case():
+    """Integer inputs in [-7, 7] whose block maxima are 7 quantize to themselves with exponent 0 on both sides: Y is the
+    plain integer matrix product."""
+    rng = np.random.default_rng(12)
+    M, K, N = 5, 96, 6
+    X = rng.integers(-7, 8, size=(M, K)).astype(np.float16); X[:, ::32] = 7
+    Wi = rng.integers(-7, 8, size=(K, N)); Wi[::32, :] = 7
+    layer = {"main": "mxint4", "branch": "none", "rank": 0, "K": K, "N": N, "bias": None}
+    layer["Wq"], layer["ew"] = O.q_weight_main_mx(Wi.astype(np.float64))
+    assert not layer["ew"].any() and np.array_equal(layer["Wq"], Wi)
+    out = O.forward(X, layer)
+    assert not out["ex"].any() and np.array_equal(out["Y"], (X.astype(np.int64) @ Wi).astype(np.float64))
