@@ -139,7 +139,7 @@ def lq_layer_info(layer) -> LqConfig:
 
 def lq_layer_export(layer) -> dict:
     cfg = lq_layer_info(layer)
-    K, N, r, G = cfg.K, cfg.N, cfg.rank, -(-cfg.K // GROUP)
+    K, N, r, G = cfg.K, cfg.N, cfg.rank, -(-cfg.K // cfg.group)
     out = {"Wq_packed": np.zeros((K, N // 2), np.uint8), "sw": np.zeros((G, N), np.float16),
            "bias": np.zeros(N, np.float16), "branch": BRANCH_NAME[cfg.branch], "rank": r, "K": K, "N": N}
     L1 = L2 = sL1 = sL2 = None
@@ -197,8 +197,9 @@ def lq_linear_forward_static(layer, X_dev_ptr: int, M: int, Y_dev_ptr: int, dtyp
 
 
 def lq_act_export(act, M: int, cfg: LqConfig, stream: int = 0) -> dict:
-    K, r, G = cfg.K, cfg.rank, -(-cfg.K // GROUP)
-    out = {"qx": np.zeros((M, K), np.int8), "sx": np.zeros((M, G), np.float16)}
+    K, r, G = cfg.K, cfg.rank, -(-cfg.K // cfg.group)
+    # SINT4: fp16 group scales; MXINT4 (group 32): int16 block exponents e (scale 2^e)
+    out = {"qx": np.zeros((M, K), np.int8), "sx": np.zeros((M, G), np.int16 if cfg.group == 32 else np.float16)}
     qb = sXb = tq = sT = None
     if r > 0 and cfg.branch != BRANCH["none"]:
         f16 = cfg.branch == BRANCH["w16a16"]

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblq.so")
-SOURCES = ["lq_api.cu", "lq_quant.cu", "lq_gemm.cu", "lq_noalloc.cu", "lq_calibrate.cpp"]
+SOURCES = ["lq_api.cu", "lq_quant.cu", "lq_gemm.cu", "lq_gemm_mx.cu", "lq_noalloc.cu", "lq_calibrate.cpp"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC,-O2,-fopenmp,-ffp-contract=off", "-cudart", "static",

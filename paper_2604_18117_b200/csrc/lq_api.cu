@@ -78,7 +78,8 @@ static lq_status check_config(const lq_config* c) {
   if (!c) return LQ_ERR_INVALID_ARG;
   if (c->K <= 0 || c->N <= 0 || c->rank < 0) return LQ_ERR_INVALID_ARG;
   if (c->branch < LQ_BRANCH_NONE || c->branch > LQ_BRANCH_W4A8) return LQ_ERR_INVALID_ARG;
-  if (c->group != LQ_GROUP) return LQ_ERR_UNSUPPORTED;
+  if (c->group != LQ_GROUP && c->group != LQ_MX_BLOCK) return LQ_ERR_UNSUPPORTED;
+  if (c->group == LQ_MX_BLOCK && c->branch == LQ_BRANCH_W16A16) return LQ_ERR_UNSUPPORTED;
   if (c->K > LQ_MAX_K || (c->K % 8) != 0) return LQ_ERR_UNSUPPORTED;
   if ((c->N % 8) != 0) return LQ_ERR_UNSUPPORTED;
   if (c->rank > LQ_MAX_RANK) return LQ_ERR_UNSUPPORTED;
@@ -96,7 +97,8 @@ lq_layer* lq_layer_new(const lq_config* cfg) {
   L->r = (cfg->branch == LQ_BRANCH_NONE) ? 0 : cfg->rank;
   if (L->r == 0) L->cfg.branch = LQ_BRANCH_NONE;
   L->cfg.rank = L->r;
-  L->G = lq_ceil_div(L->K, LQ_GROUP);
+  L->mx = cfg->group == LQ_MX_BLOCK;
+  L->G = lq_ceil_div(L->K, cfg->group);
   L->Kpad = lq_round_up(L->K, LQ_KSTAGE);
   L->Gpad = L->Kpad / LQ_GROUP;
   L->Npad = lq_round_up(L->N, LQ_BN);
@@ -106,7 +108,7 @@ lq_layer* lq_layer_new(const lq_config* cfg) {
   L->device = -1;
   L->main_kind = g_lq_main_kind;
   L->d_Wq8 = nullptr; L->d_sw = nullptr; L->d_L1f = nullptr; L->d_L1h = nullptr; L->d_sL1 = nullptr;
-  L->d_L2c = nullptr; L->d_sL2 = nullptr; L->d_bias = nullptr;
+  L->d_L2c = nullptr; L->d_sL2 = nullptr; L->d_bias = nullptr; L->d_sfb = nullptr;
   return L;
 }
 
@@ -133,8 +135,12 @@ extern "C" lq_status lq_layer_import(const lq_config* cfg, const uint8_t* Wq_pac
         L->Wq[(size_t)k * N + 2 * j + 1] = (int8_t)hi;
       }
     L->sw.assign(sw, sw + (size_t)G * N);
-    for (size_t i = 0; i < L->sw.size(); ++i)
-      if (!isfinite(h2f(L->sw[i]))) { delete L; return LQ_ERR_NUMERIC; }
+    for (size_t i = 0; i < L->sw.size(); ++i) {
+      const float v = h2f(L->sw[i]);
+      if (!isfinite(v)) { delete L; return LQ_ERR_NUMERIC; }
+      int x = 0;
+      if (L->mx && !(v > 0.f && frexpf(v, &x) == 0.5f)) { delete L; return LQ_ERR_INVALID_ARG; }   // MXINT4 scales are powers of two
+    }
     if (L->integer_branch) {
       const int qm = (1 << (lq_branch_wbits(L->cfg.branch) - 1)) - 1;
       const int8_t* a = (const int8_t*)L1; const int8_t* b = (const int8_t*)L2;
@@ -260,9 +266,9 @@ static void layer_free_device(lq_layer* L) {
   if (L->device < 0) return;
   cudaSetDevice(L->device);
   cudaFree(L->d_Wq8); cudaFree(L->d_sw); cudaFree(L->d_L1f); cudaFree(L->d_L1h); cudaFree(L->d_sL1);
-  cudaFree(L->d_L2c); cudaFree(L->d_sL2); cudaFree(L->d_bias);
+  cudaFree(L->d_L2c); cudaFree(L->d_sL2); cudaFree(L->d_bias); cudaFree(L->d_sfb);
   L->d_Wq8 = nullptr; L->d_sw = nullptr; L->d_L1f = nullptr; L->d_L1h = nullptr; L->d_sL1 = nullptr;
-  L->d_L2c = nullptr; L->d_sL2 = nullptr; L->d_bias = nullptr;
+  L->d_L2c = nullptr; L->d_sL2 = nullptr; L->d_bias = nullptr; L->d_sfb = nullptr;
   L->device = -1;
 }
 
@@ -288,10 +294,22 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
     for (int k = 0; k < K; ++k)
       for (int n = 0; n < N; ++n) w8[(size_t)n * Kpad + k] = lq_encode_code_host(L->Wq[(size_t)k * N + n], L->main_kind);
     if ((st = upload(&L->d_Wq8, w8)) != LQ_OK) return st;
-    std::vector<float> swf((size_t)Gpad * Npad, 0.f);
-    for (int g = 0; g < G; ++g)
-      for (int n = 0; n < N; ++n) swf[(size_t)g * Npad + n] = h2f(L->sw[(size_t)g * N + n]);
-    if ((st = upload(&L->d_sw, swf)) != LQ_OK) return st;
+    if (L->mx) {
+      // E8M0 bytes (exponent + 127) in the layout the block-scaled MMA reads from tensor memory; 127 = 2^0 for padding
+      std::vector<uint8_t> sfb((size_t)(Npad / 128) * (Kpad / 128) * 512, 127);
+      for (int g = 0; g < G; ++g)
+        for (int n = 0; n < N; ++n) {
+          int x = 0;
+          frexpf(h2f(L->sw[(size_t)g * N + n]), &x);              // 2^e = 0.5 * 2^(e+1)
+          sfb[lq_sf_offset(n, g, Kpad)] = (uint8_t)(x - 1 + 127);
+        }
+      if ((st = upload(&L->d_sfb, sfb)) != LQ_OK) return st;
+    } else {
+      std::vector<float> swf((size_t)Gpad * Npad, 0.f);
+      for (int g = 0; g < G; ++g)
+        for (int n = 0; n < N; ++n) swf[(size_t)g * Npad + n] = h2f(L->sw[(size_t)g * N + n]);
+      if ((st = upload(&L->d_sw, swf)) != LQ_OK) return st;
+    }
     std::vector<float> bias((size_t)Npad, 0.f);
     if (L->has_bias) for (int n = 0; n < N; ++n) bias[n] = h2f(L->bias[n]);
     if ((st = upload(&L->d_bias, bias)) != LQ_OK) return st;
@@ -334,6 +352,7 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
   if ((st = make_tmap_bytes(&L->tmL2, L->d_L2c, Npad, LQ_RCONT, LQ_BN)) != LQ_OK) return st;
   if (!lq_device_status_ptr(device)) return LQ_ERR_CUDA;
   if ((st = lq_gemm_prepare(device)) != LQ_OK) return st;
+  if (L->mx && (st = lq_gemm_mx_prepare(device)) != LQ_OK) return st;
   return LQ_OK;
 }
 
@@ -352,6 +371,7 @@ extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device,
   if (!A) return LQ_ERR_ALLOC;
   memset(A, 0, sizeof(*A));
   A->K = L->K; A->N = L->N; A->r = L->r; A->G = L->G; A->Kpad = L->Kpad; A->Gpad = L->Gpad;
+  A->mx = L->mx;
   A->branch = L->cfg.branch; A->M_max = M_max; A->Mpad = lq_round_up(M_max, LQ_BM);
   A->device = device; A->main_kind = L->main_kind; A->M = 0;
   if (cudaSetDevice(device) != cudaSuccess) { delete A; return LQ_ERR_CUDA; }
@@ -361,7 +381,8 @@ extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device,
             cudaMalloc((void**)&A->d_qb, Mp * Kp) == cudaSuccess &&
             cudaMalloc((void**)&A->d_sXb, Mp * sizeof(float)) == cudaSuccess &&
             cudaMalloc((void**)&A->d_tq, Mp * LQ_RCONT) == cudaSuccess &&
-            cudaMalloc((void**)&A->d_sT, Mp * sizeof(float)) == cudaSuccess;
+            cudaMalloc((void**)&A->d_sT, Mp * sizeof(float)) == cudaSuccess &&
+            (!A->mx || cudaMalloc((void**)&A->d_sfa, (Mp / 128) * (Kp / 128) * 512) == cudaSuccess);
   if (!ok) { lq_act_free(A); return LQ_ERR_ALLOC; }
   // padding rows/columns are read by the GEMM's tiles: start from defined contents
   cudaMemset(A->d_qx8, 0, Mp * Kp);
@@ -370,6 +391,7 @@ extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device,
   cudaMemset(A->d_sXb, 0, Mp * sizeof(float));
   cudaMemset(A->d_tq, 0, Mp * LQ_RCONT);
   cudaMemset(A->d_sT, 0, Mp * sizeof(float));
+  if (A->mx) cudaMemset(A->d_sfa, 127, (Mp / 128) * (Kp / 128) * 512);
   lq_status st;
   if ((st = make_tmap_bytes(&A->tmA, A->d_qx8, Mp, Kp, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
   if ((st = make_tmap_bytes(&A->tmT, A->d_tq, Mp, LQ_RCONT, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
@@ -381,7 +403,7 @@ extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device,
 extern "C" lq_status lq_act_free(lq_act* A) {
   if (!A) return LQ_ERR_INVALID_ARG;
   cudaSetDevice(A->device);
-  cudaFree(A->d_qx8); cudaFree(A->d_sx); cudaFree(A->d_qb); cudaFree(A->d_sXb); cudaFree(A->d_tq); cudaFree(A->d_sT);
+  cudaFree(A->d_qx8); cudaFree(A->d_sx); cudaFree(A->d_qb); cudaFree(A->d_sXb); cudaFree(A->d_tq); cudaFree(A->d_sT); cudaFree(A->d_sfa);
   cudaFree(A->d_Xstage); cudaFree(A->d_Ystage);
   if (A->pipe_ready) {
     cudaStreamDestroy(A->s_h2d); cudaStreamDestroy(A->s_d2h);
@@ -394,7 +416,7 @@ extern "C" lq_status lq_act_free(lq_act* A) {
 
 static bool act_matches(const lq_layer* L, const lq_act* A) {
   return L && A && L->device == A->device && L->device >= 0 && L->K == A->K && L->N == A->N && L->r == A->r &&
-         L->cfg.branch == A->branch && L->main_kind == A->main_kind;
+         L->cfg.branch == A->branch && L->main_kind == A->main_kind && L->mx == A->mx;
 }
 
 extern "C" lq_status lq_quantize_act(const lq_layer* L, const void* X, int32_t M, lq_act* A, void* stream) {
@@ -412,7 +434,7 @@ extern "C" lq_status lq_linear_forward(const lq_layer* L, const lq_act* A, void*
   if (A->M <= 0) return LQ_ERR_INVALID_ARG;
   if (dt != LQ_OUT_F16 && dt != LQ_OUT_F32) return LQ_ERR_INVALID_ARG;
   if (((uintptr_t)Y & 15) != 0) return LQ_ERR_INVALID_ARG;
-  return lq_launch_gemm(L, A, Y, dt, (cudaStream_t)stream);
+  return L->mx ? lq_launch_gemm_mx(L, A, Y, dt, (cudaStream_t)stream) : lq_launch_gemm(L, A, Y, dt, (cudaStream_t)stream);
 }
 
 extern "C" lq_status lq_linear_forward_host(const lq_layer* L, lq_act* A, const void* Xh, int32_t M, void* Yh,
@@ -468,11 +490,12 @@ extern "C" lq_status lq_linear_forward_host(const lq_layer* L, lq_act* A, const 
     V.d_sXb = A->d_sXb + m0;
     V.d_tq = A->d_tq + (size_t)m0 * LQ_RCONT;
     V.d_sT = A->d_sT + m0;
+    if (A->mx) V.d_sfa = A->d_sfa + (size_t)(m0 / 128) * (A->Kpad / 128) * 512;
     lq_status s;
     if ((s = make_tmap_bytes(&V.tmA, V.d_qx8, (uint64_t)(A->Mpad - m0), A->Kpad, LQ_BM)) != LQ_OK) return s;
     if ((s = make_tmap_bytes(&V.tmT, V.d_tq, (uint64_t)(A->Mpad - m0), LQ_RCONT, LQ_BM)) != LQ_OK) return s;
     if ((s = lq_launch_quantize(L, xd, Mc, &V, st)) != LQ_OK) return s;
-    if ((s = lq_launch_gemm(L, &V, yd, dt, st)) != LQ_OK) return s;
+    if ((s = (L->mx ? lq_launch_gemm_mx(L, &V, yd, dt, st) : lq_launch_gemm(L, &V, yd, dt, st))) != LQ_OK) return s;
     CUDA_OK(cudaEventRecord(A->ev_y[c], st));
     CUDA_OK(cudaStreamWaitEvent(A->s_d2h, A->ev_y[c], 0));
     CUDA_OK(cudaMemcpyAsync((uint8_t*)Yh + (size_t)m0 * A->N * esz, yd, (size_t)Mc * A->N * esz, cudaMemcpyDeviceToHost, A->s_d2h));
@@ -510,7 +533,15 @@ extern "C" lq_status lq_act_export(const lq_act* A, int8_t* qx, uint16_t* sx, in
       for (int m = 0; m < M; ++m)
         for (int k = 0; k < K; ++k) qx[(size_t)m * K + k] = (int8_t)decode_code(h[m * Kp + k], A->main_kind);
     }
-    if (sx) {
+    if (sx && A->mx) {
+      std::vector<uint8_t> h((Mp / 128) * (Kp / 128) * 512);
+      CUDA_OK(cudaMemcpy(h.data(), A->d_sfa, h.size(), cudaMemcpyDeviceToHost));
+      for (int m = 0; m < M; ++m)
+        for (int g = 0; g < G; ++g) {
+          const int e = (int)h[lq_sf_offset(m, g, (int)Kp)] - 127;
+          sx[(size_t)m * G + g] = (uint16_t)(int16_t)e;            // MXINT4: the block exponent itself (scale 2^e)
+        }
+    } else if (sx) {
       std::vector<float> h((size_t)A->Gpad * Mp);
       CUDA_OK(cudaMemcpy(h.data(), A->d_sx, h.size() * sizeof(float), cudaMemcpyDeviceToHost));
       for (int m = 0; m < M; ++m)

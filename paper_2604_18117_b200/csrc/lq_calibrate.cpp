@@ -230,17 +230,30 @@ void svd_top_r(const std::vector<double>& W, int K, int N, int r, uint64_t seed,
 
 // SINT4 along K (axis 0) per output column of A [K][N]: writes codes and half-bit scales and
 // returns the dequantized matrix in Dq (may be null).  fp32 arithmetic as in the kernels.
-void quant_main(const std::vector<double>& A, int K, int N, int8_t* codes, uint16_t* scales, double* Dq) {
-  const int G = lq_ceil_div(K, LQ_GROUP);
+// group == 32 selects MXINT4 (Appendix A.3): the scale is 2^e, e the smallest integer with 7 * 2^e >= absmax, stored
+// as the half-precision bit pattern of 2^e (weights far below 2^-24 are outside this library's range).
+void quant_main(const std::vector<double>& A, int K, int N, int8_t* codes, uint16_t* scales, double* Dq, int group) {
+  const int LQG = group;
+  const bool mx = group == 32;
+  const int G = lq_ceil_div(K, LQG);
 #pragma omp parallel for schedule(static)
   for (int g = 0; g < G; ++g) {
-    const int k0 = g * LQ_GROUP, k1 = std::min(K, k0 + LQ_GROUP);
+    const int k0 = g * LQG, k1 = std::min(K, k0 + LQG);
     std::vector<float> amax(N, 0.f), sc(N);
     for (int k = k0; k < k1; ++k)
       for (int n = 0; n < N; ++n) amax[n] = fmaxf(amax[n], fabsf((float)A[(size_t)k * N + n]));
     for (int n = 0; n < N; ++n) {
-      uint16_t hb = float_to_half_bits(amax[n] / 7.0f);
-      if (hb == 0) hb = 1;
+      uint16_t hb;
+      if (mx) {
+        int x = 0;
+        const float m = frexpf(amax[n], &x);                       // amax = m 2^x, m in [0.5, 1)
+        int e = amax[n] > 0.f ? (m <= 0.875f ? x - 3 : x - 2) : -24;
+        e = std::max(-24, std::min(15, e));                        // what a half can carry
+        hb = float_to_half_bits(ldexpf(1.0f, e));
+      } else {
+        hb = float_to_half_bits(amax[n] / 7.0f);
+        if (hb == 0) hb = 1;
+      }
       if (scales) scales[(size_t)g * N + n] = hb;
       sc[n] = half_bits_to_float(hb);
     }
@@ -310,7 +323,7 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
     const double inv_size = 1.0 / ((double)K * (double)N);
     if (r == 0) {
       std::vector<double> Dq((size_t)K * N);
-      quant_main(W, K, N, Lr->Wq.data(), Lr->sw.data(), Dq.data());
+      quant_main(W, K, N, Lr->Wq.data(), Lr->sw.data(), Dq.data(), cfg->group);
       if (trace) {
         double loss = 0;
         for (size_t i = 0; i < W.size(); ++i) loss += (Dq[i] - W[i]) * (Dq[i] - W[i]);
@@ -331,7 +344,7 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
       matmul_LR(L, R, K, N, r, D);
 #pragma omp parallel for schedule(static)
       for (long long i = 0; i < (long long)A.size(); ++i) A[i] = W[i] + D[i];
-      quant_main(A, K, N, nullptr, nullptr, E.data());            // E <- deq(Q1(W + LR))
+      quant_main(A, K, N, nullptr, nullptr, E.data(), cfg->group);            // E <- deq(Q1(W + LR))
       double loss = 0;
 #pragma omp parallel for reduction(+ : loss) schedule(static)
       for (long long i = 0; i < (long long)A.size(); ++i) {
@@ -395,7 +408,7 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
     }
     matmul_LR(L1d, L2d, K, N, r, D);
     for (size_t i = 0; i < A.size(); ++i) A[i] = W[i] - D[i];     // P = W - Q2(L1) Q2(L2)
-    quant_main(A, K, N, Lr->Wq.data(), Lr->sw.data(), nullptr);
+    quant_main(A, K, N, Lr->Wq.data(), Lr->sw.data(), nullptr, cfg->group);
     *out = Lr;
     return LQ_OK;
   } catch (const std::bad_alloc&) {

@@ -1,0 +1,528 @@
+// MXINT4 variant of the layer's main product (Appendix A.3: blocks of 32 values with a power-of-two E8M0 scale;
+// Table 2 quantizes the residual branch with it):
+//
+//   Y[m,n] = sum_b 2^(ex[m,b] + ew[b,n]) (qx_b Wq_b)[m,n] + sT[m] sL2[n] (tq L2q)[m,n] + bias[n]
+//
+// Here the tensor core applies the scales itself: tcgen05.mma kind::mxf8f6f4.block_scale takes one E8M0 scale
+// per operand row and 32-deep K block from tensor memory, so ALL blocks of a tile accumulate into ONE fp32
+// accumulator and nothing has to be drained per block.  The 4-bit codes ride in E4M3 operands as in the SINT4
+// kernel.  Products q q' 2^(e+e') are exact in fp32; their sum is rounded by the tensor core's fp32 accumulation.
+//
+// Shape of the kernel (persistent, one CTA per SM, 18 warps):
+//   warp 0      TMA producer: per stage 128 bytes of K of A (128 rows) and B (256 rows) plus the stage's scale bytes
+//               (512 B per 128 rows: four K blocks, already in the 32 x 16-byte layout tensor memory wants)
+//   warp 1      owns tensor memory; per stage: tcgen05.cp of the scale bytes into tensor-memory columns, then four
+//               K = 32 block-scaled MMAs (N = 256) into the tile's accumulator; after the last stage the accumulator is
+//               handed to the drain; the low-rank branch's up-projection (kind::i8, fp32 scales that the tensor core
+//               cannot apply) then reuses the same columns and is handed over a second time
+//   warps 2-17  drain: tcgen05.ld the main accumulator into registers (+ bias), then the branch accumulator
+//               (x sT x sL2), convert, stage rows in shared memory and store whole row segments
+// Every wait is bounded as in lq_gemm.cu.
+#include <cuda_fp16.h>
+
+#include "lq_internal.h"
+
+namespace {
+
+constexpr int UNIT = LQ_BN;                        // 128 output columns
+constexpr int NSTAGE = 3;                          // operand ring depth
+constexpr int STAGE_A_BYTES = LQ_BM * LQ_KSTAGE;   // 16 KB
+constexpr int STAGE_B_BYTES = 2 * UNIT * LQ_KSTAGE;   // 32 KB (two 128-row boxes)
+constexpr int SF_BYTES = 512;                      // scale bytes of 128 rows x 4 K blocks
+constexpr int STAGE_SF_OFF = STAGE_A_BYTES + STAGE_B_BYTES;            // SFA, then SFB of both halves
+constexpr int STAGE_BYTES = STAGE_SF_OFF + 2048;   // three scale blocks of 512 B, padded to keep the alignment
+constexpr int BR_FLOATS = LQ_BM + 2 * UNIT;        // branch stage: sT[128] then sL2[256]
+constexpr int NUM_DRAIN_WARPS = 16;
+constexpr int FIRST_DRAIN_WARP = 2;
+constexpr int GEMM_THREADS = (FIRST_DRAIN_WARP + NUM_DRAIN_WARPS) * 32;
+constexpr int OUT_ROW_BYTES = 128;                 // output bytes staged per row and pass
+constexpr int OUT_ROW_STRIDE = OUT_ROW_BYTES + 16;
+constexpr int OUT_WARP_BYTES = 32 * OUT_ROW_STRIDE;
+constexpr int SMEM_BAR_BYTES = 256;
+constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + NSTAGE * STAGE_BYTES + 2 * BR_FLOATS * 4 +
+                           NUM_DRAIN_WARPS * OUT_WARP_BYTES + SMEM_BAR_BYTES;
+static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+static_assert(STAGE_BYTES % 1024 == 0, "stages must keep the 1024-byte alignment of the swizzled tiles");
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s at 2 GHz
+// tensor-memory columns: accumulator [0, 256), then per stage 4 columns of A scales and 8 of B scales
+constexpr int TM_SFA = 256, TM_SFB = TM_SFA + 4 * NSTAGE;
+
+struct MxParams {
+  int M, N, Mpad, Npad;
+  int k_stages;           // Kpad / 128
+  int branch_mmas;        // 0: no branch; else MMAs of the branch stage (32 bytes of r each)
+  int tiles_m, units_n;
+  const uint8_t* sfa;     // [Mpad/128][k_stages][512]
+  const uint8_t* sfb;     // [Npad/128][k_stages][512]
+  const float* sT;        // [Mpad]
+  const float* sL2;       // [Npad]
+  const float* bias;      // [Npad]
+  void* Y;
+  int out_f32;
+  int32_t* status;
+};
+
+// ---- PTX wrappers -------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  Returns false when the CTA is aborting or the deadline passed (then it
+// raises the abort flag and records who gave up).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                            int role, long long limit = WAIT_LIMIT_CYCLES) {
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 0xFF) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > limit) {
+        *abort_flag = 1;
+        if (atomicCAS(status, 0, (int)LQ_ERR_TIMEOUT) == 0) status[1] = role;
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                          int role) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status, role);
+}
+// The same wait for a whole warp whose control flow must stay provably uniform (the producer
+// and the MMA warp keep their loop state in uniform registers).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                               int role) {
+  const bool ok = mbar_wait(bar, parity, abort_flag, status, role);
+  return __all_sync(0xffffffffu, ok);
+}
+
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.b32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+template <int KIND>   // 0: i8, 1: f8f6f4, 2: f16
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  if constexpr (KIND == 0) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else if constexpr (KIND == 1) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
+}
+
+// 32 lanes x 16 consecutive 32-bit columns: thread t of the warp receives row (lane base + t).
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
+// 8-row atoms 1024 bytes apart.  Adding (bytes >> 4) steps along K inside the swizzled row.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
+  const uint32_t lo = ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16);          // start address, LBO = 1 (unused)
+  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);              // SBO = 1024 B, version 1, SWIZZLE_128B
+  return ((uint64_t)hi << 32) | lo;
+}
+
+// instruction descriptor: accumulator format, operand formats, N >> 3 at bit 17, M >> 4 at bit 24
+__device__ __forceinline__ constexpr uint32_t idesc_shape(int n) { return ((uint32_t)(n >> 3) << 17) | ((uint32_t)(LQ_BM >> 4) << 24); }
+constexpr uint32_t IDESC_I8 = (2u << 4) | (1u << 7) | (1u << 10);    // S8 x S8 -> S32
+constexpr uint32_t IDESC_F8 = (1u << 4) | (0u << 7) | (0u << 10);    // E4M3 x E4M3 -> F32
+constexpr uint32_t IDESC_F16 = (1u << 4) | (0u << 7) | (0u << 10);   // F16 x F16 -> F32
+
+
+// Shared-memory matrix descriptor without swizzle (K-major, 8-row x 16-byte core matrices stored contiguously).
+__device__ __forceinline__ uint64_t make_smem_desc_plain(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
+  const uint32_t lo = ((smem_addr & 0x3FFFFu) >> 4) | ((lbo >> 4) << 16);
+  const uint32_t hi = (sbo >> 4) | (1u << 14);                             // version 1, no swizzle
+  return ((uint64_t)hi << 32) | lo;
+}
+// 32 rows x 16 bytes of shared memory -> 4 tensor-memory columns, replicated into the four 32-lane quarters
+__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+// block-scaled MMA: E4M3 operands, E8M0 scales (one per row and 32-deep K block) read from tensor memory
+__device__ __forceinline__ void tc_mma_mx(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t tsfa,
+                                          uint32_t tsfb, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
+      : "memory");
+}
+// instruction descriptor of the block-scaled kind: E4M3 x E4M3, E8M0 scales, K-major operands, scale-byte ids
+__device__ __forceinline__ constexpr uint32_t idesc_mx(int n, int sf_id) {
+  return ((uint32_t)sf_id << 4) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(LQ_BM >> 4) << 24) | ((uint32_t)sf_id << 29);
+}
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmL2, const MxParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
+  constexpr int OFF_BR = NSTAGE * STAGE_BYTES;
+  constexpr int OFF_OUT = OFF_BR + 2 * BR_FLOATS * 4;
+  constexpr int OFF_BAR = OFF_OUT + NUM_DRAIN_WARPS * OUT_WARP_BYTES;
+  const uint32_t sm_stage = base, sm_br = base + OFF_BR, sm_bar = base + OFF_BAR;
+  const float* br_ptr = reinterpret_cast<const float*>(smem + OFF_BR);
+  uint8_t* out_ptr = smem + OFF_OUT;
+  uint8_t* bar_ptr = smem + OFF_BAR;
+  // barrier map (8 bytes each)
+  constexpr int B_FULL = 0, B_EMPTY = NSTAGE, B_TFULL = 2 * NSTAGE, B_TEMPTY = B_TFULL + 1, B_RFULL = B_TEMPTY + 1,
+                B_REMPTY = B_RFULL + 2, NBAR = B_REMPTY + 2;
+  auto bar = [&](int idx) { return sm_bar + 8u * (uint32_t)idx; };
+  static_assert(NBAR * 8 + 16 <= SMEM_BAR_BYTES, "barrier area too small");
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + NBAR * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_ptr + NBAR * 8 + 8);
+
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // provably warp-uniform
+  const int lane = threadIdx.x & 31;
+  const bool has_branch = p.branch_mmas > 0;
+  const int stages_per_tile = p.k_stages + (has_branch ? 1 : 0);
+  const long long units = (long long)p.tiles_m * p.units_n;
+  const int u_begin = (int)((units * blockIdx.x) / gridDim.x);
+  const int u_end = (int)((units * (blockIdx.x + 1)) / gridDim.x);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NSTAGE; ++s) { mbar_init(bar(B_FULL + s), 1); mbar_init(bar(B_EMPTY + s), 1); }
+    mbar_init(bar(B_TFULL), 1);
+    mbar_init(bar(B_TEMPTY), NUM_DRAIN_WARPS);
+    for (int b = 0; b < 2; ++b) { mbar_init(bar(B_RFULL + b), 1); mbar_init(bar(B_REMPTY + b), NUM_DRAIN_WARPS); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    uint32_t it = 0, tc = 0;
+    bool ok = true;
+    for (int u = u_begin; u < u_end && ok; ++tc) {
+      const int mb = u / p.units_n, nu = u - mb * p.units_n;
+      const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
+      const int m0 = mb * LQ_BM, n0 = nu * UNIT;
+      for (int s = 0; s < stages_per_tile && ok; ++s, ++it) {
+        const int st = it % NSTAGE;
+        ok = mbar_wait_warp(bar(B_EMPTY + st), ((it / NSTAGE) & 1) ^ 1, abort_flag, p.status, LQ_STAGE_PRODUCER);
+        if (!ok) break;
+        const uint32_t a_dst = sm_stage + st * STAGE_BYTES, b_dst = a_dst + STAGE_A_BYTES, sf_dst = a_dst + STAGE_SF_OFF;
+        const uint32_t full = bar(B_FULL + st);
+        if (s < p.k_stages) {
+          if (elect_one()) {
+            mbar_expect_tx(full, STAGE_A_BYTES + width * (UNIT * LQ_KSTAGE) + (1 + width) * SF_BYTES);
+            tma_load_2d(a_dst, &tmA, s * LQ_KSTAGE, m0, full);
+            tma_load_2d(b_dst, &tmB, s * LQ_KSTAGE, n0, full);
+            if (width == 2) tma_load_2d(b_dst + UNIT * LQ_KSTAGE, &tmB, s * LQ_KSTAGE, n0 + UNIT, full);
+            bulk_load(sf_dst, p.sfa + ((size_t)mb * p.k_stages + s) * SF_BYTES, SF_BYTES, full);
+            for (int h = 0; h < width; ++h)
+              bulk_load(sf_dst + (1 + h) * SF_BYTES, p.sfb + ((size_t)(nu + h) * p.k_stages + s) * SF_BYTES, SF_BYTES, full);
+          }
+          __syncwarp();
+        } else {
+          const int rb = tc & 1;
+          ok = mbar_wait_warp(bar(B_REMPTY + rb), ((tc >> 1) & 1) ^ 1, abort_flag, p.status, LQ_STAGE_PRODUCER);
+          if (!ok) break;
+          if (elect_one()) {
+            mbar_expect_tx(full, STAGE_A_BYTES + width * (UNIT * LQ_KSTAGE));
+            tma_load_2d(a_dst, &tmT, 0, m0, full);
+            tma_load_2d(b_dst, &tmL2, 0, n0, full);
+            if (width == 2) tma_load_2d(b_dst + UNIT * LQ_KSTAGE, &tmL2, 0, n0 + UNIT, full);
+            const uint32_t rfull = bar(B_RFULL + rb);
+            mbar_expect_tx(rfull, (LQ_BM + width * UNIT) * 4);
+            bulk_load(sm_br + rb * BR_FLOATS * 4, p.sT + m0, LQ_BM * 4, rfull);
+            bulk_load(sm_br + rb * BR_FLOATS * 4 + LQ_BM * 4, p.sL2 + n0, width * UNIT * 4, rfull);
+          }
+          __syncwarp();
+        }
+      }
+      u += width;
+    }
+    if (!ok) {   // let copies in flight land before the CTA's shared memory goes away
+      const long long t0 = clock64();
+      while (clock64() - t0 < 2000000ll) { }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    uint32_t it = 0, hv = 0;            // hv counts accumulator hand-overs (main, then branch, of every tile)
+    bool ok = true;
+    for (int u = u_begin; u < u_end && ok;) {
+      const int mb = u / p.units_n, nu = u - mb * p.units_n;
+      const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
+      const int ncols = width * UNIT;
+      // the accumulator is free once the drain has read the previous hand-over
+      ok = mbar_wait_warp(bar(B_TEMPTY), (hv & 1) ^ 1, abort_flag, p.status, LQ_STAGE_MMA);
+      if (!ok) break;
+      tc_fence_after();
+      for (int s = 0; s < p.k_stages && ok; ++s, ++it) {
+        const int st = it % NSTAGE;
+        ok = mbar_wait_warp(bar(B_FULL + st), (it / NSTAGE) & 1, abort_flag, p.status, LQ_STAGE_MMA);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a_addr = sm_stage + st * STAGE_BYTES, b_addr = a_addr + STAGE_A_BYTES, sf_addr = a_addr + STAGE_SF_OFF;
+        const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
+        const uint32_t tsfa = tmem_base + TM_SFA + st * 4, tsfb = tmem_base + TM_SFB + st * 8;
+        if (elect_one()) {
+          tc_cp_sf(tsfa, make_smem_desc_plain(sf_addr, 16, 128));
+          tc_cp_sf(tsfb, make_smem_desc_plain(sf_addr + SF_BYTES, 16, 128));
+          if (width == 2) tc_cp_sf(tsfb + 4, make_smem_desc_plain(sf_addr + 2 * SF_BYTES, 16, 128));
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            tc_mma_mx(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc_mx(ncols, j), tsfa, tsfb, (uint32_t)(s | j));
+          tc_commit(bar(B_EMPTY + st));
+        }
+        __syncwarp();
+      }
+      if (!ok) break;
+      if (elect_one()) tc_commit(bar(B_TFULL));
+      __syncwarp();
+      ++hv;
+      if (has_branch) {
+        const int st = it % NSTAGE;
+        ok = mbar_wait_warp(bar(B_FULL + st), (it / NSTAGE) & 1, abort_flag, p.status, LQ_STAGE_MMA);
+        if (!ok) break;
+        ok = mbar_wait_warp(bar(B_TEMPTY), (hv & 1) ^ 1, abort_flag, p.status, LQ_STAGE_MMA);   // main part is in registers
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a_addr = sm_stage + st * STAGE_BYTES, b_addr = a_addr + STAGE_A_BYTES;
+        const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
+        if (elect_one()) {
+          for (int j = 0; j < p.branch_mmas; ++j) {
+            const uint64_t off = (uint64_t)((j * 32) >> 4);
+            tc_mma<0>(tmem_base, adesc + off, bdesc + off, IDESC_I8 | idesc_shape(ncols), (uint32_t)j);
+          }
+          tc_commit(bar(B_TFULL));
+          tc_commit(bar(B_EMPTY + st));
+        }
+        __syncwarp();
+        ++hv; ++it;
+      }
+      u += width;
+    }
+  } else {
+    // ------------------------------------------------------------------ drain + epilogue
+    const int quad = warp & 3;                          // tensor-memory lanes 32*quad .. 32*quad+31
+    const int cgi = (warp - FIRST_DRAIN_WARP) >> 2;     // which 32 columns of each 128-column half
+    const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(cgi * 32);
+    uint8_t* out_row = out_ptr + (warp - FIRST_DRAIN_WARP) * OUT_WARP_BYTES + lane * OUT_ROW_STRIDE;
+    uint32_t hv = 0, tc = 0;
+    bool ok = true;
+    for (int u = u_begin; u < u_end && ok; ++tc) {
+      const int mb = u / p.units_n, nu = u - mb * p.units_n;
+      const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
+      const int m0 = mb * LQ_BM, n0 = nu * UNIT;
+      float acc[2][2][16];                              // [half][16-column chunk][column]
+      // main part: the tensor core has already applied the block scales
+      ok = mbar_wait(bar(B_TFULL), hv & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
+      if (!ok) break;
+      tc_fence_after();
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (h < width) {
+          const float4* b4 = reinterpret_cast<const float4*>(p.bias + n0 + h * UNIT + cgi * 32);
+#pragma unroll
+          for (int ch = 0; ch < 2; ++ch) {
+            uint32_t v[16];
+            tmem_ld_32x16(tlane + h * UNIT + ch * 16, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+              const float4 b = __ldg(b4 + 4 * ch + c4);
+              acc[h][ch][4 * c4 + 0] = __uint_as_float(v[4 * c4 + 0]) + b.x;
+              acc[h][ch][4 * c4 + 1] = __uint_as_float(v[4 * c4 + 1]) + b.y;
+              acc[h][ch][4 * c4 + 2] = __uint_as_float(v[4 * c4 + 2]) + b.z;
+              acc[h][ch][4 * c4 + 3] = __uint_as_float(v[4 * c4 + 3]) + b.w;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_TEMPTY));
+      ++hv;
+      // branch part: acc += U * (sT * sL2), U exact int32 (|U| < 2^22: converted exactly with the 1.5 * 2^23 trick)
+      if (has_branch) {
+        const int rb = tc & 1;
+        ok = mbar_wait(bar(B_RFULL + rb), (tc >> 1) & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
+        if (!ok) break;
+        ok = mbar_wait(bar(B_TFULL), hv & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
+        if (!ok) break;
+        tc_fence_after();
+        const float* br = br_ptr + rb * BR_FLOATS;
+        const float stv = br[quad * 32 + lane];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (h < width) {
+            const float* sl2 = br + LQ_BM + h * UNIT + cgi * 32;
+#pragma unroll
+            for (int ch = 0; ch < 2; ++ch) {
+              uint32_t v[16];
+              tmem_ld_32x16(tlane + h * UNIT + ch * 16, v);
+              tmem_ld_wait();
+#pragma unroll
+              for (int c = 0; c < 16; ++c) {
+                const float uf = __int_as_float((int)v[c] + 0x4B400000) - 12582912.0f;
+                acc[h][ch][c] = fmaf(uf, stv * sl2[ch * 16 + c], acc[h][ch][c]);
+              }
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) { mbar_arrive(bar(B_TEMPTY)); mbar_arrive(bar(B_REMPTY + rb)); }
+        ++hv;
+      }
+      // epilogue: convert, stage this thread's 32-column row segment of each half in the warp's shared-memory
+      // rows, read it back with lanes along the row and store whole 64/128-byte row segments
+      const int rbase = m0 + quad * 32;
+      const int esize = p.out_f32 ? 4 : 2;
+      const int lpr = 32 * esize / 16;                                   // lanes per row: 4 (fp16) or 8 (fp32)
+      const int rpi = 32 / lpr;                                          // rows per instruction
+      const int cpl = 16 / esize;                                        // columns per lane
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (h < width) {
+          __syncwarp();                                                  // the previous half has been read back
+          if (p.out_f32) {
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc)
+#pragma unroll
+              for (int c4 = 0; c4 < 4; ++c4)
+                *reinterpret_cast<float4*>(out_row + cc * 64 + c4 * 16) =
+                    make_float4(acc[h][cc][4 * c4], acc[h][cc][4 * c4 + 1], acc[h][cc][4 * c4 + 2], acc[h][cc][4 * c4 + 3]);
+          } else {
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc)
+#pragma unroll
+              for (int c8 = 0; c8 < 2; ++c8) {
+                __half2 hh[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) hh[j] = __floats2half2_rn(acc[h][cc][c8 * 8 + 2 * j], acc[h][cc][c8 * 8 + 2 * j + 1]);
+                *reinterpret_cast<uint4*>(out_row + cc * 32 + c8 * 16) = *reinterpret_cast<uint4*>(hh);
+              }
+          }
+          __syncwarp();
+          const int lcol = n0 + h * UNIT + cgi * 32 + (lane % lpr) * cpl;
+          const uint8_t* wbase = out_ptr + (warp - FIRST_DRAIN_WARP) * OUT_WARP_BYTES + (lane % lpr) * 16;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            if (i * rpi < 32) {
+              const int rl = i * rpi + lane / lpr;
+              const uint4 val = *reinterpret_cast<const uint4*>(wbase + rl * OUT_ROW_STRIDE);
+              if (rbase + rl < p.M && lcol < p.N)
+                *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.Y) + ((size_t)(rbase + rl) * p.N + lcol) * esize) = val;
+            }
+          }
+        }
+      }
+      u += width;
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+}  // namespace
+
+lq_status lq_gemm_mx_prepare(int device) {
+  if (cudaSetDevice(device) != cudaSuccess) return LQ_ERR_CUDA;
+  if (lq_note_cuda(cudaFuncSetAttribute(lq_gemm_mx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) !=
+      cudaSuccess)
+    return LQ_ERR_CUDA;
+  return LQ_OK;
+}
+
+lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_dtype dt, cudaStream_t st) {
+  if (cudaSetDevice(A->device) != cudaSuccess) return LQ_ERR_CUDA;
+  if (!L->mx || !A->mx || L->f16_branch) return LQ_ERR_UNSUPPORTED;
+  MxParams p;
+  p.M = A->M; p.N = L->N; p.Mpad = A->Mpad; p.Npad = L->Npad;
+  p.k_stages = L->Kpad / LQ_KSTAGE;
+  p.branch_mmas = L->r == 0 ? 0 : lq_ceil_div(L->r, 32);
+  p.tiles_m = lq_ceil_div(A->M, LQ_BM);
+  p.units_n = L->Npad / UNIT;
+  p.sfa = A->d_sfa; p.sfb = L->d_sfb; p.sT = A->d_sT; p.sL2 = L->d_sL2; p.bias = L->d_bias;
+  p.Y = Y; p.out_f32 = dt == LQ_OUT_F32 ? 1 : 0;
+  p.status = lq_device_status_ptr(A->device);
+  if (!p.status) return LQ_ERR_CUDA;
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, A->device) != cudaSuccess) return LQ_ERR_CUDA;
+  int ctas = g_lq_gemm_ctas > 0 ? g_lq_gemm_ctas : sms;
+  const long long units = (long long)p.tiles_m * p.units_n;
+  if (ctas > units) ctas = (int)units;
+  lq_gemm_mx_kernel<<<ctas, GEMM_THREADS, SMEM_BYTES, st>>>(A->tmA, L->tmB, A->tmT, L->tmL2, p);
+  return lq_note_cuda(cudaGetLastError()) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
+}

@@ -10,6 +10,7 @@
 #include "lq.h"
 
 #define LQ_GROUP 64
+#define LQ_MX_BLOCK 32          // MXINT4: blocks of 32 with a power-of-two (E8M0) scale
 #define LQ_BM 128            // rows per output tile (one tcgen05 MMA, M = 128)
 #define LQ_BN 128            // columns per output tile
 #define LQ_KSTAGE 128        // bytes of K per shared-memory stage row (two groups of 64 codes)
@@ -26,6 +27,11 @@ enum { LQ_KIND_I8 = 0, LQ_KIND_E4M3 = 1 };
 static inline int lq_ceil_div(int a, int b) { return (a + b - 1) / b; }
 static inline int lq_round_up(int a, int b) { return lq_ceil_div(a, b) * b; }
 
+// offset of the scale byte of row (or column) i and 32-block kb inside its [tile][kb/4] chunk of 512 bytes
+static inline size_t lq_sf_offset(int i, int kb, int Kpad) {
+  return ((size_t)(i / 128) * (Kpad / 128) + kb / 4) * 512 + 16 * (i % 32) + 4 * ((i % 128) / 32) + kb % 4;
+}
+
 static inline int lq_branch_wbits(int branch) {
   return branch == LQ_BRANCH_W8A8 ? 8 : branch == LQ_BRANCH_W6A6 ? 6 : branch == LQ_BRANCH_W4A8 ? 4 : 0;
 }
@@ -38,6 +44,7 @@ struct lq_layer {
   int K, N, r, G;          // logical sizes
   int Kpad, Npad, Gpad;    // Kpad: multiple of 128; Npad: multiple of LQ_BN; Gpad = Kpad / 64
   bool integer_branch, f16_branch, has_bias;
+  bool mx;                     // MXINT4 main branch (cfg.group == 32): G counts blocks of 32, sw holds powers of two
   // host copy, canonical layouts
   std::vector<int8_t> Wq;      // [K][N]
   std::vector<uint16_t> sw;    // [G][N] half bits
@@ -58,12 +65,16 @@ struct lq_layer {
   uint8_t* d_L2c;              // [Npad][LQ_RCONT] bytes: int8 codes (or up to 64 halves) of column n, r contiguous
   float* d_sL2;                // [Npad]  (ones for W16A16)
   float* d_bias;               // [Npad]  (zeros without bias)
+  uint8_t* d_sfb;              // MXINT4: E8M0 bytes of the weight scales, [Npad/128][Kpad/128][512] in the 32 x 16-byte
+                               // layout tensor memory wants (byte 16*(n%32) + 4*((n%128)/32) + block%4)
   CUtensorMap tmB;             // over d_Wq8, box [LQ_BN][128B], 128B swizzle
   CUtensorMap tmL2;            // over d_L2c, box [LQ_BN][128B], 128B swizzle
 };
 
 struct lq_act {
   int K, N, r, G, Kpad, Gpad, branch;
+  bool mx;
+  uint8_t* d_sfa;              // MXINT4: E8M0 bytes of the activation scales, [Mpad/128][Kpad/128][512], same layout
   int M_max, Mpad, device, main_kind;
   int M;                       // rows of the last lq_quantize_act
   uint8_t* d_qx8;              // [Mpad][Kpad] operand bytes of the 4-bit codes (A operand, K-major)
@@ -92,6 +103,8 @@ int32_t* lq_device_status_ptr(int device);
 lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A, cudaStream_t st);
 lq_status lq_launch_gemm(const lq_layer* L, const lq_act* A, void* Y, lq_out_dtype dt, cudaStream_t st);
 lq_status lq_gemm_prepare(int device);
+lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_dtype dt, cudaStream_t st);
+lq_status lq_gemm_mx_prepare(int device);
 lq_status lq_launch_wait_probe(int device, cudaStream_t st);   // bounded-wait self-test kernel   // sets the kernel's shared-memory attribute once per device
 
 // byte an MMA operand carries for a 4-bit code q in [-7, 7]

@@ -61,6 +61,7 @@ struct QuantParams {
   int M, K, Kpad, Mpad, G;
   uint8_t* qx8;         // [Mpad][Kpad]
   float* sx;            // [Gpad][Mpad]
+  uint8_t* sfa;         // MXINT4: E8M0 scale bytes [Mpad/128][Kpad/128][512]
   int8_t* qb;           // [Mpad][Kpad] or null (not stored)
   float* sXb;           // [Mpad]
   const uint2* L1f;     // [Kpad/32][rpad/8][32] fragment-major first factor
@@ -75,7 +76,7 @@ struct QuantParams {
 // RELOAD: rows too long for the register file are read twice, chunk by chunk - once for the row maximum,
 // once to quantize; the second read is served by the L2 (the row was touched microseconds earlier), so DRAM
 // still sees X once, and the kernel keeps 64 registers per thread and full occupancy.
-template <int NCHUNK, int WARPS, bool RELOAD>
+template <int NCHUNK, int WARPS, bool RELOAD, bool MX>
 __global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams p) {
   extern __shared__ __align__(16) uint8_t qsm[];
   constexpr int RPW = ROWS / WARPS;    // rows per warp
@@ -154,14 +155,27 @@ __global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams 
       }
       a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
       a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
-      a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 4));
+      if constexpr (!MX) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 4));   // SINT4: 64 values = 8 lanes; MXINT4: 32 = 4 lanes
       if (k0 < p.Kpad) {
         uint32_t w0 = 0, w1 = 0, b0 = 0, b1 = 0;
         if (k0 < p.K) {
-          __half s16 = __float2half_rn(__fmul_rn(a, 0.142857149243354797f));   // fl32(1/7)
-          const unsigned short sbits = __half_as_ushort(s16);
-          if (sbits == 0) s16 = __ushort_as_half((unsigned short)1);             // floor 2^-24
-          const float s = __half2float(s16);
+          __half s16;
+          unsigned short sbits;
+          float s;
+          int mx_e = -127;
+          if constexpr (MX) {
+            // 2^e with e the smallest integer such that 7 * 2^e >= a: a = 1.f * 2^E, e = E - 2 if 1.f <= 1.75 else E - 1
+            const uint32_t ab = __float_as_uint(a);
+            if (a > 0.f) mx_e = (int)(ab >> 23) - 127 - (((ab & 0x7FFFFFu) <= 0x600000u) ? 2 : 1);
+            s = __uint_as_float((uint32_t)(mx_e + 127) << 23);                  // a == 0: 2^-127 is never used (codes are 0)
+            if (a == 0.f) s = 1.0f;
+            sbits = 0x3C00; s16 = __ushort_as_half(sbits);                       // not a subnormal-scale case
+          } else {
+            s16 = __float2half_rn(__fmul_rn(a, 0.142857149243354797f));          // fl32(1/7)
+            sbits = __half_as_ushort(s16);
+            if (sbits == 0) s16 = __ushort_as_half((unsigned short)1);           // floor 2^-24
+            s = __half2float(s16);
+          }
           const __half2* h2 = reinterpret_cast<const __half2*>(&vc);
           float x[8], q[8], t[8];
 #pragma unroll
@@ -169,7 +183,8 @@ __global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams 
             const float2 f = __half22float2(h2[i]);
             x[2 * i] = f.x; x[2 * i + 1] = f.y;
           }
-          const float inv = rcp_fast(s), hs = 0.5f * s;
+          // MXINT4: 1/s = 2^-e is exact, so x * (1/s) is exact and the magic-number rounding is already the definition's
+          const float inv = MX ? __uint_as_float((uint32_t)(127 - (a > 0.f ? mx_e : 0)) << 23) : rcp_fast(s), hs = 0.5f * s;
           bool exact = sbits < 0x0400;          // subnormal scale: quotient may exceed 7, use the plain definition
           bool near = false;
 #pragma unroll
@@ -181,6 +196,7 @@ __global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams 
             const float eb = __fmaf_rn(-__fadd_rn(t[i], -MAGIC), sb, x[i]);
             near |= !(fabsf(eb) < thr);
           }
+          if constexpr (MX) exact = false;
           if (exact) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) q[i] = fminf(fmaxf(rintf(__fdiv_rn(x[i], s)), -7.f), 7.f);
@@ -196,7 +212,13 @@ __global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams 
           b1 = __byte_perm(__byte_perm(__float_as_uint(t[4]), __float_as_uint(t[5]), 0x0040),
                            __byte_perm(__float_as_uint(t[6]), __float_as_uint(t[7]), 0x0040), 0x5410);
           *reinterpret_cast<uint2*>(p.qx8 + (size_t)m * p.Kpad + k0) = make_uint2(w0, w1);
-          if ((lane & 7) == 0) sx_s[(k0 >> 6) * ROWS + rl] = s;
+          if constexpr (MX) {
+            if ((lane & 3) == 0)
+              p.sfa[((size_t)(m >> 7) * (p.Kpad >> 7) + (k0 >> 7)) * 512 + 16 * (m & 31) + 4 * ((m & 127) >> 5) + ((k0 >> 5) & 3)] =
+                  (uint8_t)(mx_e + 127);
+          } else {
+            if ((lane & 7) == 0) sx_s[(k0 >> 6) * ROWS + rl] = s;
+          }
           if (p.qb != nullptr && p.branch_qmax > 0) *reinterpret_cast<uint2*>(p.qb + (size_t)m * p.Kpad + k0) = make_uint2(b0, b1);
         }
         if (p.branch_qmax > 0) *reinterpret_cast<uint2*>(qb_s + rl * qb_stride + k0) = make_uint2(b0, b1);
@@ -206,7 +228,7 @@ __global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams 
   __syncthreads();
 
   // group scales, transposed: [g][m0 .. m0+15] are 64-byte segments
-  for (int i = threadIdx.x; i < p.G * ROWS; i += WARPS * 32) {
+  for (int i = threadIdx.x; !MX && i < p.G * ROWS; i += WARPS * 32) {
     const int g = i / ROWS, rl = i % ROWS;
     if (m0 + rl < p.M) p.sx[(size_t)g * p.Mpad + m0 + rl] = sx_s[g * ROWS + rl];
   }
@@ -296,17 +318,17 @@ __global__ void __launch_bounds__(256) lq_down_f16_kernel(const __half* __restri
   if (lane == 0) sT[m] = 1.0f;
 }
 
-template <int NCHUNK, int WARPS, bool RELOAD>
+template <int NCHUNK, int WARPS, bool RELOAD, bool MX>
 cudaError_t launch_quant(const QuantParams& p, size_t smem, cudaStream_t st) {
   static bool attr_set[64] = {false};
   int dev = 0;
   cudaGetDevice(&dev);
   if (smem > 48 * 1024 && !attr_set[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(lq_quant_kernel<NCHUNK, WARPS, RELOAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(lq_quant_kernel<NCHUNK, WARPS, RELOAD, MX>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e != cudaSuccess) return e;
     attr_set[dev & 63] = true;
   }
-  lq_quant_kernel<NCHUNK, WARPS, RELOAD><<<lq_ceil_div(p.M, ROWS), WARPS * 32, smem, st>>>(p);
+  lq_quant_kernel<NCHUNK, WARPS, RELOAD, MX><<<lq_ceil_div(p.M, ROWS), WARPS * 32, smem, st>>>(p);
   return cudaGetLastError();
 }
 
@@ -319,7 +341,7 @@ lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A,
   QuantParams p;
   p.X = reinterpret_cast<const uint4*>(X);
   p.M = M; p.K = K; p.Kpad = Kpad; p.Mpad = A->Mpad; p.G = L->G;
-  p.qx8 = A->d_qx8; p.sx = A->d_sx;
+  p.qx8 = A->d_qx8; p.sx = A->d_sx; p.sfa = A->d_sfa;
   p.qb = g_lq_store_qb ? A->d_qb : nullptr;
   p.sXb = A->d_sXb;
   p.L1f = reinterpret_cast<const uint2*>(L->d_L1f);
@@ -331,14 +353,17 @@ lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A,
   const int nchunk = lq_ceil_div(Kpad, 256);
   cudaError_t e;
   if (A->main_kind != LQ_KIND_E4M3) return LQ_ERR_UNSUPPORTED;
-  if (nchunk <= 2) e = launch_quant<2, 16, false>(p, smem, st);        // the row stays in registers (one warp per row)
-  else if (nchunk <= 5) e = launch_quant<5, 16, false>(p, smem, st);
-  else if (nchunk <= 9) e = launch_quant<9, 16, true>(p, smem, st);     // longer rows: read twice, second time from the L2
-  else if (nchunk <= 12) e = launch_quant<12, 16, true>(p, smem, st);
-  else if (nchunk <= 18) e = launch_quant<18, 16, true>(p, smem, st);
-  else if (nchunk <= 22) e = launch_quant<22, 16, true>(p, smem, st);
-  else if (nchunk <= 32) e = launch_quant<32, 16, true>(p, smem, st);
+#define LQ_QUANT_DISPATCH(MXF)                                                                                          \
+  if (nchunk <= 2) e = launch_quant<2, 16, false, MXF>(p, smem, st);   /* the row stays in registers (one warp per row) */ \
+  else if (nchunk <= 5) e = launch_quant<5, 16, false, MXF>(p, smem, st);                                               \
+  else if (nchunk <= 9) e = launch_quant<9, 16, true, MXF>(p, smem, st);   /* longer rows: read twice, 2nd time from L2 */ \
+  else if (nchunk <= 12) e = launch_quant<12, 16, true, MXF>(p, smem, st);                                              \
+  else if (nchunk <= 18) e = launch_quant<18, 16, true, MXF>(p, smem, st);                                              \
+  else if (nchunk <= 22) e = launch_quant<22, 16, true, MXF>(p, smem, st);                                              \
+  else if (nchunk <= 32) e = launch_quant<32, 16, true, MXF>(p, smem, st);                                              \
   else return LQ_ERR_UNSUPPORTED;
+  if (L->mx) { LQ_QUANT_DISPATCH(true) } else { LQ_QUANT_DISPATCH(false) }
+#undef LQ_QUANT_DISPATCH
   if (lq_note_cuda(e) != cudaSuccess) return LQ_ERR_CUDA;
   if (L->f16_branch) {
     lq_down_f16_kernel<<<lq_ceil_div(M, 8), 256, 0, st>>>(reinterpret_cast<const __half*>(X),

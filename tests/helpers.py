@@ -8,13 +8,17 @@ def import_oracle_layer(layer: dict):
     """Feeds a layer produced by the CPU oracle to lq_layer_import (the direction data flows in
     every parity test: oracle -> library, never the reverse)."""
     cfg = B.lq_config_default(layer["K"], layer["N"], layer["rank"], layer["branch"])
+    mx = layer.get("main", "sint4") == "mxint4"
+    if mx:
+        cfg.group = 32                                     # MXINT4: blocks of 32, power-of-two scales (passed as halves 2^e)
     if layer["branch"] == "w16a16":
         L1, L2, s1, s2 = layer["L1h"], layer["L2h"], None, None
     elif layer["branch"] == "none" or layer["rank"] == 0:
         L1 = L2 = s1 = s2 = None
     else:
         L1, L2, s1, s2 = layer["L1q"], layer["L2q"], layer["sL1"], layer["sL2"]
-    h = B.lq_layer_import(cfg, B.pack_nibbles(layer["Wq"]), layer["sw"], L1, s1, L2, s2, layer.get("bias"))
+    sw = np.exp2(layer["ew"].astype(np.float64)).astype(np.float16) if mx else layer["sw"]
+    h = B.lq_layer_import(cfg, B.pack_nibbles(layer["Wq"]), sw, L1, s1, L2, s2, layer.get("bias"))
     return h, cfg
 
 
@@ -54,7 +58,10 @@ def rel_fro(Y, Yref) -> float:
 
 def assert_codes_equal(ex: dict, ref: dict, branch: str, with_qb: bool = True):
     assert np.array_equal(ex["qx"], ref["qx"]), "qx differs"
-    assert np.array_equal(ex["sx"].view(np.uint16), ref["sx"].view(np.uint16)), "sx differs"
+    if "ex" in ref:                                        # MXINT4: the library exports the block exponents
+        assert np.array_equal(ex["sx"], ref["ex"]), "block exponents differ"
+    else:
+        assert np.array_equal(ex["sx"].view(np.uint16), ref["sx"].view(np.uint16)), "sx differs"
     if branch in ("w8a8", "w6a6", "w4a8"):
         if with_qb:
             assert np.array_equal(ex["qb"], ref["qb"]), "qb differs"

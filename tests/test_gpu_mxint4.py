@@ -1,0 +1,96 @@
+"""GPU parity of the MXINT4 main branch (Appendix A.3: blocks of 32 values, power-of-two E8M0 scales; the
+residual-branch format of Table 2): codes and block exponents bit for bit against the oracle, Y within a relative
+Frobenius error of 1e-3 (fp16 output) / 2e-5 (fp32 output: the tensor core sums the block-scaled products in fp32)."""
+import numpy as np
+import pytest
+
+from oracle import lq_oracle as O
+from paper_2604_18117_b200 import inputs as I
+from tests.helpers import assert_codes_equal, gpu_forward, rel_fro
+
+pytestmark = pytest.mark.gpu
+
+TOL_F16 = 1e-3
+TOL_F32 = 2e-5
+
+
+def _mx_layer(rng, K, N, r, branch, wscale=0.02, bias=True):
+    layer = {"main": "mxint4", "branch": branch if r > 0 else "none", "rank": r, "K": K, "N": N,
+             "bias": (rng.standard_normal(N) * 0.05).astype(np.float16) if bias else None}
+    W = rng.standard_normal((K, N)) * wscale
+    W[:: max(1, K // 7), :] *= 10                                       # outlier input channels: exponents vary per block
+    layer["Wq"], layer["ew"] = O.q_weight_main_mx(W)
+    if r > 0:
+        bw, _ = O.BRANCH_BITS[branch]
+        layer["L1q"], layer["sL1"] = O.q_factor(rng.standard_normal((K, r)) * 0.05, bw)
+        layer["L2q"], layer["sL2"] = O.q_factor(rng.standard_normal((r, N)) * 0.05, bw)
+    return layer
+
+
+def _check(layer, X):
+    ref = O.forward(X, layer)
+    Y32, ex = gpu_forward(layer, X, out_f32=True)
+    assert np.isfinite(Y32).all()
+    assert_codes_equal(ex, ref, layer["branch"])
+    e32 = rel_fro(Y32, ref["Y"])
+    assert e32 <= TOL_F32, f"fp32 output error {e32}"
+    Y16, _ = gpu_forward(layer, X, out_f32=False, export=False)
+    e16 = rel_fro(Y16, ref["Y"])
+    assert e16 <= TOL_F16, f"fp16 output error {e16}"
+    return e32, e16
+
+
+def test_mx_integer_exact_product_with_varied_exponents():
+    """Integer codes times per-block powers of two on both sides: every product is exact, so Y must equal the oracle's
+    fp64 sum to fp32 rounding - and a wrong scale byte, block id or row/column mapping changes Y by a factor of two or more."""
+    rng = np.random.default_rng(0)
+    M, K, N = 256, 512, 384
+    ea = rng.integers(-3, 4, size=(M, K // 32)); eb = rng.integers(-5, 2, size=(K // 32, N))
+    Xi = rng.integers(-7, 8, size=(M, K)); Xi[:, ::32] = 7
+    Wi = rng.integers(-7, 8, size=(K, N)); Wi[::32, :] = 7
+    X = (Xi * np.exp2(np.repeat(ea, 32, axis=1))).astype(np.float16)
+    W = Wi * np.exp2(np.repeat(eb, 32, axis=0))
+    layer = {"main": "mxint4", "branch": "none", "rank": 0, "K": K, "N": N, "bias": None}
+    layer["Wq"], layer["ew"] = O.q_weight_main_mx(W)
+    assert np.array_equal(layer["Wq"], Wi) and np.array_equal(layer["ew"], eb)
+    ref = O.forward(X, layer)
+    assert np.array_equal(ref["qx"], Xi) and np.array_equal(ref["ex"], ea)
+    Y, ex = gpu_forward(layer, X, out_f32=True)
+    assert_codes_equal(ex, ref, "none")
+    assert rel_fro(Y, ref["Y"]) <= 1e-6
+    assert np.abs(Y - ref["Y"]).max() <= 1e-5 * np.abs(ref["Y"]).max()
+
+
+@pytest.mark.parametrize("branch", ["none", "w8a8", "w6a6", "w4a8"])
+def test_mx_small_shapes_all_branches(branch):
+    rng = np.random.default_rng(1)
+    M, K, N, r = 200, 328, 200, 0 if branch == "none" else 32          # ragged M, N; K = 10.25 blocks
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    X[:, 7] *= 20
+    X[3, :] = 0; X[4, :64] = 0; X[5, :] = np.float16(2.0 ** -24)
+    _check(_mx_layer(rng, K, N, r, branch), X)
+
+
+def test_mx_wide_and_narrow_tiles_long_k():
+    rng = np.random.default_rng(2)
+    M, K, N, r = 300, 4608, 392, 64
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    X[:, rng.integers(0, K, 8)] *= 20
+    _check(_mx_layer(rng, K, N, r, "w8a8"), X)
+
+
+def test_mx_sana_shape_sampled_rows():
+    """K = 5600, N = 2240 at M = 8192 with the seeded benchmark activations; 160 sampled rows against the oracle."""
+    rng = np.random.default_rng(3)
+    wl = I.workload(3)
+    spec = I.SANA_LAYERS[3]
+    X, _, _ = I.layer_inputs(wl, spec, M=8192)
+    layer = _mx_layer(rng, spec.K, spec.N, 32, "w4a8")
+    rows = np.unique(np.concatenate([[0, 127, 128, 8191], rng.choice(8192, 156, replace=False)]))
+    ref = O.forward(X[rows], layer)
+    Y, ex = gpu_forward(layer, X, out_f32=False)
+    assert np.array_equal(ex["qx"][rows], ref["qx"])
+    assert np.array_equal(ex["sx"][rows], ref["ex"])
+    assert np.array_equal(ex["tq"][rows], ref["tq"])
+    assert np.isfinite(Y.astype(np.float32)).all()
+    assert rel_fro(Y[rows], ref["Y"]) <= TOL_F16
