@@ -108,6 +108,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   if (mbar_try_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, abort_flag, status, role);
 }
+// Wait of a role that is idle for a long time (the drain during a tile's main loop): polling at full speed would take
+// issue slots from the producer and the MMA issuer that share its scheduler, so it sleeps between polls.
+__device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                               int role) {
+  for (int i = 0; i < 64; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(200);
+  }
+  return mbar_wait_slow(bar, parity, abort_flag, status, role);
+}
 // The same wait for a whole warp whose control flow must stay provably uniform (the producer
 // and the MMA warp keep their loop state in uniform registers).
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
@@ -380,7 +390,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int m0 = mb * LQ_BM, n0 = nu * UNIT;
       float acc[2][2][16];                              // [half][16-column chunk][column]
       // main part: the tensor core has already applied the block scales
-      ok = mbar_wait(bar(B_TFULL), hv & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
+      ok = mbar_wait_idle(bar(B_TFULL), hv & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
       if (!ok) break;
       tc_fence_after();
 #pragma unroll
