@@ -53,15 +53,16 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
-def gemm_traffic_bytes():
-    """DRAM bytes of one step's GEMM launches as measured by ncu (profiles/gemm_dram_traffic.json),
-    or None when the GEMM source differs from the one that was profiled."""
+def gemm_traffic_bytes(main="sint4"):
+    """DRAM bytes of one step's GEMM launches as measured by ncu (profiles/gemm*_dram_traffic.json),
+    or None when the GEMM source differs from the one that was profiled (or none was taken)."""
     import hashlib
-    rec = os.path.join(ROOT, "profiles", "gemm_dram_traffic.json")
-    src = os.path.join(ROOT, "paper_2604_18117_b200", "csrc", "lq_gemm.cu")
+    stem = "lq_gemm_mx" if main == "mxint4" else "lq_gemm"
+    rec = os.path.join(ROOT, "profiles", "gemm_mx_dram_traffic.json" if main == "mxint4" else "gemm_dram_traffic.json")
+    src = os.path.join(ROOT, "paper_2604_18117_b200", "csrc", stem + ".cu")
     try:
         d = json.load(open(rec))
-        if hashlib.sha256(open(src, "rb").read()).hexdigest() != d["lq_gemm_cu_sha256"]:
+        if hashlib.sha256(open(src, "rb").read()).hexdigest() != d[stem + "_cu_sha256"]:
             return None
         return int(d["dram_bytes_per_step"])
     except (OSError, KeyError, ValueError):
@@ -140,7 +141,7 @@ def run_reference(args):
     layers = []
     for spec in wl.layers:
         X, W, _ = I.layer_inputs(wl, spec, M=SAMPLE_ROWS)
-        layer, _ = O.calibrate(W, wl.rank, wl.branch, steps=args.calib_steps)
+        layer, _ = O.calibrate(W, wl.rank, wl.branch, steps=args.calib_steps, main=args.main)
         layers.append((spec, X, layer))
     ops_sample = sum(layer_ops(SAMPLE_ROWS, s.K, s.N, wl.rank) for s, _, _ in layers)
     for _ in range(args.warmup):
@@ -165,11 +166,14 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+MAIN_NAMES = {"sint4": "SINT4 group 64 (fp16 scales)", "mxint4": "MXINT4 block 32 (power-of-two scales)"}
+
+
 def workload_config(wl, args):
     return {"workload": f"config{wl.config}: PixArt-class block linears (qkv 1152->3456, attn-out 1152->1152, "
                         f"fc1 1152->4608, fc2 4608->1152), M={wl.M} rows (4096 tokens x batch 2), rank {wl.rank}, "
-                        f"main W4A4 SINT4 group 64, branch {wl.branch}" if wl.config in (1, 2) else f"config{wl.config}",
-            "rows": wl.M, "rank": wl.rank, "branch": wl.branch, "layers": [s.name for s in wl.layers],
+                        f"main W4A4 {MAIN_NAMES[args.main]}, branch {wl.branch}" if wl.config in (1, 2) else f"config{wl.config}",
+            "main": args.main, "rows": wl.M, "rank": wl.rank, "branch": wl.branch, "layers": [s.name for s in wl.layers],
             "calibration_steps": args.calib_steps,
             "l2": ("L2 flushed (256 MiB write) before every timed step; layers inside a step run back to back"
                    if args.l2 == "flush" else
@@ -184,7 +188,7 @@ def cpu_baseline(wl, I, args):
     layers = []
     for spec in wl.layers:
         X, W, _ = I.layer_inputs(wl, spec, M=SAMPLE_ROWS)
-        layer, _ = O.calibrate(W, wl.rank, wl.branch, steps=0)
+        layer, _ = O.calibrate(W, wl.rank, wl.branch, steps=0, main=args.main)
         layers.append((spec, X, layer))
     ops = sum(layer_ops(SAMPLE_ROWS, s.K, s.N, wl.rank) for s, _, _ in layers)
     for _, X, layer in layers:
@@ -226,6 +230,8 @@ def run_ours(args):
         Xh, W, bias = I.layer_inputs(wl, spec, seed=D.shard_seed(0, rank), with_bias=True)
         cfg = B.lq_config_default(spec.K, spec.N, r, wl.branch)
         cfg.steps = args.calib_steps
+        if args.main == "mxint4":
+            cfg.group = 32
         h, _ = B.lq_calibrate(cfg, W, bias)
         B.lq_layer_to_device(h, local)
         act = B.lq_act_create(h, M, local)
@@ -333,7 +339,9 @@ def run_ours(args):
         achieved = gops_step / (gemm_avg_ms * 1e-3) / 1e12
         # algorithmic bytes per row of the quantizer: X read once (2K); packed 4-bit codes (K/2), 8-bit branch
         # codes (K), fp16 group scales (2G), the per-token scale (4), r intermediate codes and their scale (4)
-        k1_bytes = sum(M * (2 * L["spec"].K + L["spec"].K // 2 + L["spec"].K + 2 * (-(-L["spec"].K // 64)) + 4 + r + 4)
+        # (MXINT4: one scale byte per block of 32 instead)
+        sc_bytes = (lambda K: -(-K // 32)) if args.main == "mxint4" else (lambda K: 2 * (-(-K // 64)))
+        k1_bytes = sum(M * (2 * L["spec"].K + L["spec"].K // 2 + L["spec"].K + sc_bytes(L["spec"].K) + 4 + r + 4)
                        for L in layers)
         quant_avg_ms = float(np.mean(quant_ms))
         line = {
@@ -348,9 +356,10 @@ def run_ours(args):
                     "d2h_bytes_per_step": int(sum(M * L["spec"].N * 2 for L in layers)),
                     "ms_per_step": e2e_s / e2e_steps * 1e3},
             "gpu_launches": args.steps * len(layers) * (3 if wl.branch == "w16a16" else 2),
-            "roofline": {"kernel": "lq_gemm_kernel (4 launches per step, one per layer)", "bound": "tensor",
+            "roofline": {"kernel": ("lq_gemm_mx_kernel" if args.main == "mxint4" else "lq_gemm_kernel") +
+                                   " (4 launches per step, one per layer)", "bound": "tensor",
                          "achieved": achieved, "peak": peak_tops, "unit": "TOP/s", "frac": achieved / peak_tops,
-                         "traffic": gemm_traffic_bytes(), "traffic_note": "DRAM read + write bytes of the four GEMM "
+                         "traffic": gemm_traffic_bytes(args.main), "traffic_note": "DRAM read + write bytes of the four GEMM "
                          "launches of one step from one ncu capture; null when the kernel source changed since",
                          "peak_source": f"2 x bf16_tflops ({peaks['bf16_tflops']}) of {peaks['source']}: 8-bit operands, "
                                         f"nominal ratio 2 to bf16",
@@ -381,6 +390,9 @@ def main():
     ap.add_argument("--config", type=int, default=1)
     ap.add_argument("--rank", type=int, default=32)
     ap.add_argument("--branch", default=None)
+    ap.add_argument("--main", default="sint4", choices=["sint4", "mxint4"],
+                    help="main-branch 4-bit format: sint4 = blocks of 64 with fp16 scales (the headline configuration), "
+                         "mxint4 = blocks of 32 with power-of-two scales applied by the tensor core")
     ap.add_argument("--calib-steps", type=int, default=2, dest="calib_steps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--l2", default="flush", choices=["flush", "working-set"],

@@ -5,7 +5,15 @@
  *
  * Notation follows the paper (Section 3.1): X in R^{m x d} activations, W in R^{d x n} weights,
  * Y = X W.  Here M = m rows (tokens x batch), K = d input features, N = n output features,
- * r = the rank of the low-rank branch, G = ceil(K / 64) groups.
+ * r = the rank of the low-rank branch, G = ceil(K / group) blocks of the 4-bit main format.
+ *
+ * Two main formats (Appendix A.3, Table 2), chosen by lq_config.group:
+ *   group = 64  SINT4: signed 4-bit codes in [-7, 7], one fp16 scale per block of 64 along K;
+ *               the per-block scale products are applied by the GEMM's epilogue warps.
+ *   group = 32  MXINT4: the same codes, one power-of-two scale 2^e per block of 32 along K,
+ *               e the smallest integer with 7 * 2^e >= max|v| of the block (the paper does not
+ *               spell the rule out; this one never clips); the scales are applied by the tensor
+ *               core itself (block-scaled MMA).  Integer branches only.
  *
  * Every function returns an lq_status; nothing throws, aborts or prints.  "host" / "device"
  * in a parameter comment says which address space the pointer lives in.  Device pointers and
@@ -49,7 +57,7 @@ typedef enum { LQ_OUT_F16 = 0, LQ_OUT_F32 = 1 } lq_out_dtype;
 /* One layer's shape and calibration settings. */
 typedef struct {
   int32_t K, N, rank; /* d, n and rho of Sections 3.1-3.2; rank in [0, 128], N even, K <= 8192    */
-  int32_t group;      /* 64: the SINT4 block of Appendix A.3 (the only supported value)           */
+  int32_t group;      /* 64 = SINT4 (default), 32 = MXINT4: block length of the 4-bit main format  */
   int32_t branch;     /* an lq_branch_fmt                                                         */
   int32_t steps;      /* Adam steps on (L, R); 1000 in Appendix A "Optimization"                  */
   float lr;           /* 1e-4 for integer formats (Appendix A)                                    */
@@ -70,12 +78,13 @@ lq_status lq_config_default(lq_config* cfg, int32_t K, int32_t N, int32_t rank, 
  * Appendix B.2): SVD initialisation L = -L0, R = R0; Adam on
  * mean((Q1(W + L R) - W - L R)^2) with the quantizer's derivative taken as zero; the best
  * iterate is kept; the factors are quantized with Q2; P = W - Q2(L1) Q2(L2) is quantized
- * with Q1 (SINT4, groups of 64 along K per output column).
+ * with Q1 (SINT4 or MXINT4 blocks along K per output column, as cfg->group says; MXINT4 weight
+ * exponents are kept within [-24, 15] so that 2^e is a finite fp16 number).
  *   W_f16_host     [K][N] row-major IEEE half bits (the paper's d x n orientation), host
  *   bias_f16_host  [N] half bits or NULL, host
  *   out            receives a new layer (host copy only; see lq_layer_to_device)
  *   objective_trace[steps + 1] doubles or NULL, host: objective at every iterate, [0] = init
- * Errors: INVALID_ARG (null / bad shape), UNSUPPORTED (rot_steps != 0, group != 64, ...),
+ * Errors: INVALID_ARG (null / bad shape), UNSUPPORTED (rot_steps != 0, group not 64 or 32, MXINT4 with the fp16 branch, ...),
  * NUMERIC (non-finite W), ALLOC. */
 lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W_f16_host,
                        const uint16_t* bias_f16_host, lq_layer** out, double* objective_trace);
@@ -83,7 +92,8 @@ lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W_f16_host,
 /* Build a layer from already quantized parts (all host pointers, copied):
  *   Wq_packed [K][N/2] bytes: codes in [-7,7] as two's-complement nibbles, column 2j in the
  *             low nibble, column 2j+1 in the high nibble
- *   sw        [G][N] half bits: SINT4 scale of group g of output column n
+ *   sw        [G][N] half bits: scale of block g of output column n (MXINT4: an exact power of
+ *             two 2^e with e in [-24, 15], anything else is INVALID_ARG)
  *   L1, L2    integer branches: int8 codes [K][rank] and [rank][N]; W16A16: half bits, same shapes
  *   sL1, sL2  fp32 per-column scales [rank] and [N]; NULL for W16A16
  *   bias      [N] half bits or NULL
@@ -113,7 +123,8 @@ lq_status lq_act_free(lq_act* act);
 /* Dynamic activation quantization fused with the branch's down-projection (Figure 1;
  * Appendix A.2 "Quantization": the activations forwarded to both branches are quantized).
  * One read of X produces
- *   qx, sx   SINT4 codes / fp16 scales per token and group of 64 along K (Appendix A.3)
+ *   qx, sx   4-bit codes / scales per token and block along K (Appendix A.3): fp16 scales per
+ *            block of 64 (SINT4) or one exponent byte per block of 32 (MXINT4)
  *   qb, sXb  per-token branch codes / fp32 scale
  *   tq, sT   per-token codes / scale of the rank-r intermediate T = deq(qb) deq(L1)
  *   X_f16_dev  [M][K] row-major half, device, 16-byte aligned
@@ -124,7 +135,8 @@ lq_status lq_quantize_act(const lq_layer* layer, const void* X_f16_dev, int32_t 
 
 /* Y = sum_g sx sw (qx_g Wq_g) + sT sL2 (tq L2q) + bias: the 4-bit main product per group on
  * the tensor cores, per-group scales and the branch's up-projection applied in one epilogue
- * (Figure 1; Section 3.3).
+ * (Figure 1; Section 3.3).  For an MXINT4 layer the tensor core applies sx sw itself and the
+ * epilogue only adds the branch and the bias.
  *   act    result of lq_quantize_act for this layer
  *   Y_dev  [M][N] row-major, half or float per `dtype`, device, 16-byte aligned
  * Asynchronous on `cuda_stream`. */
@@ -157,7 +169,8 @@ lq_status lq_linear_forward_host(const lq_layer* layer, lq_act* act, const void*
  *   Y_dev      [M][N] row-major half or float per `dtype`, device, 16-byte aligned
  * Limit: with Mp = M rounded up to 128, Kp = K rounded up to 128 and G2 = Kp / 64, the record
  * needs about 2*Mp*Kp + 4*G2*Mp + 136*Mp bytes (each part rounded up to 256); if that exceeds
- * LQ_STATIC_SCRATCH_BYTES the call returns LQ_ERR_UNSUPPORTED and launches nothing
+ * LQ_STATIC_SCRATCH_BYTES - or if the layer's main format is MXINT4, which this entry point
+ * does not cover - the call returns LQ_ERR_UNSUPPORTED and launches nothing
  * (8 MiB holds e.g. M = 256 at any supported K, or M = 1024 at K = 2240).
  * The first call on each device looks up the array's device address (one-time set-up, done
  * with that device current); make that first call before starting any stream capture.
@@ -169,7 +182,8 @@ lq_status lq_linear_forward_static(const lq_layer* layer, const void* X_f16_dev,
                                    lq_out_dtype dtype, void* cuda_stream);
 
 /* Decode the activation record of the last lq_quantize_act into plain host arrays (for
- * parity checks); NULL skips a part.  qx int8 [M][K], sx half bits [M][G], qb int8 [M][K],
+ * parity checks); NULL skips a part.  qx int8 [M][K], sx half bits [M][G] (MXINT4: the block
+ * exponents e as int16 [M][G], since 2^e may lie below the fp16 range), qb int8 [M][K],
  * sXb float [M], tq int8 [M][rank] (W16A16: half bits [M][rank]), sT float [M].
  * Synchronises `cuda_stream`. */
 lq_status lq_act_export(const lq_act* act, int8_t* qx, uint16_t* sx, int8_t* qb, float* sXb,

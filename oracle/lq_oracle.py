@@ -263,44 +263,55 @@ def svd_init(W, r: int):
     return U[:, :r] * rs[None, :], rs[:, None] * Vt[:r, :]
 
 
-def q1_dequant(A):
-    """Q1(A) as real numbers: SINT4 along K (axis 0) per output column, input rounded to fl32."""
+def q1_dequant(A, main: str = "sint4"):
+    """Q1(A) as real numbers: SINT4 (or MXINT4) along K (axis 0) per output column."""
+    if main == "mxint4":
+        c, e = q_weight_main_mx(A)
+        return deq_mx(c.T.copy(), e.T.copy()).T.copy()
     c, s = q_weight_main(A)
     return deq_weight_main(c, s)
 
 
-def residual_error(W, L, R):
+def residual_error(W, L, R, main: str = "sint4"):
     """E = Q1(W + L R) - W - L R  (Eq. "low-rank-optimization")."""
     D = L @ R
-    return q1_dequant(W + D) - W - D
+    return q1_dequant(W + D, main) - W - D
 
 
-def objective(W, L, R) -> float:
+def objective(W, L, R, main: str = "sint4") -> float:
     """MSE form of the calibration objective: mean over K*N entries of E^2."""
-    E = residual_error(W, L, R)
+    E = residual_error(W, L, R, main)
     return float(np.mean(E * E))
 
 
-def gradients(W, L, R):
+def gradients(W, L, R, main: str = "sint4"):
     """(loss, dL, dR) with the quantizer's derivative taken as zero (Appendix B.2):
     d/d(LR) = -2 E / (K N),  dL = d(LR) R^T,  dR = L^T d(LR)."""
-    E = residual_error(W, L, R)
+    E = residual_error(W, L, R, main)
     c = -2.0 / E.size
     return float(np.mean(E * E)), c * (E @ R.T), c * (L.T @ E)
 
 
 def calibrate(W16, rank: int, branch: str = "w8a8", steps: int = 1000, lr: float = 1e-4,
-              beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, bias=None):
+              beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, bias=None, main: str = "sint4"):
     """Data-free calibration of one weight.  Returns (layer dict, trace [steps+1] of the
-    objective at every iterate visited, iterate 0 = the SVD initialisation)."""
+    objective at every iterate visited, iterate 0 = the SVD initialisation).  main selects Q1:
+    "sint4" (blocks of 64, fp16 scale) or "mxint4" (blocks of 32, power-of-two scale; Table 2)."""
     W = np.asarray(W16, dtype=np.float16).astype(np.float64)
     K, N = W.shape
-    layer = {"branch": branch, "rank": int(rank), "K": K, "N": N,
+    layer = {"branch": branch, "rank": int(rank), "K": K, "N": N, "main": main,
              "bias": None if bias is None else np.asarray(bias, dtype=np.float16)}
+
+    def store_main(P):
+        if main == "mxint4":
+            layer["Wq"], layer["ew"] = q_weight_main_mx(P)
+        else:
+            layer["Wq"], layer["sw"] = q_weight_main(P)
+
     if branch == "none" or rank == 0:
         layer["branch"], layer["rank"] = "none", 0
-        layer["Wq"], layer["sw"] = q_weight_main(W)
-        E = q1_dequant(W) - W
+        store_main(W)
+        E = q1_dequant(W, main) - W
         return layer, np.array([float(np.mean(E * E))])
 
     L0, R0 = svd_init(W, rank)
@@ -310,7 +321,7 @@ def calibrate(W16, rank: int, branch: str = "w8a8", steps: int = 1000, lr: float
     trace = np.zeros(steps + 1)
     best = (np.inf, None, None)
     for t in range(steps + 1):
-        loss, gL, gR = gradients(W, L, R)
+        loss, gL, gR = gradients(W, L, R, main)
         trace[t] = loss
         if loss < best[0]:
             best = (loss, L.copy(), R.copy())
@@ -334,14 +345,17 @@ def calibrate(W16, rank: int, branch: str = "w8a8", steps: int = 1000, lr: float
         layer["L1q"], layer["sL1"] = q_factor(L1, bw)
         layer["L2q"], layer["sL2"] = q_factor(L2, bw)
         D = deq_factor(layer["L1q"], layer["sL1"]) @ deq_factor(layer["L2q"], layer["sL2"])
-    layer["Wq"], layer["sw"] = q_weight_main(W - D)       # P = W - Q2(L1) Q2(L2), then Q1
+    store_main(W - D)                                     # P = W - Q2(L1) Q2(L2), then Q1
     return layer, trace
 
 
 def effective_weight(layer):
     """float64 [K, N]: deq(Q1(P)) + deq(Q2(L1)) deq(Q2(L2)) - what the layer multiplies by
     when activations are exact."""
-    Wd = deq_weight_main(layer["Wq"], layer["sw"])
+    if layer.get("main", "sint4") == "mxint4":
+        Wd = deq_mx(layer["Wq"].T.copy(), layer["ew"].T.copy()).T.copy()
+    else:
+        Wd = deq_weight_main(layer["Wq"], layer["sw"])
     if layer["branch"] == "none" or layer["rank"] == 0:
         return Wd
     if layer["branch"] == "w16a16":

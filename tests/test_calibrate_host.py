@@ -94,3 +94,29 @@ def test_rank0_and_round_trip_of_import_export():
         assert False
     except B.LqError as e:
         assert e.code == 1
+
+
+def test_mxint4_main_calibration():
+    """group = 32 selects the MXINT4 main branch (Table 2): exported scales are powers of two,
+    the objective goes down, and the stored codes are MXINT4 of P = W - Q2(L1) Q2(L2)."""
+    W = I.make_weight(0, 0, "pin-mx", 256, 192, 2)
+    cfg = B.lq_config_default(256, 192, 8, "w8a8"); cfg.steps = 100; cfg.group = 32
+    h, trace = B.lq_calibrate(cfg, W, want_trace=True)
+    _, tr_o = O.calibrate(W, 8, "w8a8", steps=0, main="mxint4")
+    assert abs(trace[0] - tr_o[0]) <= 1e-4 * tr_o[0]
+    assert np.minimum.accumulate(trace)[-1] < 0.98 * trace[0]
+    ex = B.lq_layer_export(h)
+    sw = ex["sw"].astype(np.float64)
+    assert sw.shape == (256 // 32, 192)
+    ew = np.log2(sw)
+    assert np.array_equal(ew, np.rint(ew))
+    Wq = B.unpack_nibbles(ex["Wq_packed"])
+    D = O.deq_factor(ex["L1"], ex["sL1"]) @ O.deq_factor(ex["L2"], ex["sL2"])
+    Wq_o, ew_o = O.q_weight_main_mx(W.astype(np.float64) - D)
+    assert np.mean(ew_o == ew) > 0.999 and np.mean(Wq_o == Wq) > 0.9999
+    # the calibrated layer beats plain MXINT4 rounding of W
+    layer = {"branch": "w8a8", "rank": 8, "K": 256, "N": 192, "bias": None, "main": "mxint4",
+             "Wq": Wq, "ew": ew.astype(np.int16), "L1q": ex["L1"], "sL1": ex["sL1"], "L2q": ex["L2"], "sL2": ex["sL2"]}
+    W64 = W.astype(np.float64)
+    assert np.linalg.norm(O.effective_weight(layer) - W64) < np.linalg.norm(O.q1_dequant(W64, "mxint4") - W64)
+    B.lq_layer_free(h)
