@@ -224,6 +224,19 @@ static lq_status make_tmap_bytes(CUtensorMap* tm, void* base, uint64_t rows, uin
   return r == CUDA_SUCCESS ? LQ_OK : LQ_ERR_CUDA;
 }
 
+lq_status lq_make_tmap_out_f16(CUtensorMap* tm, void* base, uint64_t rows, uint64_t cols, uint32_t box_cols, uint32_t box_rows) {
+  encode_tiled_fn fn = get_encode_fn();
+  if (!fn) return LQ_ERR_CUDA;
+  if (((uintptr_t)base & 15) || (cols % 8)) return LQ_ERR_INVALID_ARG;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? LQ_OK : LQ_ERR_CUDA;
+}
+
 // ---- device status word ------------------------------------------------------------------
 static int32_t* g_status[64] = {nullptr};
 static std::mutex g_status_mu;
@@ -301,7 +314,7 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
         for (int n = 0; n < N; ++n) {
           int x = 0;
           frexpf(h2f(L->sw[(size_t)g * N + n]), &x);              // 2^e = 0.5 * 2^(e+1)
-          sfb[lq_sf_offset(n, g, Kpad)] = (uint8_t)(x - 1 + 127);
+          sfb[lq_sfb_offset(n, g, Npad)] = (uint8_t)(x - 1 + 127);
         }
       if ((st = upload(&L->d_sfb, sfb)) != LQ_OK) return st;
     } else {
@@ -349,6 +362,7 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
     if ((st = upload(&L->d_L2c, l2c)) != LQ_OK) return st;
   } catch (const std::bad_alloc&) { return LQ_ERR_ALLOC; }
   if ((st = make_tmap_bytes(&L->tmB, L->d_Wq8, Npad, Kpad, LQ_BN)) != LQ_OK) return st;
+  if ((st = make_tmap_bytes(&L->tmB2, L->d_Wq8, Npad, Kpad, 2 * LQ_BN)) != LQ_OK) return st;
   if ((st = make_tmap_bytes(&L->tmL2, L->d_L2c, Npad, LQ_RCONT, LQ_BN)) != LQ_OK) return st;
   if (!lq_device_status_ptr(device)) return LQ_ERR_CUDA;
   if ((st = lq_gemm_prepare(device)) != LQ_OK) return st;

@@ -9,14 +9,22 @@
 // kernel.  Products q q' 2^(e+e') are exact in fp32; their sum is rounded by the tensor core's fp32 accumulation.
 //
 // Shape of the kernel (persistent, one CTA per SM, 18 warps):
-//   warp 0      TMA producer: per stage 128 bytes of K of A (128 rows) and B (256 rows) plus the stage's scale bytes
-//               (512 B per 128 rows: four K blocks, already in the 32 x 16-byte layout tensor memory wants)
+//   warp 0      TMA producer: per stage 128 bytes of K of A (128 rows) and B (256 rows, one box) plus the stage's scale
+//               bytes (512 B per 128 rows: four K blocks, already in the 32 x 16-byte layout tensor memory wants);
+//               per tile the vectors sT, sL2 and bias for the drain
 //   warp 1      owns tensor memory; per stage: tcgen05.cp of the scale bytes into tensor-memory columns, then four
 //               K = 32 block-scaled MMAs (N = 256) into the tile's accumulator; after the last stage the accumulator is
-//               handed to the drain; the low-rank branch's up-projection (kind::i8, fp32 scales that the tensor core
-//               cannot apply) then reuses the same columns and is handed over a second time
-//   warps 2-17  drain: tcgen05.ld the main accumulator into registers (+ bias), then the branch accumulator
-//               (x sT x sL2), convert, stage rows in shared memory and store whole row segments
+//               handed to the drain - once per tile
+//   warps 2-17  drain.  While the tensor core works on the tile they compute the low-rank branch's up-projection
+//               U = tq L2q for their part of it with mma.sync (int8 -> int32, exact; 1/36 .. 1/144 of the tile's
+//               work, operands read straight from global memory in fragment order), scale it by sT sL2 and add the
+//               bias.  When the accumulator arrives they read it with tcgen05.ld in the same fragment layout
+//               (16x256b), add, release it, and store: a 4 x 4 exchange inside each quad gives every lane 16
+//               contiguous bytes of one row; fp16 rows are staged in shared memory (dense 64-byte rows, conflict-free)
+//               and leave with one TMA store per warp and half, which clips ragged edges and does not hold the warp.
+// Per tile the drain's work (branch, hand-over, stores) must stay below the tile's main loop, or the tensor core
+// waits for the accumulator: hence the batched fragment loads, the scale vectors staged by the producer and the
+// asynchronous stores.
 // Every wait is bounded as in lq_gemm.cu.
 #include <cuda_fp16.h>
 
@@ -27,22 +35,22 @@ namespace {
 constexpr int UNIT = LQ_BN;                        // 128 output columns
 constexpr int NSTAGE = 3;                          // operand ring depth
 constexpr int STAGE_A_BYTES = LQ_BM * LQ_KSTAGE;   // 16 KB
-constexpr int STAGE_B_BYTES = 2 * UNIT * LQ_KSTAGE;   // 32 KB (two 128-row boxes)
+constexpr int STAGE_B_BYTES = 2 * UNIT * LQ_KSTAGE;   // 32 KB (one 256-row box, or one 128-row box for a narrow tile)
+constexpr int STAGE_BYTES = STAGE_A_BYTES + STAGE_B_BYTES;
 constexpr int SF_BYTES = 512;                      // scale bytes of 128 rows x 4 K blocks
-constexpr int STAGE_SF_OFF = STAGE_A_BYTES + STAGE_B_BYTES;            // SFA, then SFB of both halves
-constexpr int STAGE_BYTES = STAGE_SF_OFF + 2048;   // three scale blocks of 512 B, padded to keep the alignment
-constexpr int BR_FLOATS = LQ_BM + 2 * UNIT;        // branch stage: sT[128] then sL2[256]
+constexpr int STAGE_SF_BYTES = 3 * SF_BYTES;       // SFA, then SFB of both halves
+constexpr int SC_FLOATS = LQ_BM + 4 * UNIT;        // per tile: sT[128], sL2[256], bias[256]
 constexpr int NUM_DRAIN_WARPS = 16;
 constexpr int FIRST_DRAIN_WARP = 2;
 constexpr int GEMM_THREADS = (FIRST_DRAIN_WARP + NUM_DRAIN_WARPS) * 32;
-constexpr int OUT_ROW_BYTES = 128;                 // output bytes staged per row and pass
-constexpr int OUT_ROW_STRIDE = OUT_ROW_BYTES + 16;
-constexpr int OUT_WARP_BYTES = 32 * OUT_ROW_STRIDE;
+constexpr int OUT_UNIT_BYTES = 32 * 64;            // one warp's 32 rows x 32 fp16 columns of one half: a TMA store box
+constexpr int OUT_WARP_BYTES = 2 * OUT_UNIT_BYTES; // one buffer per half
 constexpr int SMEM_BAR_BYTES = 256;
-constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + NSTAGE * STAGE_BYTES + 2 * BR_FLOATS * 4 +
+constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + NSTAGE * STAGE_BYTES + NSTAGE * STAGE_SF_BYTES + 2 * SC_FLOATS * 4 +
                            NUM_DRAIN_WARPS * OUT_WARP_BYTES + SMEM_BAR_BYTES;
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 static_assert(STAGE_BYTES % 1024 == 0, "stages must keep the 1024-byte alignment of the swizzled tiles");
+static_assert((NSTAGE * STAGE_SF_BYTES + 2 * SC_FLOATS * 4) % 128 == 0, "store staging must stay 128-byte aligned");
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s at 2 GHz
 // tensor-memory columns: accumulator [0, 256), then per stage 4 columns of A scales and 8 of B scales
 constexpr int TM_SFA = 256, TM_SFB = TM_SFA + 4 * NSTAGE;
@@ -50,10 +58,12 @@ constexpr int TM_SFA = 256, TM_SFB = TM_SFA + 4 * NSTAGE;
 struct MxParams {
   int M, N, Mpad, Npad;
   int k_stages;           // Kpad / 128
-  int branch_mmas;        // 0: no branch; else MMAs of the branch stage (32 bytes of r each)
+  int branch_steps;       // 0: no branch; else 32-byte steps along r of the up-projection
   int tiles_m, units_n;
   const uint8_t* sfa;     // [Mpad/128][k_stages][512]
-  const uint8_t* sfb;     // [Npad/128][k_stages][512]
+  const uint8_t* sfb;     // [k_stages][Npad/128][512]: the scale bytes of two neighbouring 128-column units are contiguous
+  const uint8_t* tq;      // [Mpad][LQ_RCONT] int8 codes of the rank-r intermediate
+  const uint8_t* L2c;     // [Npad][LQ_RCONT] int8 codes of the second factor, r contiguous
   const float* sT;        // [Mpad]
   const float* sL2;       // [Npad]
   const float* bias;      // [Npad]
@@ -144,6 +154,18 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                : "memory");
 }
 
+// shared -> global tile store (clipped at the tensor's edges), tracked by the issuing thread's bulk groups
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(reinterpret_cast<uint64_t>(tm)),
+               "r"(x), "r"(y), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -173,15 +195,32 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t
   }
 }
 
-// 32 lanes x 16 consecutive 32-bit columns: thread t of the warp receives row (lane base + t).
-__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[16]) {
+// 16 lanes x 32 consecutive 32-bit columns in the accumulator-fragment layout of mma.sync m16n8: with g = lane / 4 and
+// t = lane % 4, registers 4j .. 4j+3 hold (row g, columns 8j + 2t, 8j + 2t + 1) and (row g + 8, the same columns).
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
         "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(taddr)
       : "memory");
+}
+// int8 x int8 -> int32 on the legacy tensor path: A 16 x 32 row-major, B 32 x 8 column-major fragments
+__device__ __forceinline__ void mma_s8_16x8x32(int (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// 4 x 4 transpose across the four lanes of a quad: afterwards v[s] of lane t is what v[t] of lane s was.
+__device__ __forceinline__ void quad_transpose(uint32_t (&v)[4], int t) {
+  const bool hi2 = (t & 2) != 0, hi1 = (t & 1) != 0;
+  uint32_t y0 = __shfl_xor_sync(0xffffffffu, hi2 ? v[0] : v[2], 2);
+  uint32_t y1 = __shfl_xor_sync(0xffffffffu, hi2 ? v[1] : v[3], 2);
+  if (hi2) { v[0] = y0; v[1] = y1; } else { v[2] = y0; v[3] = y1; }
+  y0 = __shfl_xor_sync(0xffffffffu, hi1 ? v[0] : v[1], 1);
+  y1 = __shfl_xor_sync(0xffffffffu, hi1 ? v[2] : v[3], 1);
+  if (hi1) { v[0] = y0; v[2] = y1; } else { v[1] = y0; v[3] = y1; }
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -226,15 +265,16 @@ __device__ __forceinline__ constexpr uint32_t idesc_mx(int n, int sf_id) {
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                  const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmL2, const MxParams p) {
+                  const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmY, const MxParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
-  constexpr int OFF_BR = NSTAGE * STAGE_BYTES;
-  constexpr int OFF_OUT = OFF_BR + 2 * BR_FLOATS * 4;
+  constexpr int OFF_SF = NSTAGE * STAGE_BYTES;
+  constexpr int OFF_SC = OFF_SF + NSTAGE * STAGE_SF_BYTES;
+  constexpr int OFF_OUT = OFF_SC + 2 * SC_FLOATS * 4;
   constexpr int OFF_BAR = OFF_OUT + NUM_DRAIN_WARPS * OUT_WARP_BYTES;
-  const uint32_t sm_stage = base, sm_br = base + OFF_BR, sm_bar = base + OFF_BAR;
-  const float* br_ptr = reinterpret_cast<const float*>(smem + OFF_BR);
+  const uint32_t sm_stage = base, sm_sf = base + OFF_SF, sm_sc = base + OFF_SC, sm_out = base + OFF_OUT, sm_bar = base + OFF_BAR;
+  const float* sc_ptr = reinterpret_cast<const float*>(smem + OFF_SC);
   uint8_t* out_ptr = smem + OFF_OUT;
   uint8_t* bar_ptr = smem + OFF_BAR;
   // barrier map (8 bytes each)
@@ -247,8 +287,6 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // provably warp-uniform
   const int lane = threadIdx.x & 31;
-  const bool has_branch = p.branch_mmas > 0;
-  const int stages_per_tile = p.k_stages + (has_branch ? 1 : 0);
   const long long units = (long long)p.tiles_m * p.units_n;
   const int u_begin = (int)((units * blockIdx.x) / gridDim.x);
   const int u_end = (int)((units * (blockIdx.x + 1)) / gridDim.x);
@@ -279,39 +317,36 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int mb = u / p.units_n, nu = u - mb * p.units_n;
       const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
       const int m0 = mb * LQ_BM, n0 = nu * UNIT;
-      for (int s = 0; s < stages_per_tile && ok; ++s, ++it) {
+      const uint8_t* sfa = p.sfa + (size_t)mb * p.k_stages * SF_BYTES;
+      const uint8_t* sfb = p.sfb + (size_t)nu * SF_BYTES;
+      {   // the tile's scale vectors and bias, for the drain
+        const int rb = tc & 1;
+        ok = mbar_wait_warp(bar(B_REMPTY + rb), ((tc >> 1) & 1) ^ 1, abort_flag, p.status, LQ_STAGE_PRODUCER);
+        if (!ok) break;
+        if (elect_one()) {
+          const uint32_t rfull = bar(B_RFULL + rb), dst = sm_sc + rb * SC_FLOATS * 4;
+          mbar_expect_tx(rfull, (LQ_BM + 2 * width * UNIT) * 4);
+          bulk_load(dst, p.sT + m0, LQ_BM * 4, rfull);
+          bulk_load(dst + LQ_BM * 4, p.sL2 + n0, width * UNIT * 4, rfull);
+          bulk_load(dst + (LQ_BM + 2 * UNIT) * 4, p.bias + n0, width * UNIT * 4, rfull);
+        }
+        __syncwarp();
+      }
+      for (int s = 0; s < p.k_stages && ok; ++s, ++it) {
         const int st = it % NSTAGE;
         ok = mbar_wait_warp(bar(B_EMPTY + st), ((it / NSTAGE) & 1) ^ 1, abort_flag, p.status, LQ_STAGE_PRODUCER);
         if (!ok) break;
-        const uint32_t a_dst = sm_stage + st * STAGE_BYTES, b_dst = a_dst + STAGE_A_BYTES, sf_dst = a_dst + STAGE_SF_OFF;
+        const uint32_t a_dst = sm_stage + st * STAGE_BYTES, b_dst = a_dst + STAGE_A_BYTES, sf_dst = sm_sf + st * STAGE_SF_BYTES;
         const uint32_t full = bar(B_FULL + st);
-        if (s < p.k_stages) {
-          if (elect_one()) {
-            mbar_expect_tx(full, STAGE_A_BYTES + width * (UNIT * LQ_KSTAGE) + (1 + width) * SF_BYTES);
-            tma_load_2d(a_dst, &tmA, s * LQ_KSTAGE, m0, full);
-            tma_load_2d(b_dst, &tmB, s * LQ_KSTAGE, n0, full);
-            if (width == 2) tma_load_2d(b_dst + UNIT * LQ_KSTAGE, &tmB, s * LQ_KSTAGE, n0 + UNIT, full);
-            bulk_load(sf_dst, p.sfa + ((size_t)mb * p.k_stages + s) * SF_BYTES, SF_BYTES, full);
-            for (int h = 0; h < width; ++h)
-              bulk_load(sf_dst + (1 + h) * SF_BYTES, p.sfb + ((size_t)(nu + h) * p.k_stages + s) * SF_BYTES, SF_BYTES, full);
-          }
-          __syncwarp();
-        } else {
-          const int rb = tc & 1;
-          ok = mbar_wait_warp(bar(B_REMPTY + rb), ((tc >> 1) & 1) ^ 1, abort_flag, p.status, LQ_STAGE_PRODUCER);
-          if (!ok) break;
-          if (elect_one()) {
-            mbar_expect_tx(full, STAGE_A_BYTES + width * (UNIT * LQ_KSTAGE));
-            tma_load_2d(a_dst, &tmT, 0, m0, full);
-            tma_load_2d(b_dst, &tmL2, 0, n0, full);
-            if (width == 2) tma_load_2d(b_dst + UNIT * LQ_KSTAGE, &tmL2, 0, n0 + UNIT, full);
-            const uint32_t rfull = bar(B_RFULL + rb);
-            mbar_expect_tx(rfull, (LQ_BM + width * UNIT) * 4);
-            bulk_load(sm_br + rb * BR_FLOATS * 4, p.sT + m0, LQ_BM * 4, rfull);
-            bulk_load(sm_br + rb * BR_FLOATS * 4 + LQ_BM * 4, p.sL2 + n0, width * UNIT * 4, rfull);
-          }
-          __syncwarp();
+        if (elect_one()) {
+          mbar_expect_tx(full, STAGE_A_BYTES + width * (UNIT * LQ_KSTAGE) + (1 + width) * SF_BYTES);
+          tma_load_2d(a_dst, &tmA, s * LQ_KSTAGE, m0, full);
+          if (width == 2) tma_load_2d(b_dst, &tmB2, s * LQ_KSTAGE, n0, full);
+          else tma_load_2d(b_dst, &tmB, s * LQ_KSTAGE, n0, full);
+          bulk_load(sf_dst, sfa + (size_t)s * SF_BYTES, SF_BYTES, full);
+          bulk_load(sf_dst + SF_BYTES, sfb + (size_t)s * p.units_n * SF_BYTES, width * SF_BYTES, full);
         }
+        __syncwarp();
       }
       u += width;
     }
@@ -321,14 +356,14 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    uint32_t it = 0, hv = 0;            // hv counts accumulator hand-overs (main, then branch, of every tile)
+    uint32_t it = 0, tc = 0;
     bool ok = true;
-    for (int u = u_begin; u < u_end && ok;) {
+    for (int u = u_begin; u < u_end && ok; ++tc) {
       const int mb = u / p.units_n, nu = u - mb * p.units_n;
       const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
       const int ncols = width * UNIT;
-      // the accumulator is free once the drain has read the previous hand-over
-      ok = mbar_wait_warp(bar(B_TEMPTY), (hv & 1) ^ 1, abort_flag, p.status, LQ_STAGE_MMA);
+      // the accumulator is free once the drain has read the previous tile out of it
+      ok = mbar_wait_warp(bar(B_TEMPTY), (tc & 1) ^ 1, abort_flag, p.status, LQ_STAGE_MMA);
       if (!ok) break;
       tc_fence_after();
       for (int s = 0; s < p.k_stages && ok; ++s, ++it) {
@@ -336,7 +371,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         ok = mbar_wait_warp(bar(B_FULL + st), (it / NSTAGE) & 1, abort_flag, p.status, LQ_STAGE_MMA);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t a_addr = sm_stage + st * STAGE_BYTES, b_addr = a_addr + STAGE_A_BYTES, sf_addr = a_addr + STAGE_SF_OFF;
+        const uint32_t a_addr = sm_stage + st * STAGE_BYTES, b_addr = a_addr + STAGE_A_BYTES, sf_addr = sm_sf + st * STAGE_SF_BYTES;
         const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
         const uint32_t tsfa = tmem_base + TM_SFA + st * 4, tsfb = tmem_base + TM_SFB + st * 8;
         if (elect_one()) {
@@ -353,147 +388,180 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       if (!ok) break;
       if (elect_one()) tc_commit(bar(B_TFULL));
       __syncwarp();
-      ++hv;
-      if (has_branch) {
-        const int st = it % NSTAGE;
-        ok = mbar_wait_warp(bar(B_FULL + st), (it / NSTAGE) & 1, abort_flag, p.status, LQ_STAGE_MMA);
-        if (!ok) break;
-        ok = mbar_wait_warp(bar(B_TEMPTY), (hv & 1) ^ 1, abort_flag, p.status, LQ_STAGE_MMA);   // main part is in registers
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t a_addr = sm_stage + st * STAGE_BYTES, b_addr = a_addr + STAGE_A_BYTES;
-        const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
-        if (elect_one()) {
-          for (int j = 0; j < p.branch_mmas; ++j) {
-            const uint64_t off = (uint64_t)((j * 32) >> 4);
-            tc_mma<0>(tmem_base, adesc + off, bdesc + off, IDESC_I8 | idesc_shape(ncols), (uint32_t)j);
-          }
-          tc_commit(bar(B_TFULL));
-          tc_commit(bar(B_EMPTY + st));
-        }
-        __syncwarp();
-        ++hv; ++it;
-      }
       u += width;
     }
   } else {
     // ------------------------------------------------------------------ drain + epilogue
     const int quad = warp & 3;                          // tensor-memory lanes 32*quad .. 32*quad+31
-    const int cgi = (warp - FIRST_DRAIN_WARP) >> 2;     // which 32 columns of each 128-column half
+    const int dw = warp - FIRST_DRAIN_WARP;
+    const int cgi = dw >> 2;                            // which 32 columns of each 128-column half
+    const int g = lane >> 2, t = lane & 3;              // fragment coordinates: rows g and g + 8, column pair t
     const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(cgi * 32);
-    uint8_t* out_row = out_ptr + (warp - FIRST_DRAIN_WARP) * OUT_WARP_BYTES + lane * OUT_ROW_STRIDE;
-    uint32_t hv = 0, tc = 0;
+    uint8_t* out_w = out_ptr + dw * OUT_WARP_BYTES;
+    const uint32_t out_w_s = sm_out + dw * OUT_WARP_BYTES;
+    uint32_t tc = 0;
     bool ok = true;
     for (int u = u_begin; u < u_end && ok; ++tc) {
       const int mb = u / p.units_n, nu = u - mb * p.units_n;
       const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
       const int m0 = mb * LQ_BM, n0 = nu * UNIT;
-      float acc[2][2][16];                              // [half][16-column chunk][column]
+      const int rl = quad * 32 + g;                     // this thread's rows inside the tile: rl + 16 mt and + 8
+      const int cl = cgi * 32;                          // this warp's columns inside a half: cl + 8 nt + ...
+      const int rb = tc & 1;
+      // acc[half][m16 tile][n8 tile][fragment register]: first the branch's int32 sums, then fp32 outputs
+      int acc[2][2][4][4];
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[h][mt][nt][i] = 0;
+      // branch part, while the tensor core works on the tile: U = tq L2q (exact int32).  All fragment loads of a step
+      // are issued before the first MMA so that they share one trip to the L2.
+      for (int kk = 0; kk < p.branch_steps; ++kk) {
+        uint32_t a[2][4], b[2][4][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          const uint8_t* ap = p.tq + (size_t)(m0 + rl + 16 * mt) * LQ_RCONT + kk * 32 + 4 * t;
+          a[mt][0] = __ldg(reinterpret_cast<const uint32_t*>(ap));
+          a[mt][1] = __ldg(reinterpret_cast<const uint32_t*>(ap + 8 * LQ_RCONT));
+          a[mt][2] = __ldg(reinterpret_cast<const uint32_t*>(ap + 16));
+          a[mt][3] = __ldg(reinterpret_cast<const uint32_t*>(ap + 8 * LQ_RCONT + 16));
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+          for (int nt = 0; nt < 4; ++nt) {
+            const int hh = h < width ? h : 0;           // a narrow tile reads the same (valid) rows twice and ignores them
+            const uint8_t* bp = p.L2c + (size_t)(n0 + hh * UNIT + cl + nt * 8 + g) * LQ_RCONT + kk * 32 + 4 * t;
+            b[h][nt][0] = __ldg(reinterpret_cast<const uint32_t*>(bp));
+            b[h][nt][1] = __ldg(reinterpret_cast<const uint32_t*>(bp + 16));
+          }
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+          if (h < width) {
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+              for (int mt = 0; mt < 2; ++mt) mma_s8_16x8x32(acc[h][mt][nt], a[mt], b[h][nt][0], b[h][nt][1]);
+          }
+      }
+      // y = U sT sL2 + bias  (|U| < 2^22: converted exactly with the 1.5 * 2^23 trick)
+      ok = mbar_wait(bar(B_RFULL + rb), (tc >> 1) & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
+      if (!ok) break;
+      {
+        const float* sc = sc_ptr + rb * SC_FLOATS;
+        float stv[2][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          stv[mt][0] = sc[rl + 16 * mt];
+          stv[mt][1] = sc[rl + 16 * mt + 8];
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (h < width) {
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+              const int c = h * UNIT + cl + nt * 8 + 2 * t;
+              const float2 sl = *reinterpret_cast<const float2*>(sc + LQ_BM + c);
+              const float2 bv = *reinterpret_cast<const float2*>(sc + LQ_BM + 2 * UNIT + c);
+#pragma unroll
+              for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const float uf = __int_as_float(acc[h][mt][nt][i] + 0x4B400000) - 12582912.0f;
+                  const float y = fmaf(uf, stv[mt][i >> 1] * ((i & 1) ? sl.y : sl.x), (i & 1) ? bv.y : bv.x);
+                  acc[h][mt][nt][i] = __float_as_int(y);
+                }
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_REMPTY + rb));
       // main part: the tensor core has already applied the block scales
-      ok = mbar_wait_idle(bar(B_TFULL), hv & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
+      ok = mbar_wait(bar(B_TFULL), tc & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
       if (!ok) break;
       tc_fence_after();
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         if (h < width) {
-          const float4* b4 = reinterpret_cast<const float4*>(p.bias + n0 + h * UNIT + cgi * 32);
 #pragma unroll
-          for (int ch = 0; ch < 2; ++ch) {
+          for (int mt = 0; mt < 2; ++mt) {
             uint32_t v[16];
-            tmem_ld_32x16(tlane + h * UNIT + ch * 16, v);
+            tmem_ld_16x256b_x4(tlane + ((uint32_t)(16 * mt) << 16) + h * UNIT, v);
             tmem_ld_wait();
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-              const float4 b = __ldg(b4 + 4 * ch + c4);
-              acc[h][ch][4 * c4 + 0] = __uint_as_float(v[4 * c4 + 0]) + b.x;
-              acc[h][ch][4 * c4 + 1] = __uint_as_float(v[4 * c4 + 1]) + b.y;
-              acc[h][ch][4 * c4 + 2] = __uint_as_float(v[4 * c4 + 2]) + b.z;
-              acc[h][ch][4 * c4 + 3] = __uint_as_float(v[4 * c4 + 3]) + b.w;
-            }
+            for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                acc[h][mt][nt][i] = __float_as_int(__int_as_float(acc[h][mt][nt][i]) + __uint_as_float(v[4 * nt + i]));
           }
         }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(B_TEMPTY));
-      ++hv;
-      // branch part: acc += U * (sT * sL2), U exact int32 (|U| < 2^22: converted exactly with the 1.5 * 2^23 trick)
-      if (has_branch) {
-        const int rb = tc & 1;
-        ok = mbar_wait(bar(B_RFULL + rb), (tc >> 1) & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
-        if (!ok) break;
-        ok = mbar_wait(bar(B_TFULL), hv & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
-        if (!ok) break;
-        tc_fence_after();
-        const float* br = br_ptr + rb * BR_FLOATS;
-        const float stv = br[quad * 32 + lane];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          if (h < width) {
-            const float* sl2 = br + LQ_BM + h * UNIT + cgi * 32;
-#pragma unroll
-            for (int ch = 0; ch < 2; ++ch) {
-              uint32_t v[16];
-              tmem_ld_32x16(tlane + h * UNIT + ch * 16, v);
-              tmem_ld_wait();
-#pragma unroll
-              for (int c = 0; c < 16; ++c) {
-                const float uf = __int_as_float((int)v[c] + 0x4B400000) - 12582912.0f;
-                acc[h][ch][c] = fmaf(uf, stv * sl2[ch * 16 + c], acc[h][ch][c]);
-              }
-            }
-          }
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) { mbar_arrive(bar(B_TEMPTY)); mbar_arrive(bar(B_REMPTY + rb)); }
-        ++hv;
-      }
-      // epilogue: convert, stage this thread's 32-column row segment of each half in the warp's shared-memory
-      // rows, read it back with lanes along the row and store whole 64/128-byte row segments
-      const int rbase = m0 + quad * 32;
-      const int esize = p.out_f32 ? 4 : 2;
-      const int lpr = 32 * esize / 16;                                   // lanes per row: 4 (fp16) or 8 (fp32)
-      const int rpi = 32 / lpr;                                          // rows per instruction
-      const int cpl = 16 / esize;                                        // columns per lane
+      // epilogue
+      const int row_w = m0 + quad * 32;                 // first row of this warp's part
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         if (h < width) {
-          __syncwarp();                                                  // the previous half has been read back
+          const int col_w = n0 + h * UNIT + cl;         // first column of this warp's part of the half
           if (p.out_f32) {
+            float* Y = reinterpret_cast<float*>(p.Y);
 #pragma unroll
-            for (int cc = 0; cc < 2; ++cc)
+            for (int mt = 0; mt < 2; ++mt) {
+              const int r_lo = row_w + g + 16 * mt, r_hi = r_lo + 8;
 #pragma unroll
-              for (int c4 = 0; c4 < 4; ++c4)
-                *reinterpret_cast<float4*>(out_row + cc * 64 + c4 * 16) =
-                    make_float4(acc[h][cc][4 * c4], acc[h][cc][4 * c4 + 1], acc[h][cc][4 * c4 + 2], acc[h][cc][4 * c4 + 3]);
-          } else {
-#pragma unroll
-            for (int cc = 0; cc < 2; ++cc)
-#pragma unroll
-              for (int c8 = 0; c8 < 2; ++c8) {
-                __half2 hh[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) hh[j] = __floats2half2_rn(acc[h][cc][c8 * 8 + 2 * j], acc[h][cc][c8 * 8 + 2 * j + 1]);
-                *reinterpret_cast<uint4*>(out_row + cc * 32 + c8 * 16) = *reinterpret_cast<uint4*>(hh);
+              for (int nt = 0; nt < 4; ++nt) {
+                const int c = col_w + nt * 8 + 2 * t;
+                if (c < p.N) {
+                  if (r_lo < p.M)
+                    *reinterpret_cast<float2*>(Y + (size_t)r_lo * p.N + c) =
+                        make_float2(__int_as_float(acc[h][mt][nt][0]), __int_as_float(acc[h][mt][nt][1]));
+                  if (r_hi < p.M)
+                    *reinterpret_cast<float2*>(Y + (size_t)r_hi * p.N + c) =
+                        make_float2(__int_as_float(acc[h][mt][nt][2]), __int_as_float(acc[h][mt][nt][3]));
+                }
               }
-          }
-          __syncwarp();
-          const int lcol = n0 + h * UNIT + cgi * 32 + (lane % lpr) * cpl;
-          const uint8_t* wbase = out_ptr + (warp - FIRST_DRAIN_WARP) * OUT_WARP_BYTES + (lane % lpr) * 16;
+            }
+          } else {
+            // The half's buffer was last read by the store of the previous tile: at most this tile's other half may
+            // still be in flight.
+            if (lane == 0) { if (h == 0) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
+            __syncwarp();
+            uint8_t* buf = out_w + h * OUT_UNIT_BYTES;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            if (i * rpi < 32) {
-              const int rl = i * rpi + lane / lpr;
-              const uint4 val = *reinterpret_cast<const uint4*>(wbase + rl * OUT_ROW_STRIDE);
-              if (rbase + rl < p.M && lcol < p.N)
-                *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.Y) + ((size_t)(rbase + rl) * p.N + lcol) * esize) = val;
+            for (int mt = 0; mt < 2; ++mt) {
+              // pack to fp16, then exchange inside the quad: lane t ends up with columns 8 t .. 8 t + 7 of both rows
+              uint32_t lo[4], hi[4];
+#pragma unroll
+              for (int nt = 0; nt < 4; ++nt) {
+                const __half2 l2 = __floats2half2_rn(__int_as_float(acc[h][mt][nt][0]), __int_as_float(acc[h][mt][nt][1]));
+                const __half2 h2 = __floats2half2_rn(__int_as_float(acc[h][mt][nt][2]), __int_as_float(acc[h][mt][nt][3]));
+                lo[nt] = *reinterpret_cast<const uint32_t*>(&l2);
+                hi[nt] = *reinterpret_cast<const uint32_t*>(&h2);
+              }
+              quad_transpose(lo, t);
+              quad_transpose(hi, t);
+              *reinterpret_cast<uint4*>(buf + (16 * mt + g) * 64 + 16 * t) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+              *reinterpret_cast<uint4*>(buf + (16 * mt + g + 8) * 64 + 16 * t) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              if (col_w < p.N && row_w < p.M) tma_store_2d(&tmY, col_w, row_w, out_w_s + h * OUT_UNIT_BYTES);
+              bulk_commit();
             }
           }
         }
       }
       u += width;
     }
+    if (lane == 0) bulk_wait_all();                      // the staged rows must stay until the last store has read them
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -521,10 +589,10 @@ lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_
   MxParams p;
   p.M = A->M; p.N = L->N; p.Mpad = A->Mpad; p.Npad = L->Npad;
   p.k_stages = L->Kpad / LQ_KSTAGE;
-  p.branch_mmas = L->r == 0 ? 0 : lq_ceil_div(L->r, 32);
+  p.branch_steps = L->r == 0 ? 0 : lq_ceil_div(L->r, 32);
   p.tiles_m = lq_ceil_div(A->M, LQ_BM);
   p.units_n = L->Npad / UNIT;
-  p.sfa = A->d_sfa; p.sfb = L->d_sfb; p.sT = A->d_sT; p.sL2 = L->d_sL2; p.bias = L->d_bias;
+  p.sfa = A->d_sfa; p.sfb = L->d_sfb; p.tq = A->d_tq; p.L2c = L->d_L2c; p.sT = A->d_sT; p.sL2 = L->d_sL2; p.bias = L->d_bias;
   p.Y = Y; p.out_f32 = dt == LQ_OUT_F32 ? 1 : 0;
   p.status = lq_device_status_ptr(A->device);
   if (!p.status) return LQ_ERR_CUDA;
@@ -533,6 +601,13 @@ lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_
   int ctas = g_lq_gemm_ctas > 0 ? g_lq_gemm_ctas : sms;
   const long long units = (long long)p.tiles_m * p.units_n;
   if (ctas > units) ctas = (int)units;
-  lq_gemm_mx_kernel<<<ctas, GEMM_THREADS, SMEM_BYTES, st>>>(A->tmA, L->tmB, A->tmT, L->tmL2, p);
+  // fp16 rows leave through TMA stores: a tensor map over the caller's Y (32 x 32 boxes, clipped at M and N); the fp32
+  // variant stores from registers and does not use it
+  CUtensorMap tmY = A->tmA;
+  if (dt == LQ_OUT_F16) {
+    const lq_status ts = lq_make_tmap_out_f16(&tmY, Y, (uint64_t)A->M, (uint64_t)L->N, 32, 32);
+    if (ts != LQ_OK) return ts;
+  }
+  lq_gemm_mx_kernel<<<ctas, GEMM_THREADS, SMEM_BYTES, st>>>(A->tmA, L->tmB, L->tmB2, tmY, p);
   return lq_note_cuda(cudaGetLastError()) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
 }

@@ -32,6 +32,11 @@ static inline size_t lq_sf_offset(int i, int kb, int Kpad) {
   return ((size_t)(i / 128) * (Kpad / 128) + kb / 4) * 512 + 16 * (i % 32) + 4 * ((i % 128) / 32) + kb % 4;
 }
 
+// the same for the weight scales, whose chunks are ordered [kb/4][tile] so that neighbouring column tiles are contiguous
+static inline size_t lq_sfb_offset(int n, int kb, int Npad) {
+  return ((size_t)(kb / 4) * (Npad / 128) + n / 128) * 512 + 16 * (n % 32) + 4 * ((n % 128) / 32) + kb % 4;
+}
+
 static inline int lq_branch_wbits(int branch) {
   return branch == LQ_BRANCH_W8A8 ? 8 : branch == LQ_BRANCH_W6A6 ? 6 : branch == LQ_BRANCH_W4A8 ? 4 : 0;
 }
@@ -65,9 +70,10 @@ struct lq_layer {
   uint8_t* d_L2c;              // [Npad][LQ_RCONT] bytes: int8 codes (or up to 64 halves) of column n, r contiguous
   float* d_sL2;                // [Npad]  (ones for W16A16)
   float* d_bias;               // [Npad]  (zeros without bias)
-  uint8_t* d_sfb;              // MXINT4: E8M0 bytes of the weight scales, [Npad/128][Kpad/128][512] in the 32 x 16-byte
+  uint8_t* d_sfb;              // MXINT4: E8M0 bytes of the weight scales, [Kpad/128][Npad/128][512] in the 32 x 16-byte
                                // layout tensor memory wants (byte 16*(n%32) + 4*((n%128)/32) + block%4)
   CUtensorMap tmB;             // over d_Wq8, box [LQ_BN][128B], 128B swizzle
+  CUtensorMap tmB2;            // over d_Wq8, box [2 LQ_BN][128B]: both halves of a 256-column tile in one copy
   CUtensorMap tmL2;            // over d_L2c, box [LQ_BN][128B], 128B swizzle
 };
 
@@ -105,6 +111,8 @@ lq_status lq_launch_gemm(const lq_layer* L, const lq_act* A, void* Y, lq_out_dty
 lq_status lq_gemm_prepare(int device);
 lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_dtype dt, cudaStream_t st);
 lq_status lq_gemm_mx_prepare(int device);
+// tensor map over an fp16 output [rows][cols] in the caller's memory (16-byte aligned, cols % 8 == 0), no swizzle
+lq_status lq_make_tmap_out_f16(CUtensorMap* tm, void* base, uint64_t rows, uint64_t cols, uint32_t box_cols, uint32_t box_rows);
 lq_status lq_launch_wait_probe(int device, cudaStream_t st);   // bounded-wait self-test kernel   // sets the kernel's shared-memory attribute once per device
 
 // byte an MMA operand carries for a 4-bit code q in [-7, 7]
