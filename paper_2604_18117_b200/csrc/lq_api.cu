@@ -224,19 +224,6 @@ static lq_status make_tmap_bytes(CUtensorMap* tm, void* base, uint64_t rows, uin
   return r == CUDA_SUCCESS ? LQ_OK : LQ_ERR_CUDA;
 }
 
-lq_status lq_make_tmap_out_f16(CUtensorMap* tm, void* base, uint64_t rows, uint64_t cols, uint32_t box_cols, uint32_t box_rows) {
-  encode_tiled_fn fn = get_encode_fn();
-  if (!fn) return LQ_ERR_CUDA;
-  if (((uintptr_t)base & 15) || (cols % 8)) return LQ_ERR_INVALID_ARG;
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
-  cuuint32_t box[2] = {box_cols, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? LQ_OK : LQ_ERR_CUDA;
-}
-
 // ---- device status word ------------------------------------------------------------------
 static int32_t* g_status[64] = {nullptr};
 static std::mutex g_status_mu;

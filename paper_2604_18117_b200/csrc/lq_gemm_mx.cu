@@ -11,20 +11,25 @@
 // Shape of the kernel (persistent, one CTA per SM, 18 warps):
 //   warp 0      TMA producer: per stage 128 bytes of K of A (128 rows) and B (256 rows, one box) plus the stage's scale
 //               bytes (512 B per 128 rows: four K blocks, already in the 32 x 16-byte layout tensor memory wants);
-//               per tile the vectors sT, sL2 and bias for the drain
+//               per tile one more stage with the branch operands (tq, L2q) and the vectors sT, sL2, bias for the drain
 //   warp 1      owns tensor memory; per stage: tcgen05.cp of the scale bytes into tensor-memory columns, then four
-//               K = 32 block-scaled MMAs (N = 256) into the tile's accumulator; after the last stage the accumulator is
-//               handed to the drain - once per tile
-//   warps 2-17  drain.  While the tensor core works on the tile they compute the low-rank branch's up-projection
-//               U = tq L2q for their part of it with mma.sync (int8 -> int32, exact; 1/36 .. 1/144 of the tile's
-//               work, operands read straight from global memory in fragment order), scale it by sT sL2 and add the
-//               bias.  When the accumulator arrives they read it with tcgen05.ld in the same fragment layout
-//               (16x256b), add, release it, and store: a 4 x 4 exchange inside each quad gives every lane 16
-//               contiguous bytes of one row; fp16 rows are staged in shared memory (dense 64-byte rows, conflict-free)
-//               and leave with one TMA store per warp and half, which clips ragged edges and does not hold the warp.
-// Per tile the drain's work (branch, hand-over, stores) must stay below the tile's main loop, or the tensor core
-// waits for the accumulator: hence the batched fragment loads, the scale vectors staged by the producer and the
-// asynchronous stores.
+//               K = 32 block-scaled MMAs (N = 256) into the tile's accumulator; after the last stage the low-rank
+//               branch's up-projection U = tq L2q (kind::i8, exact int32; its fp32 scales cannot be applied by the
+//               tensor core) into a second accumulator, then ONE hand-over of both to the drain
+//   warps 2-17  drain: tcgen05.ld the main accumulator (mma.sync fragment layout, 16x256b) straight into registers and
+//               release it - the next tile's main loop starts - then read the branch accumulator,
+//               y = main + sT sL2 U + bias, release that too, convert; a 4 x 4 exchange inside each quad gives
+//               every lane 16 contiguous bytes of one row, so each store instruction writes whole 32-byte sectors
+//               straight from registers.
+// Tensor memory has 512 columns: main accumulator [0, 256), branch accumulator [256, 512).  The 12 scale-factor
+// columns of a stage (one slot: the tensor pipe executes one thread's tcgen05 copies and MMAs in issue order) alias the
+// first 16 columns of the branch accumulator: they are live only while the tile's block-scaled MMAs run, the branch
+// accumulator only from the branch MMA (issued after them) until the drain has read it.  The four drain warps that own
+// those 16 columns read them together with the main accumulator, before the hand-over; the rest of the branch
+// accumulator is read afterwards, under the next tile's main loop, and is needed again only by that tile's branch MMA.
+// What was measured on the way here (PixArt block, four GEMMs): the branch on mma.sync in the drain warps took tensor
+// time from the main loop; TMA stores of the output (32 boxes of 2 KB, or 8 of 8 KB, per tile) cost 15 % against
+// plain stores - they share the TMA unit with the operand loads; a fourth ring stage gained 3 %.
 // Every wait is bounded as in lq_gemm.cu.
 #include <cuda_fp16.h>
 
@@ -33,7 +38,7 @@
 namespace {
 
 constexpr int UNIT = LQ_BN;                        // 128 output columns
-constexpr int NSTAGE = 3;                          // operand ring depth
+constexpr int NSTAGE = 4;                          // operand ring depth
 constexpr int STAGE_A_BYTES = LQ_BM * LQ_KSTAGE;   // 16 KB
 constexpr int STAGE_B_BYTES = 2 * UNIT * LQ_KSTAGE;   // 32 KB (one 256-row box, or one 128-row box for a narrow tile)
 constexpr int STAGE_BYTES = STAGE_A_BYTES + STAGE_B_BYTES;
@@ -43,27 +48,24 @@ constexpr int SC_FLOATS = LQ_BM + 4 * UNIT;        // per tile: sT[128], sL2[256
 constexpr int NUM_DRAIN_WARPS = 16;
 constexpr int FIRST_DRAIN_WARP = 2;
 constexpr int GEMM_THREADS = (FIRST_DRAIN_WARP + NUM_DRAIN_WARPS) * 32;
-constexpr int OUT_UNIT_BYTES = 32 * 64;            // one warp's 32 rows x 32 fp16 columns of one half: a TMA store box
-constexpr int OUT_WARP_BYTES = 2 * OUT_UNIT_BYTES; // one buffer per half
 constexpr int SMEM_BAR_BYTES = 256;
 constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + NSTAGE * STAGE_BYTES + NSTAGE * STAGE_SF_BYTES + 2 * SC_FLOATS * 4 +
-                           NUM_DRAIN_WARPS * OUT_WARP_BYTES + SMEM_BAR_BYTES;
+                           SMEM_BAR_BYTES;
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 static_assert(STAGE_BYTES % 1024 == 0, "stages must keep the 1024-byte alignment of the swizzled tiles");
-static_assert((NSTAGE * STAGE_SF_BYTES + 2 * SC_FLOATS * 4) % 128 == 0, "store staging must stay 128-byte aligned");
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s at 2 GHz
-// tensor-memory columns: accumulator [0, 256), then per stage 4 columns of A scales and 8 of B scales
-constexpr int TM_SFA = 256, TM_SFB = TM_SFA + 4 * NSTAGE;
+// tensor-memory columns: main accumulator [0, 256), branch accumulator [256, 512); 4 columns of A scales and 8 of B
+// scales alias the start of the branch accumulator (disjoint lifetimes, see the top of the file)
+constexpr int TM_BR = 256, TM_SFA = 256, TM_SFB = TM_SFA + 4, TM_SF_ALIASED = 16;
 
 struct MxParams {
   int M, N, Mpad, Npad;
   int k_stages;           // Kpad / 128
-  int branch_steps;       // 0: no branch; else 32-byte steps along r of the up-projection
+  int branch_steps;       // 0: no branch; else MMAs of the branch stage (32 bytes of r each)
   int tiles_m, units_n;
+  int by_units;           // how the CTAs share the work: 0 whole tiles, 1 128-column units
   const uint8_t* sfa;     // [Mpad/128][k_stages][512]
   const uint8_t* sfb;     // [k_stages][Npad/128][512]: the scale bytes of two neighbouring 128-column units are contiguous
-  const uint8_t* tq;      // [Mpad][LQ_RCONT] int8 codes of the rank-r intermediate
-  const uint8_t* L2c;     // [Npad][LQ_RCONT] int8 codes of the second factor, r contiguous
   const float* sT;        // [Mpad]
   const float* sL2;       // [Npad]
   const float* bias;      // [Npad]
@@ -154,18 +156,6 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                : "memory");
 }
 
-// shared -> global tile store (clipped at the tensor's edges), tracked by the issuing thread's bulk groups
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, int x, int y, uint32_t src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(reinterpret_cast<uint64_t>(tm)),
-               "r"(x), "r"(y), "r"(src)
-               : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -206,12 +196,6 @@ __device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&v)
       : "r"(taddr)
       : "memory");
 }
-// int8 x int8 -> int32 on the legacy tensor path: A 16 x 32 row-major, B 32 x 8 column-major fragments
-__device__ __forceinline__ void mma_s8_16x8x32(int (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-               : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 // 4 x 4 transpose across the four lanes of a quad: afterwards v[s] of lane t is what v[t] of lane s was.
 __device__ __forceinline__ void quad_transpose(uint32_t (&v)[4], int t) {
   const bool hi2 = (t & 2) != 0, hi1 = (t & 1) != 0;
@@ -221,6 +205,12 @@ __device__ __forceinline__ void quad_transpose(uint32_t (&v)[4], int t) {
   y0 = __shfl_xor_sync(0xffffffffu, hi1 ? v[0] : v[1], 1);
   y1 = __shfl_xor_sync(0xffffffffu, hi1 ? v[2] : v[3], 1);
   if (hi1) { v[0] = y0; v[2] = y1; } else { v[1] = y0; v[3] = y1; }
+}
+__device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, uint32_t (&v)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(taddr)
+               : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -263,23 +253,37 @@ __device__ __forceinline__ constexpr uint32_t idesc_mx(int n, int sf_id) {
   return ((uint32_t)sf_id << 4) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(LQ_BM >> 4) << 24) | ((uint32_t)sf_id << 29);
 }
 
+// y = main + U sT sL2 + bias for one n8 fragment (registers: row g columns 2t, 2t+1, then row g + 8 the same columns).
+// U is an exact int32 with |U| < 2^22: converted exactly with the 1.5 * 2^23 trick.
+__device__ __forceinline__ void combine_fragment(float (&a)[4], const uint32_t* u, bool has_branch, float st_lo, float st_hi,
+                                                 float2 sl, float2 bv) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float y = a[i] + ((i & 1) ? bv.y : bv.x);
+    if (has_branch) {
+      const float uf = __int_as_float((int)u[i] + 0x4B400000) - 12582912.0f;
+      y = fmaf(uf, ((i >> 1) ? st_hi : st_lo) * ((i & 1) ? sl.y : sl.x), y);
+    }
+    a[i] = y;
+  }
+}
+
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                  const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmY, const MxParams p) {
+                  const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmT,
+                  const __grid_constant__ CUtensorMap tmL2, const MxParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem = smem_raw + (base - smem_u32(smem_raw));
   constexpr int OFF_SF = NSTAGE * STAGE_BYTES;
   constexpr int OFF_SC = OFF_SF + NSTAGE * STAGE_SF_BYTES;
-  constexpr int OFF_OUT = OFF_SC + 2 * SC_FLOATS * 4;
-  constexpr int OFF_BAR = OFF_OUT + NUM_DRAIN_WARPS * OUT_WARP_BYTES;
-  const uint32_t sm_stage = base, sm_sf = base + OFF_SF, sm_sc = base + OFF_SC, sm_out = base + OFF_OUT, sm_bar = base + OFF_BAR;
+  constexpr int OFF_BAR = OFF_SC + 2 * SC_FLOATS * 4;
+  const uint32_t sm_stage = base, sm_sf = base + OFF_SF, sm_sc = base + OFF_SC, sm_bar = base + OFF_BAR;
   const float* sc_ptr = reinterpret_cast<const float*>(smem + OFF_SC);
-  uint8_t* out_ptr = smem + OFF_OUT;
   uint8_t* bar_ptr = smem + OFF_BAR;
   // barrier map (8 bytes each)
   constexpr int B_FULL = 0, B_EMPTY = NSTAGE, B_TFULL = 2 * NSTAGE, B_TEMPTY = B_TFULL + 1, B_RFULL = B_TEMPTY + 1,
-                B_REMPTY = B_RFULL + 2, NBAR = B_REMPTY + 2;
+                B_REMPTY = B_RFULL + 2, B_BEMPTY = B_REMPTY + 2, NBAR = B_BEMPTY + 1;
   auto bar = [&](int idx) { return sm_bar + 8u * (uint32_t)idx; };
   static_assert(NBAR * 8 + 16 <= SMEM_BAR_BYTES, "barrier area too small");
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + NBAR * 8);
@@ -287,15 +291,34 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // provably warp-uniform
   const int lane = threadIdx.x & 31;
-  const long long units = (long long)p.tiles_m * p.units_n;
-  const int u_begin = (int)((units * blockIdx.x) / gridDim.x);
-  const int u_end = (int)((units * (blockIdx.x + 1)) / gridDim.x);
+  const bool has_branch = p.branch_steps > 0;
+  // Each CTA takes a contiguous, equal share of the work and walks it as 256-wide tiles (128-wide where a row block or
+  // the share ends).  A 128-wide tile costs nearly as much as a 256-wide one (a stage's time is set by its hand-shakes
+  // and instruction count, not its MMA width).  by_units = 0 shares whole tiles - row blocks cut into 256-wide tiles
+  // plus at most one 128-wide one - which avoids needless narrow tiles; by_units = 1 shares 128-column units, which
+  // balances better when a CTA gets only two or three tiles and the row blocks have an odd number of units.
+  const int tiles_n = (p.units_n + 1) >> 1;
+  const long long work = (long long)p.tiles_m * (p.by_units ? p.units_n : tiles_n);
+  const int w_begin = (int)((work * blockIdx.x) / gridDim.x);
+  const int w_end = (int)((work * (blockIdx.x + 1)) / gridDim.x);
+  // position w -> row block, first unit and width of the tile that starts there
+  auto tile_at = [&](int w, int& mb, int& nu, int& width) {
+    if (p.by_units) {
+      mb = w / p.units_n; nu = w - mb * p.units_n;
+      width = (nu + 1 < p.units_n && w + 1 < w_end) ? 2 : 1;
+      return w + width;
+    }
+    mb = w / tiles_n; nu = 2 * (w - mb * tiles_n);
+    width = (nu + 1 < p.units_n) ? 2 : 1;
+    return w + 1;
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < NSTAGE; ++s) { mbar_init(bar(B_FULL + s), 1); mbar_init(bar(B_EMPTY + s), 1); }
     mbar_init(bar(B_TFULL), 1);
     mbar_init(bar(B_TEMPTY), NUM_DRAIN_WARPS);
     for (int b = 0; b < 2; ++b) { mbar_init(bar(B_RFULL + b), 1); mbar_init(bar(B_REMPTY + b), NUM_DRAIN_WARPS); }
+    mbar_init(bar(B_BEMPTY), NUM_DRAIN_WARPS);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -313,9 +336,9 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // ------------------------------------------------------------------ TMA producer
     uint32_t it = 0, tc = 0;
     bool ok = true;
-    for (int u = u_begin; u < u_end && ok; ++tc) {
-      const int mb = u / p.units_n, nu = u - mb * p.units_n;
-      const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
+    for (int w = w_begin, w_next; w < w_end && ok; w = w_next, ++tc) {
+      int mb, nu, width;
+      w_next = tile_at(w, mb, nu, width);
       const int m0 = mb * LQ_BM, n0 = nu * UNIT;
       const uint8_t* sfa = p.sfa + (size_t)mb * p.k_stages * SF_BYTES;
       const uint8_t* sfb = p.sfb + (size_t)nu * SF_BYTES;
@@ -348,7 +371,21 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
         __syncwarp();
       }
-      u += width;
+      if (has_branch && ok) {   // the branch operands: the containers of tq (128 rows) and L2q (256 rows), r contiguous
+        const int st = it % NSTAGE;
+        ok = mbar_wait_warp(bar(B_EMPTY + st), ((it / NSTAGE) & 1) ^ 1, abort_flag, p.status, LQ_STAGE_PRODUCER);
+        if (!ok) break;
+        const uint32_t a_dst = sm_stage + st * STAGE_BYTES, b_dst = a_dst + STAGE_A_BYTES;
+        const uint32_t full = bar(B_FULL + st);
+        if (elect_one()) {
+          mbar_expect_tx(full, STAGE_A_BYTES + width * (UNIT * LQ_KSTAGE));
+          tma_load_2d(a_dst, &tmT, 0, m0, full);
+          tma_load_2d(b_dst, &tmL2, 0, n0, full);
+          if (width == 2) tma_load_2d(b_dst + UNIT * LQ_KSTAGE, &tmL2, 0, n0 + UNIT, full);
+        }
+        __syncwarp();
+        ++it;
+      }
     }
     if (!ok) {   // let copies in flight land before the CTA's shared memory goes away
       const long long t0 = clock64();
@@ -358,9 +395,9 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // ------------------------------------------------------------------ MMA issuer
     uint32_t it = 0, tc = 0;
     bool ok = true;
-    for (int u = u_begin; u < u_end && ok; ++tc) {
-      const int mb = u / p.units_n, nu = u - mb * p.units_n;
-      const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
+    for (int w = w_begin, w_next; w < w_end && ok; w = w_next, ++tc) {
+      int mb, nu, width;
+      w_next = tile_at(w, mb, nu, width);
       const int ncols = width * UNIT;
       // the accumulator is free once the drain has read the previous tile out of it
       ok = mbar_wait_warp(bar(B_TEMPTY), (tc & 1) ^ 1, abort_flag, p.status, LQ_STAGE_MMA);
@@ -373,7 +410,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         tc_fence_after();
         const uint32_t a_addr = sm_stage + st * STAGE_BYTES, b_addr = a_addr + STAGE_A_BYTES, sf_addr = sm_sf + st * STAGE_SF_BYTES;
         const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
-        const uint32_t tsfa = tmem_base + TM_SFA + st * 4, tsfb = tmem_base + TM_SFB + st * 8;
+        const uint32_t tsfa = tmem_base + TM_SFA, tsfb = tmem_base + TM_SFB;
         if (elect_one()) {
           tc_cp_sf(tsfa, make_smem_desc_plain(sf_addr, 16, 128));
           tc_cp_sf(tsfb, make_smem_desc_plain(sf_addr + SF_BYTES, 16, 128));
@@ -386,130 +423,112 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         __syncwarp();
       }
       if (!ok) break;
+      if (has_branch) {
+        const int st = it % NSTAGE;
+        ok = mbar_wait_warp(bar(B_FULL + st), (it / NSTAGE) & 1, abort_flag, p.status, LQ_STAGE_MMA);
+        if (!ok) break;
+        // the drain has read the previous tile's branch accumulator (long ago: it does that under this tile's main loop)
+        ok = mbar_wait_warp(bar(B_BEMPTY), (tc & 1) ^ 1, abort_flag, p.status, LQ_STAGE_MMA);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a_addr = sm_stage + st * STAGE_BYTES, b_addr = a_addr + STAGE_A_BYTES;
+        const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
+        if (elect_one()) {
+          for (int j = 0; j < p.branch_steps; ++j)
+            tc_mma<0>(tmem_base + TM_BR, adesc + 2 * j, bdesc + 2 * j, IDESC_I8 | idesc_shape(ncols), (uint32_t)j);
+          tc_commit(bar(B_EMPTY + st));
+        }
+        __syncwarp();
+        ++it;
+      }
       if (elect_one()) tc_commit(bar(B_TFULL));
       __syncwarp();
-      u += width;
     }
   } else {
     // ------------------------------------------------------------------ drain + epilogue
     const int quad = warp & 3;                          // tensor-memory lanes 32*quad .. 32*quad+31
-    const int dw = warp - FIRST_DRAIN_WARP;
-    const int cgi = dw >> 2;                            // which 32 columns of each 128-column half
+    const int cgi = (warp - FIRST_DRAIN_WARP) >> 2;     // which 32 columns of each 128-column half
     const int g = lane >> 2, t = lane & 3;              // fragment coordinates: rows g and g + 8, column pair t
     const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(cgi * 32);
-    uint8_t* out_w = out_ptr + dw * OUT_WARP_BYTES;
-    const uint32_t out_w_s = sm_out + dw * OUT_WARP_BYTES;
     uint32_t tc = 0;
     bool ok = true;
-    for (int u = u_begin; u < u_end && ok; ++tc) {
-      const int mb = u / p.units_n, nu = u - mb * p.units_n;
-      const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
+    for (int w = w_begin, w_next; w < w_end && ok; w = w_next, ++tc) {
+      int mb, nu, width;
+      w_next = tile_at(w, mb, nu, width);
       const int m0 = mb * LQ_BM, n0 = nu * UNIT;
       const int rl = quad * 32 + g;                     // this thread's rows inside the tile: rl + 16 mt and + 8
       const int cl = cgi * 32;                          // this warp's columns inside a half: cl + 8 nt + ...
       const int rb = tc & 1;
-      // acc[half][m16 tile][n8 tile][fragment register]: first the branch's int32 sums, then fp32 outputs
-      int acc[2][2][4][4];
+      float acc[2][2][4][4];                            // [half][m16 tile][n8 tile][fragment register]
+      uint32_t w0[2][8];                                // cgi == 0: the branch columns that the scale factors alias
+      ok = mbar_wait_idle(bar(B_TFULL), tc & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
+      if (!ok) break;
+      tc_fence_after();
+      // hand-over: every load is issued before the one wait; the main accumulator lands in the registers it stays in
 #pragma unroll
       for (int h = 0; h < 2; ++h)
+        if (h < width) {
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-          for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) acc[h][mt][nt][i] = 0;
-      // branch part, while the tensor core works on the tile: U = tq L2q (exact int32).  All fragment loads of a step
-      // are issued before the first MMA so that they share one trip to the L2.
-      for (int kk = 0; kk < p.branch_steps; ++kk) {
-        uint32_t a[2][4], b[2][4][2];
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-          const uint8_t* ap = p.tq + (size_t)(m0 + rl + 16 * mt) * LQ_RCONT + kk * 32 + 4 * t;
-          a[mt][0] = __ldg(reinterpret_cast<const uint32_t*>(ap));
-          a[mt][1] = __ldg(reinterpret_cast<const uint32_t*>(ap + 8 * LQ_RCONT));
-          a[mt][2] = __ldg(reinterpret_cast<const uint32_t*>(ap + 16));
-          a[mt][3] = __ldg(reinterpret_cast<const uint32_t*>(ap + 8 * LQ_RCONT + 16));
+          for (int mt = 0; mt < 2; ++mt)
+            tmem_ld_16x256b_x4(tlane + ((uint32_t)(16 * mt) << 16) + h * UNIT, reinterpret_cast<uint32_t(&)[16]>(acc[h][mt]));
         }
+      if (has_branch && cgi == 0) {
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-          for (int nt = 0; nt < 4; ++nt) {
-            const int hh = h < width ? h : 0;           // a narrow tile reads the same (valid) rows twice and ignores them
-            const uint8_t* bp = p.L2c + (size_t)(n0 + hh * UNIT + cl + nt * 8 + g) * LQ_RCONT + kk * 32 + 4 * t;
-            b[h][nt][0] = __ldg(reinterpret_cast<const uint32_t*>(bp));
-            b[h][nt][1] = __ldg(reinterpret_cast<const uint32_t*>(bp + 16));
-          }
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-          if (h < width) {
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-              for (int mt = 0; mt < 2; ++mt) mma_s8_16x8x32(acc[h][mt][nt], a[mt], b[h][nt][0], b[h][nt][1]);
-          }
+        for (int mt = 0; mt < 2; ++mt) tmem_ld_16x256b_x2(tlane + ((uint32_t)(16 * mt) << 16) + TM_BR, w0[mt]);
       }
-      // y = U sT sL2 + bias  (|U| < 2^22: converted exactly with the 1.5 * 2^23 trick)
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_TEMPTY));
+      // y = main + U sT sL2 + bias, under the next tile's main loop (the tensor core has already applied the block
+      // scales to main)
       ok = mbar_wait(bar(B_RFULL + rb), (tc >> 1) & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
       if (!ok) break;
       {
         const float* sc = sc_ptr + rb * SC_FLOATS;
-        float stv[2][2];
+        const float* sc_l2 = sc + LQ_BM + cl + 2 * t;
+        const float* sc_b = sc + LQ_BM + 2 * UNIT + cl + 2 * t;
+        if (has_branch && cgi == 0) {                  // the early-read columns first: their registers are free again
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-          stv[mt][0] = sc[rl + 16 * mt];
-          stv[mt][1] = sc[rl + 16 * mt + 8];
+          for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt)
+              combine_fragment(acc[0][mt][nt], &w0[mt][4 * nt], true, sc[rl + 16 * mt], sc[rl + 16 * mt + 8],
+                               *reinterpret_cast<const float2*>(sc_l2 + nt * 8), *reinterpret_cast<const float2*>(sc_b + nt * 8));
         }
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           if (h < width) {
 #pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-              const int c = h * UNIT + cl + nt * 8 + 2 * t;
-              const float2 sl = *reinterpret_cast<const float2*>(sc + LQ_BM + c);
-              const float2 bv = *reinterpret_cast<const float2*>(sc + LQ_BM + 2 * UNIT + c);
+            for (int mt = 0; mt < 2; ++mt) {
+              uint32_t w[16];
+              const bool early = has_branch && cgi == 0 && h == 0;       // fragments 0 and 1 are done already
+              if (has_branch) {
+                const uint32_t ta = tlane + ((uint32_t)(16 * mt) << 16) + TM_BR + h * UNIT;
+                if (early) tmem_ld_16x256b_x2(ta + TM_SF_ALIASED, reinterpret_cast<uint32_t(&)[8]>(w[8]));
+                else tmem_ld_16x256b_x4(ta, w);
+                tmem_ld_wait();
+              }
+              const float st_lo = sc[rl + 16 * mt], st_hi = sc[rl + 16 * mt + 8];
 #pragma unroll
-              for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  const float uf = __int_as_float(acc[h][mt][nt][i] + 0x4B400000) - 12582912.0f;
-                  const float y = fmaf(uf, stv[mt][i >> 1] * ((i & 1) ? sl.y : sl.x), (i & 1) ? bv.y : bv.x);
-                  acc[h][mt][nt][i] = __float_as_int(y);
-                }
+              for (int nt = 0; nt < 4; ++nt) {
+                if (nt < 2 && early) continue;
+                combine_fragment(acc[h][mt][nt], &w[4 * nt], has_branch, st_lo, st_hi,
+                                 *reinterpret_cast<const float2*>(sc_l2 + h * UNIT + nt * 8),
+                                 *reinterpret_cast<const float2*>(sc_b + h * UNIT + nt * 8));
+              }
             }
-          }
-        }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_REMPTY + rb));
-      // main part: the tensor core has already applied the block scales
-      ok = mbar_wait(bar(B_TFULL), tc & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
-      if (!ok) break;
-      tc_fence_after();
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        if (h < width) {
-#pragma unroll
-          for (int mt = 0; mt < 2; ++mt) {
-            uint32_t v[16];
-            tmem_ld_16x256b_x4(tlane + ((uint32_t)(16 * mt) << 16) + h * UNIT, v);
-            tmem_ld_wait();
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-              for (int i = 0; i < 4; ++i)
-                acc[h][mt][nt][i] = __float_as_int(__int_as_float(acc[h][mt][nt][i]) + __uint_as_float(v[4 * nt + i]));
           }
         }
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(B_TEMPTY));
+      if (lane == 0) { mbar_arrive(bar(B_BEMPTY)); mbar_arrive(bar(B_REMPTY + rb)); }
       // epilogue
-      const int row_w = m0 + quad * 32;                 // first row of this warp's part
+      const int row_w = m0 + quad * 32;                 // first row of this group's part
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         if (h < width) {
-          const int col_w = n0 + h * UNIT + cl;         // first column of this warp's part of the half
           if (p.out_f32) {
             float* Y = reinterpret_cast<float*>(p.Y);
 #pragma unroll
@@ -517,51 +536,40 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               const int r_lo = row_w + g + 16 * mt, r_hi = r_lo + 8;
 #pragma unroll
               for (int nt = 0; nt < 4; ++nt) {
-                const int c = col_w + nt * 8 + 2 * t;
+                const int c = n0 + h * UNIT + cl + nt * 8 + 2 * t;
                 if (c < p.N) {
-                  if (r_lo < p.M)
-                    *reinterpret_cast<float2*>(Y + (size_t)r_lo * p.N + c) =
-                        make_float2(__int_as_float(acc[h][mt][nt][0]), __int_as_float(acc[h][mt][nt][1]));
-                  if (r_hi < p.M)
-                    *reinterpret_cast<float2*>(Y + (size_t)r_hi * p.N + c) =
-                        make_float2(__int_as_float(acc[h][mt][nt][2]), __int_as_float(acc[h][mt][nt][3]));
+                  if (r_lo < p.M) *reinterpret_cast<float2*>(Y + (size_t)r_lo * p.N + c) = make_float2(acc[h][mt][nt][0], acc[h][mt][nt][1]);
+                  if (r_hi < p.M) *reinterpret_cast<float2*>(Y + (size_t)r_hi * p.N + c) = make_float2(acc[h][mt][nt][2], acc[h][mt][nt][3]);
                 }
               }
             }
           } else {
-            // The half's buffer was last read by the store of the previous tile: at most this tile's other half may
-            // still be in flight.
-            if (lane == 0) { if (h == 0) bulk_wait_read<0>(); else bulk_wait_read<1>(); }
-            __syncwarp();
-            uint8_t* buf = out_w + h * OUT_UNIT_BYTES;
+            __half* Y = reinterpret_cast<__half*>(p.Y);
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt) {
               // pack to fp16, then exchange inside the quad: lane t ends up with columns 8 t .. 8 t + 7 of both rows
               uint32_t lo[4], hi[4];
 #pragma unroll
               for (int nt = 0; nt < 4; ++nt) {
-                const __half2 l2 = __floats2half2_rn(__int_as_float(acc[h][mt][nt][0]), __int_as_float(acc[h][mt][nt][1]));
-                const __half2 h2 = __floats2half2_rn(__int_as_float(acc[h][mt][nt][2]), __int_as_float(acc[h][mt][nt][3]));
+                const __half2 l2 = __floats2half2_rn(acc[h][mt][nt][0], acc[h][mt][nt][1]);
+                const __half2 h2 = __floats2half2_rn(acc[h][mt][nt][2], acc[h][mt][nt][3]);
                 lo[nt] = *reinterpret_cast<const uint32_t*>(&l2);
                 hi[nt] = *reinterpret_cast<const uint32_t*>(&h2);
               }
               quad_transpose(lo, t);
               quad_transpose(hi, t);
-              *reinterpret_cast<uint4*>(buf + (16 * mt + g) * 64 + 16 * t) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-              *reinterpret_cast<uint4*>(buf + (16 * mt + g + 8) * 64 + 16 * t) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            }
-            fence_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-              if (col_w < p.N && row_w < p.M) tma_store_2d(&tmY, col_w, row_w, out_w_s + h * OUT_UNIT_BYTES);
-              bulk_commit();
+              // each lane owns 16 contiguous bytes of a row: a store instruction writes whole 32-byte sectors
+              const int c = n0 + h * UNIT + cl + 8 * t;
+              const int r_lo = row_w + g + 16 * mt, r_hi = r_lo + 8;
+              if (c < p.N) {
+                if (r_lo < p.M) *reinterpret_cast<uint4*>(Y + (size_t)r_lo * p.N + c) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                if (r_hi < p.M) *reinterpret_cast<uint4*>(Y + (size_t)r_hi * p.N + c) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+              }
             }
           }
         }
       }
-      u += width;
     }
-    if (lane == 0) bulk_wait_all();                      // the staged rows must stay until the last store has read them
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -592,22 +600,16 @@ lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_
   p.branch_steps = L->r == 0 ? 0 : lq_ceil_div(L->r, 32);
   p.tiles_m = lq_ceil_div(A->M, LQ_BM);
   p.units_n = L->Npad / UNIT;
-  p.sfa = A->d_sfa; p.sfb = L->d_sfb; p.tq = A->d_tq; p.L2c = L->d_L2c; p.sT = A->d_sT; p.sL2 = L->d_sL2; p.bias = L->d_bias;
+  p.sfa = A->d_sfa; p.sfb = L->d_sfb; p.sT = A->d_sT; p.sL2 = L->d_sL2; p.bias = L->d_bias;
   p.Y = Y; p.out_f32 = dt == LQ_OUT_F32 ? 1 : 0;
   p.status = lq_device_status_ptr(A->device);
   if (!p.status) return LQ_ERR_CUDA;
   int sms = 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, A->device) != cudaSuccess) return LQ_ERR_CUDA;
   int ctas = g_lq_gemm_ctas > 0 ? g_lq_gemm_ctas : sms;
-  const long long units = (long long)p.tiles_m * p.units_n;
-  if (ctas > units) ctas = (int)units;
-  // fp16 rows leave through TMA stores: a tensor map over the caller's Y (32 x 32 boxes, clipped at M and N); the fp32
-  // variant stores from registers and does not use it
-  CUtensorMap tmY = A->tmA;
-  if (dt == LQ_OUT_F16) {
-    const lq_status ts = lq_make_tmap_out_f16(&tmY, Y, (uint64_t)A->M, (uint64_t)L->N, 32, 32);
-    if (ts != LQ_OK) return ts;
-  }
-  lq_gemm_mx_kernel<<<ctas, GEMM_THREADS, SMEM_BYTES, st>>>(A->tmA, L->tmB, L->tmB2, tmY, p);
+  const long long tiles = (long long)p.tiles_m * ((p.units_n + 1) / 2);
+  if (ctas > tiles) ctas = (int)tiles;
+  p.by_units = (p.units_n & 1) && tiles < 4ll * ctas;
+  lq_gemm_mx_kernel<<<ctas, GEMM_THREADS, SMEM_BYTES, st>>>(A->tmA, L->tmB, L->tmB2, A->tmT, L->tmL2, p);
   return lq_note_cuda(cudaGetLastError()) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
 }

@@ -111,8 +111,6 @@ lq_status lq_launch_gemm(const lq_layer* L, const lq_act* A, void* Y, lq_out_dty
 lq_status lq_gemm_prepare(int device);
 lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_dtype dt, cudaStream_t st);
 lq_status lq_gemm_mx_prepare(int device);
-// tensor map over an fp16 output [rows][cols] in the caller's memory (16-byte aligned, cols % 8 == 0), no swizzle
-lq_status lq_make_tmap_out_f16(CUtensorMap* tm, void* base, uint64_t rows, uint64_t cols, uint32_t box_cols, uint32_t box_rows);
 lq_status lq_launch_wait_probe(int device, cudaStream_t st);   // bounded-wait self-test kernel   // sets the kernel's shared-memory attribute once per device
 
 // byte an MMA operand carries for a 4-bit code q in [-7, 7]
