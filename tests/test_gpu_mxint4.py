@@ -94,3 +94,33 @@ def test_mx_sana_shape_sampled_rows():
     assert np.array_equal(ex["tq"][rows], ref["tq"])
     assert np.isfinite(Y.astype(np.float32)).all()
     assert rel_fro(Y[rows], ref["Y"]) <= TOL_F16
+
+
+@pytest.mark.parametrize("spec", I.PIXART_LAYERS, ids=lambda s: s.name)
+def test_mx_config1_pixart_block_linears(spec):
+    """The benchmark's launch configuration (M = 8192, r = 32, W8A8 branch) with the MXINT4 main branch: the seeded
+    config-1 activations, 160 sampled rows against the oracle.  qkv and fc1 share the work by tiles, attn-out and fc2
+    (nine 128-column units per row block, few tiles per CTA) by units."""
+    rng = np.random.default_rng(4)
+    wl = I.workload(1)
+    X, _, _ = I.layer_inputs(wl, spec, M=8192)
+    layer = _mx_layer(rng, spec.K, spec.N, 32, "w8a8")
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, 8063, 8064, 8190, 8191], rng.choice(8192, 152, replace=False)]))
+    ref = O.forward(X[rows], layer)
+    Y, ex = gpu_forward(layer, X, out_f32=False)
+    assert np.array_equal(ex["qx"][rows], ref["qx"])
+    assert np.array_equal(ex["sx"][rows], ref["ex"])
+    assert np.array_equal(ex["tq"][rows], ref["tq"])
+    assert np.isfinite(Y.astype(np.float32)).all()
+    assert (np.abs(Y.astype(np.float32)).sum(axis=1) > 0).all()
+    assert rel_fro(Y[rows], ref["Y"]) <= TOL_F16
+
+
+@pytest.mark.parametrize("r,branch", [(128, "w8a8"), (16, "w6a6"), (0, "none")])
+def test_mx_odd_unit_count_ragged_rows_and_ranks(r, branch):
+    """N = 1152 (nine units: one 128-wide tile per row block), ragged M, ranks up to the maximum (four branch MMAs)."""
+    rng = np.random.default_rng(5)
+    M, K, N = 1000, 1152, 1152
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    X[:, rng.integers(0, K, 8)] *= 20
+    _check(_mx_layer(rng, K, N, r, branch), X)
