@@ -13,7 +13,8 @@
  *   group = 32  MXINT4: the same codes, one power-of-two scale 2^e per block of 32 along K,
  *               e the smallest integer with 7 * 2^e >= max|v| of the block (the paper does not
  *               spell the rule out; this one never clips); the scales are applied by the tensor
- *               core itself (block-scaled MMA).  Integer branches only.
+ *               core itself (block-scaled MMA).  Every branch format; with the fp16 reference branch the
+ *               tensor core also adds the branch product onto the same accumulator.
  *
  * Every function returns an lq_status; nothing throws, aborts or prints.  "host" / "device"
  * in a parameter comment says which address space the pointer lives in.  Device pointers and
@@ -84,7 +85,7 @@ lq_status lq_config_default(lq_config* cfg, int32_t K, int32_t N, int32_t rank, 
  *   bias_f16_host  [N] half bits or NULL, host
  *   out            receives a new layer (host copy only; see lq_layer_to_device)
  *   objective_trace[steps + 1] doubles or NULL, host: objective at every iterate, [0] = init
- * Errors: INVALID_ARG (null / bad shape), UNSUPPORTED (rot_steps != 0, group not 64 or 32, MXINT4 with the fp16 branch, ...),
+ * Errors: INVALID_ARG (null / bad shape), UNSUPPORTED (rot_steps != 0, group not 64 or 32, ...),
  * NUMERIC (non-finite W), ALLOC. */
 lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W_f16_host,
                        const uint16_t* bias_f16_host, lq_layer** out, double* objective_trace);

@@ -79,7 +79,6 @@ static lq_status check_config(const lq_config* c) {
   if (c->K <= 0 || c->N <= 0 || c->rank < 0) return LQ_ERR_INVALID_ARG;
   if (c->branch < LQ_BRANCH_NONE || c->branch > LQ_BRANCH_W4A8) return LQ_ERR_INVALID_ARG;
   if (c->group != LQ_GROUP && c->group != LQ_MX_BLOCK) return LQ_ERR_UNSUPPORTED;
-  if (c->group == LQ_MX_BLOCK && c->branch == LQ_BRANCH_W16A16) return LQ_ERR_UNSUPPORTED;
   if (c->K > LQ_MAX_K || (c->K % 8) != 0) return LQ_ERR_UNSUPPORTED;
   if ((c->N % 8) != 0) return LQ_ERR_UNSUPPORTED;
   if (c->rank > LQ_MAX_RANK) return LQ_ERR_UNSUPPORTED;

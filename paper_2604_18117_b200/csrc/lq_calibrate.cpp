@@ -303,7 +303,6 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
   if (cfg->K <= 0 || cfg->N <= 0 || cfg->rank < 0 || cfg->steps < 0) return LQ_ERR_INVALID_ARG;
   if (cfg->branch < LQ_BRANCH_NONE || cfg->branch > LQ_BRANCH_W4A8) return LQ_ERR_INVALID_ARG;
   if ((cfg->group != LQ_GROUP && cfg->group != LQ_MX_BLOCK) || cfg->rot_steps != 0) return LQ_ERR_UNSUPPORTED;
-  if (cfg->group == LQ_MX_BLOCK && cfg->branch == LQ_BRANCH_W16A16) return LQ_ERR_UNSUPPORTED;
   if (cfg->K > LQ_MAX_K || (cfg->K % 8) || (cfg->N % 8) || cfg->rank > LQ_MAX_RANK) return LQ_ERR_UNSUPPORTED;
   if (cfg->branch == LQ_BRANCH_W16A16 && cfg->rank > 64) return LQ_ERR_UNSUPPORTED;
   if (cfg->rank > std::min(cfg->K, cfg->N)) return LQ_ERR_INVALID_ARG;

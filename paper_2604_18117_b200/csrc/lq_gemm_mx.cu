@@ -62,6 +62,7 @@ struct MxParams {
   int M, N, Mpad, Npad;
   int k_stages;           // Kpad / 128
   int branch_steps;       // 0: no branch; else MMAs of the branch stage (32 bytes of r each)
+  int branch_f16;         // the branch operands are halves (W16A16 reference branch): no scales, summed by the tensor core
   int tiles_m, units_n;
   int by_units;           // how the CTAs share the work: 0 whole tiles, 1 128-column units
   const uint8_t* sfa;     // [Mpad/128][k_stages][512]
@@ -292,6 +293,9 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // provably warp-uniform
   const int lane = threadIdx.x & 31;
   const bool has_branch = p.branch_steps > 0;
+  // An fp16 branch has no scales: its product is accumulated onto the main accumulator by the tensor core and the drain
+  // sees no branch at all.  An integer branch needs its fp32 scales applied per element: second accumulator.
+  const bool branch_acc = has_branch && !p.branch_f16;
   // Each CTA takes a contiguous, equal share of the work and walks it as 256-wide tiles (128-wide where a row block or
   // the share ends).  A 128-wide tile costs nearly as much as a 256-wide one (a stage's time is set by its hand-shakes
   // and instruction count, not its MMA width).  by_units = 0 shares whole tiles - row blocks cut into 256-wide tiles
@@ -427,15 +431,19 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int st = it % NSTAGE;
         ok = mbar_wait_warp(bar(B_FULL + st), (it / NSTAGE) & 1, abort_flag, p.status, LQ_STAGE_MMA);
         if (!ok) break;
-        // the drain has read the previous tile's branch accumulator (long ago: it does that under this tile's main loop)
-        ok = mbar_wait_warp(bar(B_BEMPTY), (tc & 1) ^ 1, abort_flag, p.status, LQ_STAGE_MMA);
-        if (!ok) break;
+        if (branch_acc) {
+          // the drain has read the previous tile's branch accumulator (long ago: it does that under this tile's main loop)
+          ok = mbar_wait_warp(bar(B_BEMPTY), (tc & 1) ^ 1, abort_flag, p.status, LQ_STAGE_MMA);
+          if (!ok) break;
+        }
         tc_fence_after();
         const uint32_t a_addr = sm_stage + st * STAGE_BYTES, b_addr = a_addr + STAGE_A_BYTES;
         const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
         if (elect_one()) {
-          for (int j = 0; j < p.branch_steps; ++j)
-            tc_mma<0>(tmem_base + TM_BR, adesc + 2 * j, bdesc + 2 * j, IDESC_I8 | idesc_shape(ncols), (uint32_t)j);
+          for (int j = 0; j < p.branch_steps; ++j) {
+            if (branch_acc) tc_mma<0>(tmem_base + TM_BR, adesc + 2 * j, bdesc + 2 * j, IDESC_I8 | idesc_shape(ncols), (uint32_t)j);
+            else tc_mma<2>(tmem_base, adesc + 2 * j, bdesc + 2 * j, IDESC_F16 | idesc_shape(ncols), 1u);   // 16 halves each
+          }
           tc_commit(bar(B_EMPTY + st));
         }
         __syncwarp();
@@ -472,7 +480,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           for (int mt = 0; mt < 2; ++mt)
             tmem_ld_16x256b_x4(tlane + ((uint32_t)(16 * mt) << 16) + h * UNIT, reinterpret_cast<uint32_t(&)[16]>(acc[h][mt]));
         }
-      if (has_branch && cgi == 0) {
+      if (branch_acc && cgi == 0) {
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) tmem_ld_16x256b_x2(tlane + ((uint32_t)(16 * mt) << 16) + TM_BR, w0[mt]);
       }
@@ -488,7 +496,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const float* sc = sc_ptr + rb * SC_FLOATS;
         const float* sc_l2 = sc + LQ_BM + cl + 2 * t;
         const float* sc_b = sc + LQ_BM + 2 * UNIT + cl + 2 * t;
-        if (has_branch && cgi == 0) {                  // the early-read columns first: their registers are free again
+        if (branch_acc && cgi == 0) {                  // the early-read columns first: their registers are free again
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
@@ -502,8 +510,8 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt) {
               uint32_t w[16];
-              const bool early = has_branch && cgi == 0 && h == 0;       // fragments 0 and 1 are done already
-              if (has_branch) {
+              const bool early = branch_acc && cgi == 0 && h == 0;       // fragments 0 and 1 are done already
+              if (branch_acc) {
                 const uint32_t ta = tlane + ((uint32_t)(16 * mt) << 16) + TM_BR + h * UNIT;
                 if (early) tmem_ld_16x256b_x2(ta + TM_SF_ALIASED, reinterpret_cast<uint32_t(&)[8]>(w[8]));
                 else tmem_ld_16x256b_x4(ta, w);
@@ -513,7 +521,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
               for (int nt = 0; nt < 4; ++nt) {
                 if (nt < 2 && early) continue;
-                combine_fragment(acc[h][mt][nt], &w[4 * nt], has_branch, st_lo, st_hi,
+                combine_fragment(acc[h][mt][nt], &w[4 * nt], branch_acc, st_lo, st_hi,
                                  *reinterpret_cast<const float2*>(sc_l2 + h * UNIT + nt * 8),
                                  *reinterpret_cast<const float2*>(sc_b + h * UNIT + nt * 8));
               }
@@ -593,11 +601,12 @@ lq_status lq_gemm_mx_prepare(int device) {
 
 lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_dtype dt, cudaStream_t st) {
   if (cudaSetDevice(A->device) != cudaSuccess) return LQ_ERR_CUDA;
-  if (!L->mx || !A->mx || L->f16_branch) return LQ_ERR_UNSUPPORTED;
+  if (!L->mx || !A->mx) return LQ_ERR_UNSUPPORTED;
   MxParams p;
   p.M = A->M; p.N = L->N; p.Mpad = A->Mpad; p.Npad = L->Npad;
   p.k_stages = L->Kpad / LQ_KSTAGE;
-  p.branch_steps = L->r == 0 ? 0 : lq_ceil_div(L->r, 32);
+  p.branch_f16 = L->f16_branch ? 1 : 0;
+  p.branch_steps = L->r == 0 ? 0 : lq_ceil_div(L->r, L->f16_branch ? 16 : 32);
   p.tiles_m = lq_ceil_div(A->M, LQ_BM);
   p.units_n = L->Npad / UNIT;
   p.sfa = A->d_sfa; p.sfb = L->d_sfb; p.sT = A->d_sT; p.sL2 = L->d_sL2; p.bias = L->d_bias;

@@ -20,7 +20,10 @@ def _mx_layer(rng, K, N, r, branch, wscale=0.02, bias=True):
     W = rng.standard_normal((K, N)) * wscale
     W[:: max(1, K // 7), :] *= 10                                       # outlier input channels: exponents vary per block
     layer["Wq"], layer["ew"] = O.q_weight_main_mx(W)
-    if r > 0:
+    if r > 0 and branch == "w16a16":
+        layer["L1h"], _ = O.q_factor(rng.standard_normal((K, r)) * 0.05, None)
+        layer["L2h"], _ = O.q_factor(rng.standard_normal((r, N)) * 0.05, None)
+    elif r > 0:
         bw, _ = O.BRANCH_BITS[branch]
         layer["L1q"], layer["sL1"] = O.q_factor(rng.standard_normal((K, r)) * 0.05, bw)
         layer["L2q"], layer["sL2"] = O.q_factor(rng.standard_normal((r, N)) * 0.05, bw)
@@ -61,7 +64,7 @@ def test_mx_integer_exact_product_with_varied_exponents():
     assert np.abs(Y - ref["Y"]).max() <= 1e-5 * np.abs(ref["Y"]).max()
 
 
-@pytest.mark.parametrize("branch", ["none", "w8a8", "w6a6", "w4a8"])
+@pytest.mark.parametrize("branch", ["none", "w8a8", "w6a6", "w4a8", "w16a16"])
 def test_mx_small_shapes_all_branches(branch):
     rng = np.random.default_rng(1)
     M, K, N, r = 200, 328, 200, 0 if branch == "none" else 32          # ragged M, N; K = 10.25 blocks
@@ -116,7 +119,7 @@ def test_mx_config1_pixart_block_linears(spec):
     assert rel_fro(Y[rows], ref["Y"]) <= TOL_F16
 
 
-@pytest.mark.parametrize("r,branch", [(128, "w8a8"), (16, "w6a6"), (0, "none")])
+@pytest.mark.parametrize("r,branch", [(128, "w8a8"), (16, "w6a6"), (0, "none"), (64, "w16a16")])
 def test_mx_odd_unit_count_ragged_rows_and_ranks(r, branch):
     """N = 1152 (nine units: one 128-wide tile per row block), ragged M, ranks up to the maximum (four branch MMAs)."""
     rng = np.random.default_rng(5)
