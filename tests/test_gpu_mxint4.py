@@ -127,3 +127,38 @@ def test_mx_odd_unit_count_ragged_rows_and_ranks(r, branch):
     X = rng.standard_normal((M, K)).astype(np.float16)
     X[:, rng.integers(0, K, 8)] *= 20
     _check(_mx_layer(rng, K, N, r, branch), X)
+
+
+def test_mx_host_entry_point_pipelines_row_chunks():
+    """lq_linear_forward_host with an MXINT4 layer: the row-chunk views of the activation record (codes, scale bytes in
+    chunks of 128 rows, branch codes) must give the same bits as one call over all rows."""
+    import torch
+    from paper_2604_18117_b200 import binding as B
+    from tests.helpers import import_oracle_layer
+    rng = np.random.default_rng(6)
+    M, K, N, r = 1300, 1152, 392, 32                       # four chunks, the last one ragged; N not a multiple of 128
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    layer = _mx_layer(rng, K, N, r, "w8a8")
+    ref = O.forward(X, layer)
+    h, cfg = import_oracle_layer(layer)
+    B.lq_layer_to_device(h, 0)
+    act = B.lq_act_create(h, M, 0)
+    try:
+        st = torch.cuda.current_stream().cuda_stream
+        Xp = torch.from_numpy(X).pin_memory()
+        Yp = torch.full((M, N), float("nan"), dtype=torch.float16).pin_memory()
+        B.lq_linear_forward_host(h, act, Xp.data_ptr(), M, Yp.data_ptr(), B.OUT_F16, st)
+        assert B.lq_get_device_status(0)[0] == 0
+        Yh = Yp.numpy().copy()
+        ex = B.lq_act_export(act, M, cfg, st)
+        assert_codes_equal(ex, ref, "w8a8", with_qb=False)
+        Xd = torch.from_numpy(X).cuda()
+        Yd = torch.full((M, N), float("nan"), dtype=torch.float16, device="cuda")
+        B.lq_quantize_act(h, Xd.data_ptr(), M, act, st)
+        B.lq_linear_forward(h, act, Yd.data_ptr(), B.OUT_F16, st)
+        torch.cuda.synchronize()
+        assert np.array_equal(Yh, Yd.cpu().numpy())
+        assert rel_fro(Yh, ref["Y"]) <= TOL_F16
+    finally:
+        B.lq_act_free(act)
+        B.lq_layer_free(h)
