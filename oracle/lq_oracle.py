@@ -292,11 +292,59 @@ def gradients(W, L, R, main: str = "sint4"):
     return float(np.mean(E * E)), c * (E @ R.T), c * (L.T @ E)
 
 
+def q2_dequant(F, bits):
+    """Q2(F) as real numbers (per-column integer quantizer; bits None = fp16 rounding)."""
+    q, s = q_factor(F, bits)
+    return deq_factor(q, s)
+
+
+def rotation_loss(L, R, Om, bits):
+    """Loss of the rotation-aware step (Eq. "loss-rotation-aware"), each term a mean of squares:
+    mean((Q2(L Om) - L Om)^2) + mean((Q2(Om^T R) - Om^T R)^2).  Returns (loss, E1, E2)."""
+    A, B = L @ Om, Om.T @ R
+    E1, E2 = q2_dequant(A, bits) - A, q2_dequant(B, bits) - B
+    return float(np.mean(E1 * E1) + np.mean(E2 * E2)), E1, E2
+
+
+def rotation_gradient(L, R, Om, bits):
+    """(loss, dLoss/dOm) with Q2's derivative taken as zero, as for Q1 in Appendix B.2:
+    d/dOm mean((Q - L Om)^2) = -2 L^T E1 / (K r),  d/dOm mean((Q' - Om^T R)^2) = -2 R E2^T / (r N)."""
+    loss, E1, E2 = rotation_loss(L, R, Om, bits)
+    G = -2.0 * (L.T @ E1) / E1.size - 2.0 * (R @ E2.T) / E2.size
+    return loss, G
+
+
+def optimize_rotation(L, R, bits, steps: int = 500, lr: float = 0.5):
+    """Rotation-aware step of Section 3.3: an orthogonal Om [r, r] that lowers the Q2 error of L Om and Om^T R while
+    (L Om)(Om^T R) = L R.  The paper names Cayley SGD as its inspiration and gives the learning rate and the step count;
+    the update taken here is the plain Cayley retraction of that method without momentum: with the skew-symmetric
+    S = G Om^T - Om G^T,  Om <- (I + lr/2 S)^-1 (I - lr/2 S) Om, which keeps Om orthogonal to rounding.  Starts at the
+    identity and returns the best iterate seen, with the trace [steps+1] of the loss."""
+    r = L.shape[1]
+    Om = np.eye(r)
+    I = np.eye(r)
+    trace = np.zeros(steps + 1)
+    best = (np.inf, Om)
+    for t in range(steps + 1):
+        loss, G = rotation_gradient(L, R, Om, bits)
+        trace[t] = loss
+        if loss < best[0]:
+            best = (loss, Om.copy())
+        if t == steps:
+            break
+        S = G @ Om.T - Om @ G.T
+        Om = np.linalg.solve(I + 0.5 * lr * S, (I - 0.5 * lr * S) @ Om)
+    return best[1], trace
+
+
 def calibrate(W16, rank: int, branch: str = "w8a8", steps: int = 1000, lr: float = 1e-4,
-              beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, bias=None, main: str = "sint4"):
+              beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, bias=None, main: str = "sint4",
+              rot_steps: int = 0, rot_lr: float = 0.5):
     """Data-free calibration of one weight.  Returns (layer dict, trace [steps+1] of the
     objective at every iterate visited, iterate 0 = the SVD initialisation).  main selects Q1:
-    "sint4" (blocks of 64, fp16 scale) or "mxint4" (blocks of 32, power-of-two scale; Table 2)."""
+    "sint4" (blocks of 64, fp16 scale) or "mxint4" (blocks of 32, power-of-two scale; Table 2).
+    rot_steps > 0 adds the rotation-aware step before the factors are quantized (its loss trace is
+    stored as layer["rot_trace"])."""
     W = np.asarray(W16, dtype=np.float16).astype(np.float64)
     K, N = W.shape
     layer = {"branch": branch, "rank": int(rank), "K": K, "N": N, "main": main,
@@ -337,6 +385,10 @@ def calibrate(W16, rank: int, branch: str = "w8a8", steps: int = 1000, lr: float
     # Figure 1 sign: W ~ P + L1 L2 with L1 = -L*, L2 = R*
     L1, L2 = -best[1], best[2]
     bw, _ = BRANCH_BITS[branch]
+    if rot_steps > 0:                                     # Section 3.3: Q2(L1 Om), Q2(Om^T L2); the product is unchanged
+        Om, rot_trace = optimize_rotation(L1, L2, bw, rot_steps, rot_lr)
+        L1, L2 = L1 @ Om, Om.T @ L2
+        layer["rot_trace"] = rot_trace
     if branch == "w16a16":
         layer["L1h"], _ = q_factor(L1, None)
         layer["L2h"], _ = q_factor(L2, None)

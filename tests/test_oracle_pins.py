@@ -537,3 +537,78 @@ def test_forward_mxint4_exact_integer_case():
     assert not layer["ew"].any() and np.array_equal(layer["Wq"], Wi)
     out = O.forward(X, layer)
     assert not out["ex"].any() and np.array_equal(out["Y"], (X.astype(np.int64) @ Wi).astype(np.float64))
+
+
+# ----------------------------------------------------------------------------------------------
+# Rotation-aware step (Section 3.3, Eq. "rotation-optimization" / "loss-rotation-aware")
+def _rot_factors(seed, K=192, N=160, r=12):
+    rng = np.random.default_rng(seed)
+    L = rng.standard_normal((K, r)) * 0.1
+    R = rng.standard_normal((r, N)) * 0.1
+    L[:, 0] *= 6.0
+    R[2, :] *= 5.0
+    return L, R
+
+
+@pytest.mark.parametrize("bits,lr", [(8, 0.5), (4, 0.5), (6, 0.1)])
+def test_rotation_stays_orthogonal_and_keeps_the_product(bits, lr):
+    L, R = _rot_factors(0)
+    Om, trace = O.optimize_rotation(L, R, bits, steps=60, lr=lr)
+    r = L.shape[1]
+    assert np.abs(Om.T @ Om - np.eye(r)).max() < 1e-12 and abs(abs(np.linalg.det(Om)) - 1.0) < 1e-10
+    assert np.abs((L @ Om) @ (Om.T @ R) - L @ R).max() < 1e-12 * np.abs(L @ R).max() + 1e-14
+    # the returned rotation is the best iterate: its loss is the trace's minimum, not above the identity's
+    loss_best, _, _ = O.rotation_loss(L, R, Om, bits)
+    assert loss_best == trace.min() and trace.min() < trace[0]
+    assert np.all(np.diff(np.minimum.accumulate(trace)) <= 0)
+
+
+def test_rotation_loss_is_the_two_q2_errors_and_zero_steps_is_identity():
+    L, R = _rot_factors(1)
+    Om, trace = O.optimize_rotation(L, R, 8, steps=0, lr=0.5)
+    assert np.array_equal(Om, np.eye(L.shape[1])) and trace.shape == (1,)
+    q1, s1 = O.q_factor(L, 8); q2, s2 = O.q_factor(R, 8)
+    e1 = O.deq_factor(q1, s1) - L; e2 = O.deq_factor(q2, s2) - R
+    assert abs(trace[0] - (np.mean(e1 ** 2) + np.mean(e2 ** 2))) <= 1e-18 + 1e-12 * trace[0]
+
+
+def test_rotation_gradient_matches_finite_differences_with_q2_frozen():
+    """The derivative treats Q2's output as a constant: compare with central differences of that surrogate."""
+    L, R = _rot_factors(2, K=40, N=36, r=5)
+    rng = np.random.default_rng(3)
+    A = rng.standard_normal((5, 5)); Om0, _ = np.linalg.qr(A)
+    _, G = O.rotation_gradient(L, R, Om0, 6)
+    Qa, Qb = O.q2_dequant(L @ Om0, 6), O.q2_dequant(Om0.T @ R, 6)
+
+    def surrogate(Om):
+        return float(np.mean((Qa - L @ Om) ** 2) + np.mean((Qb - Om.T @ R) ** 2))
+
+    for _ in range(4):
+        D = rng.standard_normal((5, 5))
+        h = 1e-6
+        fd = (surrogate(Om0 + h * D) - surrogate(Om0 - h * D)) / (2 * h)
+        assert abs(fd - float(np.sum(G * D))) <= 1e-7 * max(1.0, abs(fd)) + 1e-12
+
+
+def test_rotation_leaves_exactly_representable_factors_alone():
+    """Factors already on Q2's grid have zero loss and zero gradient: the identity is kept."""
+    rng = np.random.default_rng(4)
+    L = rng.integers(-127, 128, size=(32, 4)).astype(np.float64); L[0, :] = 127
+    R = rng.integers(-127, 128, size=(4, 24)).astype(np.float64); R[0, :] = 127
+    Om, trace = O.optimize_rotation(L, R, 8, steps=5, lr=0.5)
+    assert trace[0] == 0.0 and np.array_equal(Om, np.eye(4))
+
+
+def test_calibrate_with_rotation_keeps_the_decomposition_consistent():
+    W = I.make_weight(0, 0, "rot", 128, 96, 2)
+    lay0, _ = O.calibrate(W, 8, "w4a8", steps=3)
+    lay1, _ = O.calibrate(W, 8, "w4a8", steps=3, rot_steps=40, rot_lr=0.5)
+    assert lay1["rot_trace"].shape == (41,) and lay1["rot_trace"].min() < lay1["rot_trace"][0]
+    W64 = W.astype(np.float64)
+    # stored residual codes are still Q1 of P = W - Q2(L1) Q2(L2)
+    D1 = O.deq_factor(lay1["L1q"], lay1["sL1"]) @ O.deq_factor(lay1["L2q"], lay1["sL2"])
+    Wq, sw = O.q_weight_main(W64 - D1)
+    assert np.array_equal(Wq, lay1["Wq"]) and np.array_equal(sw, lay1["sw"])
+    # both layers approximate the same product L1 L2: they differ by Q2's error only
+    D0 = O.deq_factor(lay0["L1q"], lay0["sL1"]) @ O.deq_factor(lay0["L2q"], lay0["sL2"])
+    assert np.linalg.norm(D1 - D0) <= 0.5 * np.linalg.norm(D0)
