@@ -63,8 +63,8 @@ typedef struct {
   int32_t steps;      /* Adam steps on (L, R); 1000 in Appendix A "Optimization"                  */
   float lr;           /* 1e-4 for integer formats (Appendix A)                                    */
   float beta1, beta2, eps; /* Adam moments / epsilon; the paper is silent: 0.9, 0.999, 1e-8       */
-  int32_t rot_steps;  /* rotation steps of Section 3.3; must be 0 (rotation is not built)         */
-  float rot_lr;
+  int32_t rot_steps;  /* steps of the rotation-aware optimisation of Section 3.3; 0 (default) = none,  */
+  float rot_lr;       /* 500 steps at 0.5 (0.1 for the mixed-precision study) in Appendix A           */
   uint64_t seed;      /* start vectors of the host SVD iteration                                  */
 } lq_config;
 
@@ -78,14 +78,16 @@ lq_status lq_config_default(lq_config* cfg, int32_t K, int32_t N, int32_t rank, 
 /* Data-free calibration of one weight, entirely on the host (Sections 3.2-3.3, Appendix A,
  * Appendix B.2): SVD initialisation L = -L0, R = R0; Adam on
  * mean((Q1(W + L R) - W - L R)^2) with the quantizer's derivative taken as zero; the best
- * iterate is kept; the factors are quantized with Q2; P = W - Q2(L1) Q2(L2) is quantized
+ * iterate is kept; with cfg->rot_steps > 0 an orthogonal rotation Om of the factors (L1 Om,
+ * Om^T L2: the same product) is then optimised to lower Q2's error (Cayley retraction steps,
+ * best iterate kept); the factors are quantized with Q2; P = W - Q2(L1) Q2(L2) is quantized
  * with Q1 (SINT4 or MXINT4 blocks along K per output column, as cfg->group says; MXINT4 weight
  * exponents are kept within [-24, 15] so that 2^e is a finite fp16 number).
  *   W_f16_host     [K][N] row-major IEEE half bits (the paper's d x n orientation), host
  *   bias_f16_host  [N] half bits or NULL, host
  *   out            receives a new layer (host copy only; see lq_layer_to_device)
  *   objective_trace[steps + 1] doubles or NULL, host: objective at every iterate, [0] = init
- * Errors: INVALID_ARG (null / bad shape), UNSUPPORTED (rot_steps != 0, group not 64 or 32, ...),
+ * Errors: INVALID_ARG (null / bad shape), UNSUPPORTED (group not 64 or 32, ...),
  * NUMERIC (non-finite W), ALLOC. */
 lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W_f16_host,
                        const uint16_t* bias_f16_host, lq_layer** out, double* objective_trace);

@@ -83,7 +83,7 @@ static lq_status check_config(const lq_config* c) {
   if ((c->N % 8) != 0) return LQ_ERR_UNSUPPORTED;
   if (c->rank > LQ_MAX_RANK) return LQ_ERR_UNSUPPORTED;
   if (c->branch == LQ_BRANCH_W16A16 && c->rank > 64) return LQ_ERR_UNSUPPORTED;
-  if (c->rot_steps != 0) return LQ_ERR_UNSUPPORTED;
+  if (c->rot_steps < 0) return LQ_ERR_INVALID_ARG;
   return LQ_OK;
 }
 

@@ -295,6 +295,138 @@ void matmul_LR(const std::vector<double>& L, const std::vector<double>& R, int K
   }
 }
 
+// deq(Q2(F)) - F for F [rows][cols] with one scale per column (bits > 0) or fp16 rounding (bits == 0); returns the sum of squares
+double q2_error(const std::vector<double>& F, int rows, int cols, int bits, std::vector<double>& E) {
+  double sum = 0;
+  if (bits == 0) {
+    for (size_t i = 0; i < F.size(); ++i) {
+      E[i] = (double)half_bits_to_float(float_to_half_bits((float)F[i])) - F[i];
+      sum += E[i] * E[i];
+    }
+    return sum;
+  }
+  const float qm = (float)((1 << (bits - 1)) - 1);
+  for (int c = 0; c < cols; ++c) {
+    float a = 0.f;
+    for (int t = 0; t < rows; ++t) a = fmaxf(a, fabsf((float)F[(size_t)t * cols + c]));
+    const float s = a == 0.f ? 1.0f : a / qm;
+    for (int t = 0; t < rows; ++t) {
+      const size_t i = (size_t)t * cols + c;
+      const float q = fminf(fmaxf(rintf((float)F[i] / s), -qm), qm);
+      E[i] = (double)q * (double)s - F[i];
+      sum += E[i] * E[i];
+    }
+  }
+  return sum;
+}
+
+// X <- A^-1 B for A [n][n], B [n][n] (Gaussian elimination with partial pivoting; A and B are overwritten)
+bool solve_square(std::vector<double>& A, std::vector<double>& B, int n) {
+  for (int c = 0; c < n; ++c) {
+    int piv = c;
+    for (int i = c + 1; i < n; ++i)
+      if (fabs(A[(size_t)i * n + c]) > fabs(A[(size_t)piv * n + c])) piv = i;
+    if (A[(size_t)piv * n + c] == 0.0) return false;
+    if (piv != c)
+      for (int j = 0; j < n; ++j) { std::swap(A[(size_t)c * n + j], A[(size_t)piv * n + j]); std::swap(B[(size_t)c * n + j], B[(size_t)piv * n + j]); }
+    const double inv = 1.0 / A[(size_t)c * n + c];
+    for (int i = c + 1; i < n; ++i) {
+      const double f = A[(size_t)i * n + c] * inv;
+      if (f == 0.0) continue;
+      for (int j = c; j < n; ++j) A[(size_t)i * n + j] -= f * A[(size_t)c * n + j];
+      for (int j = 0; j < n; ++j) B[(size_t)i * n + j] -= f * B[(size_t)c * n + j];
+    }
+  }
+  for (int c = n - 1; c >= 0; --c) {
+    const double inv = 1.0 / A[(size_t)c * n + c];
+    for (int j = 0; j < n; ++j) {
+      double v = B[(size_t)c * n + j];
+      for (int k = c + 1; k < n; ++k) v -= A[(size_t)c * n + k] * B[(size_t)k * n + j];
+      B[(size_t)c * n + j] = v * inv;
+    }
+  }
+  return true;
+}
+
+// Rotation-aware step (Section 3.3): an orthogonal Om [r][r] that lowers mean((Q2(L1 Om) - L1 Om)^2) +
+// mean((Q2(Om^T L2) - Om^T L2)^2); (L1 Om)(Om^T L2) = L1 L2.  Q2's derivative is taken as zero, as Q1's in Appendix B.2:
+// G = -2 L1^T E1 / (K r) - 2 L2 E2^T / (r N).  Update: the Cayley retraction of Cayley SGD (the paper's stated
+// inspiration) without momentum, S = G Om^T - Om G^T, Om <- (I + lr/2 S)^-1 (I - lr/2 S) Om; the best iterate is kept.
+// On return L1 and L2 hold the rotated factors.
+void rotate_factors(std::vector<double>& L1, std::vector<double>& L2, int K, int N, int r, int bits, int steps, double lr) {
+  std::vector<double> Om((size_t)r * r, 0.0), bestOm, A((size_t)K * r), B((size_t)r * N), E1(A.size()), E2(B.size());
+  std::vector<double> G((size_t)r * r), S((size_t)r * r), P((size_t)r * r), Q((size_t)r * r);
+  for (int i = 0; i < r; ++i) Om[(size_t)i * r + i] = 1.0;
+  bestOm = Om;
+  double best = INFINITY;
+  for (int t = 0; t <= steps; ++t) {
+#pragma omp parallel for schedule(static)
+    for (int k = 0; k < K; ++k)                                   // A = L1 Om
+      for (int j = 0; j < r; ++j) {
+        double v = 0;
+        for (int i = 0; i < r; ++i) v += L1[(size_t)k * r + i] * Om[(size_t)i * r + j];
+        A[(size_t)k * r + j] = v;
+      }
+#pragma omp parallel for schedule(static)
+    for (int j = 0; j < r; ++j) {                                 // B = Om^T L2
+      double* b = &B[(size_t)j * N];
+      for (int n = 0; n < N; ++n) b[n] = 0;
+      for (int i = 0; i < r; ++i) {
+        const double o = Om[(size_t)i * r + j];
+        const double* l2 = &L2[(size_t)i * N];
+        for (int n = 0; n < N; ++n) b[n] += o * l2[n];
+      }
+    }
+    const double loss = q2_error(A, K, r, bits, E1) / (double)A.size() + q2_error(B, r, N, bits, E2) / (double)B.size();
+    if (loss < best) { best = loss; bestOm = Om; }
+    if (t == steps) break;
+    const double c1 = -2.0 / (double)A.size(), c2 = -2.0 / (double)B.size();
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < r; ++i)
+      for (int j = 0; j < r; ++j) {
+        double a = 0, b = 0;
+        for (int k = 0; k < K; ++k) a += L1[(size_t)k * r + i] * E1[(size_t)k * r + j];          // (L1^T E1)[i][j]
+        const double* l2 = &L2[(size_t)i * N];
+        const double* e2 = &E2[(size_t)j * N];
+        for (int n = 0; n < N; ++n) b += l2[n] * e2[n];                                           // (L2 E2^T)[i][j]
+        G[(size_t)i * r + j] = c1 * a + c2 * b;
+      }
+    for (int i = 0; i < r; ++i)
+      for (int j = 0; j < r; ++j) {
+        double v = 0;
+        for (int k = 0; k < r; ++k) v += G[(size_t)i * r + k] * Om[(size_t)j * r + k] - Om[(size_t)i * r + k] * G[(size_t)j * r + k];
+        S[(size_t)i * r + j] = v;                                                                 // G Om^T - Om G^T
+      }
+    for (int i = 0; i < r; ++i)
+      for (int j = 0; j < r; ++j) {
+        const double h = 0.5 * lr * S[(size_t)i * r + j], id = i == j ? 1.0 : 0.0;
+        P[(size_t)i * r + j] = id + h;
+        double v = 0;
+        for (int k = 0; k < r; ++k) v += ((i == k ? 1.0 : 0.0) - 0.5 * lr * S[(size_t)i * r + k]) * Om[(size_t)k * r + j];
+        Q[(size_t)i * r + j] = v;                                                                 // (I - lr/2 S) Om
+      }
+    if (!solve_square(P, Q, r)) break;
+    Om = Q;
+  }
+  // L1 <- L1 bestOm, L2 <- bestOm^T L2
+  for (int k = 0; k < K; ++k)
+    for (int j = 0; j < r; ++j) {
+      double v = 0;
+      for (int i = 0; i < r; ++i) v += L1[(size_t)k * r + i] * bestOm[(size_t)i * r + j];
+      A[(size_t)k * r + j] = v;
+    }
+  for (int j = 0; j < r; ++j) {
+    double* b = &B[(size_t)j * N];
+    for (int n = 0; n < N; ++n) b[n] = 0;
+    for (int i = 0; i < r; ++i) {
+      const double o = bestOm[(size_t)i * r + j];
+      for (int n = 0; n < N; ++n) b[n] += o * L2[(size_t)i * N + n];
+    }
+  }
+  L1 = A;
+  L2 = B;
+}
+
 }  // namespace
 
 extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, const uint16_t* bias16, lq_layer** out,
@@ -302,7 +434,7 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
   if (!cfg || !W16 || !out) return LQ_ERR_INVALID_ARG;
   if (cfg->K <= 0 || cfg->N <= 0 || cfg->rank < 0 || cfg->steps < 0) return LQ_ERR_INVALID_ARG;
   if (cfg->branch < LQ_BRANCH_NONE || cfg->branch > LQ_BRANCH_W4A8) return LQ_ERR_INVALID_ARG;
-  if ((cfg->group != LQ_GROUP && cfg->group != LQ_MX_BLOCK) || cfg->rot_steps != 0) return LQ_ERR_UNSUPPORTED;
+  if ((cfg->group != LQ_GROUP && cfg->group != LQ_MX_BLOCK) || cfg->rot_steps < 0) return LQ_ERR_UNSUPPORTED;
   if (cfg->K > LQ_MAX_K || (cfg->K % 8) || (cfg->N % 8) || cfg->rank > LQ_MAX_RANK) return LQ_ERR_UNSUPPORTED;
   if (cfg->branch == LQ_BRANCH_W16A16 && cfg->rank > 64) return LQ_ERR_UNSUPPORTED;
   if (cfg->rank > std::min(cfg->K, cfg->N)) return LQ_ERR_INVALID_ARG;
@@ -391,6 +523,7 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
     // Figure 1's sign: W ~ P + L1 L2 with L1 = -L*, L2 = R*
     std::vector<double> L1 = bestL, L2 = bestR;
     for (double& v : L1) v = -v;
+    if (cfg->rot_steps > 0) rotate_factors(L1, L2, K, N, r, Lr->f16_branch ? 0 : lq_branch_wbits(cfg->branch), cfg->rot_steps, (double)cfg->rot_lr);
     std::vector<double> L1d(L1.size()), L2d(L2.size());
     if (Lr->f16_branch) {
       Lr->L1h.resize(L1.size()); Lr->L2h.resize(L2.size());

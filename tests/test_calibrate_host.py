@@ -120,3 +120,34 @@ def test_mxint4_main_calibration():
     W64 = W.astype(np.float64)
     assert np.linalg.norm(O.effective_weight(layer) - W64) < np.linalg.norm(O.q1_dequant(W64, "mxint4") - W64)
     B.lq_layer_free(h)
+
+
+def test_rotation_aware_step_on_the_host():
+    """cfg.rot_steps > 0 (Section 3.3): the rotated factors multiply to the same product, so the layer still
+    approximates W; the factors' quantization error - measured as the distance of Q2(L1) Q2(L2) to the fp16-branch product of
+    the same seed, which is almost unquantized - goes down; the residual codes are still Q1 of W - Q2(L1) Q2(L2)."""
+    W = I.make_weight(0, 0, "rot-host", 256, 192, 2)
+    W64 = W.astype(np.float64)
+
+    def run(branch, rot):
+        cfg = B.lq_config_default(256, 192, 16, branch); cfg.steps = 3; cfg.rot_steps = rot; cfg.rot_lr = 0.5
+        h, _ = B.lq_calibrate(cfg, W)
+        ex = B.lq_layer_export(h)
+        B.lq_layer_free(h)
+        return ex
+
+    ref = run("w16a16", 0)
+    D_ref = ref["L1"].astype(np.float64) @ ref["L2"].astype(np.float64)
+    ex0, ex1 = run("w4a8", 0), run("w4a8", 60)
+    D0 = O.deq_factor(ex0["L1"], ex0["sL1"]) @ O.deq_factor(ex0["L2"], ex0["sL2"])
+    D1 = O.deq_factor(ex1["L1"], ex1["sL1"]) @ O.deq_factor(ex1["L2"], ex1["sL2"])
+    e0, e1 = np.linalg.norm(D0 - D_ref), np.linalg.norm(D1 - D_ref)
+    assert e1 < e0, (e0, e1)
+    assert not np.array_equal(ex0["L1"], ex1["L1"])                      # the factors really were rotated
+    Wq, sw = O.q_weight_main(W64 - D1)
+    assert np.mean(Wq == B.unpack_nibbles(ex1["Wq_packed"])) > 0.9999 and np.mean(sw == ex1["sw"]) > 0.999
+    # same loss at the identity and a comparable gain as the oracle's statement of the step (trajectories are not bit-equal)
+    L1 = ref["L1"].astype(np.float64); L2 = ref["L2"].astype(np.float64)
+    _, tr = O.optimize_rotation(L1, L2, 4, steps=60, lr=0.5)
+    loss_host_0 = np.mean((O.q2_dequant(L1, 4) - L1) ** 2) + np.mean((O.q2_dequant(L2, 4) - L2) ** 2)
+    assert abs(loss_host_0 - tr[0]) <= 1e-12 * tr[0] and tr.min() < tr[0]
