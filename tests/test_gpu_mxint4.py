@@ -162,3 +162,28 @@ def test_mx_host_entry_point_pipelines_row_chunks():
     finally:
         B.lq_act_free(act)
         B.lq_layer_free(h)
+
+
+@pytest.mark.parametrize("ctas", [0, 7])
+@pytest.mark.parametrize("M,K,N,r,branch", [(1, 32, 8, 0, "none"), (129, 96, 136, 8, "w6a6"), (257, 8192, 128, 128, "w8a8"),
+                                            (5, 160, 264, 32, "w16a16"), (1000, 40, 2000, 24, "w8a8"), (333, 5600, 24, 48, "w16a16")])
+def test_mx_edge_shapes(ctas, M, K, N, r, branch):
+    """One row, one block of K, the maximum K and rank, N below one tile, K and N that end inside a tile - with one CTA per
+    SM and with seven CTAs (long runs of tiles per CTA)."""
+    from paper_2604_18117_b200 import binding as B
+    rng = np.random.default_rng(11)
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    X[:, rng.integers(0, K, 2)] *= 20
+    layer = _mx_layer(rng, K, N, r, branch)
+    ref = O.forward(X, layer)
+    B.lq_set_option("gemm_ctas", ctas)
+    try:
+        Y32, ex = gpu_forward(layer, X, out_f32=True)
+        Y16, _ = gpu_forward(layer, X, out_f32=False, export=False)
+    finally:
+        B.lq_set_option("gemm_ctas", 0)
+    assert_codes_equal(ex, ref, layer["branch"])
+    assert np.isfinite(Y32).all()
+    # fp16 reference branch: T is rounded to fp16 from an fp32 sum here and from an fp64 sum in the oracle
+    assert rel_fro(Y32, ref["Y"]) <= (3e-4 if branch == "w16a16" else TOL_F32)
+    assert rel_fro(Y16, ref["Y"]) <= TOL_F16
