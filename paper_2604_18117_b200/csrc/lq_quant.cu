@@ -302,20 +302,67 @@ __global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams 
 }
 
 // W16A16 reference branch: T = X L1 accumulated in fp32, rounded once to fp16; no scales.
-__global__ void __launch_bounds__(256) lq_down_f16_kernel(const __half* __restrict__ X, const __half* __restrict__ L1h,
+// A CTA of four warps owns 16 rows; the warps split K in chunks of 32 (chunk c goes to warp c % 4), multiply with
+// mma.sync m16n8k16 (fp16 x fp16 -> fp32) and add their partial sums in shared memory.  Both operands are fetched with
+// 16-byte loads: lane (g, t) holds elements 8t .. 8t+7 of the chunk for row g (A) or factor column g (B).  A sum over k does
+// not care which k sits in which fragment slot as long as A and B agree, so the lane's first four elements feed one k16 step
+// and its last four the next - no shuffles, and X is read once with full sectors.
+__device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int NT>   // NT: 8-column tiles of the rank (rank <= 8 NT)
+__global__ void __launch_bounds__(128) lq_down_f16_kernel(const __half* __restrict__ X, const __half* __restrict__ L1h,
                                                           int M, int K, int Kpad, int r, uint8_t* __restrict__ tq,
                                                           float* __restrict__ sT) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m = blockIdx.x * 8 + warp;
-  if (m >= M) return;
-  const __half* xrow = X + (size_t)m * K;
-  for (int j = lane; j < r; j += 32) {
-    const __half* brow = L1h + (size_t)j * Kpad;
-    float a = 0.f;
-    for (int k = 0; k < K; ++k) a = fmaf(__half2float(xrow[k]), __half2float(brow[k]), a);
-    reinterpret_cast<__half*>(tq + (size_t)m * LQ_RCONT)[j] = __float2half_rn(a);
+  __shared__ float part[4][16][NT * 8 + 1];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int m0 = blockIdx.x * 16;
+  const int r_lo = m0 + g, r_hi = m0 + g + 8;
+  float acc[NT][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[nt][i] = 0.f;
+  const uint4 zero = make_uint4(0, 0, 0, 0);
+  const int chunks = (K + 31) / 32;
+#pragma unroll 3
+  for (int c = warp; c < chunks; c += 4) {
+    const int k = c * 32 + 8 * t;
+    const bool kin = k < K;                                                        // K is a multiple of 8
+    const uint4 alo = (kin && r_lo < M) ? __ldg(reinterpret_cast<const uint4*>(X + (size_t)r_lo * K + k)) : zero;
+    const uint4 ahi = (kin && r_hi < M) ? __ldg(reinterpret_cast<const uint4*>(X + (size_t)r_hi * K + k)) : zero;
+    uint4 b[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const int j = nt * 8 + g;
+      b[nt] = (j < r) ? __ldg(reinterpret_cast<const uint4*>(L1h + (size_t)j * Kpad + k)) : zero;   // zero-padded up to Kpad
+    }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      mma_f16_16816(acc[nt], alo.x, ahi.x, alo.y, ahi.y, b[nt].x, b[nt].y);
+      mma_f16_16816(acc[nt], alo.z, ahi.z, alo.w, ahi.w, b[nt].z, b[nt].w);
+    }
   }
-  if (lane == 0) sT[m] = 1.0f;
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    part[warp][g][nt * 8 + 2 * t] = acc[nt][0];
+    part[warp][g][nt * 8 + 2 * t + 1] = acc[nt][1];
+    part[warp][g + 8][nt * 8 + 2 * t] = acc[nt][2];
+    part[warp][g + 8][nt * 8 + 2 * t + 1] = acc[nt][3];
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < 16 * NT * 8; i += 128) {
+    const int row = i / (NT * 8), j = i % (NT * 8);
+    const int m = m0 + row;
+    if (m < M && j < r) {
+      const float v = (part[0][row][j] + part[1][row][j]) + (part[2][row][j] + part[3][row][j]);
+      reinterpret_cast<__half*>(tq + (size_t)m * LQ_RCONT)[j] = __float2half_rn(v);
+    }
+  }
+  if (threadIdx.x < 16 && m0 + threadIdx.x < M) sT[m0 + threadIdx.x] = 1.0f;
 }
 
 template <int NCHUNK, int WARPS, bool RELOAD, bool MX>
@@ -366,9 +413,12 @@ lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A,
 #undef LQ_QUANT_DISPATCH
   if (lq_note_cuda(e) != cudaSuccess) return LQ_ERR_CUDA;
   if (L->f16_branch) {
-    lq_down_f16_kernel<<<lq_ceil_div(M, 8), 256, 0, st>>>(reinterpret_cast<const __half*>(X),
-                                                          reinterpret_cast<const __half*>(L->d_L1h), M, K, Kpad, L->r,
-                                                          A->d_tq, A->d_sT);
+    const __half* Xh = reinterpret_cast<const __half*>(X);
+    const __half* L1 = reinterpret_cast<const __half*>(L->d_L1h);
+    const int blocks = lq_ceil_div(M, 16);
+    if (L->r <= 16) lq_down_f16_kernel<2><<<blocks, 128, 0, st>>>(Xh, L1, M, K, Kpad, L->r, A->d_tq, A->d_sT);
+    else if (L->r <= 32) lq_down_f16_kernel<4><<<blocks, 128, 0, st>>>(Xh, L1, M, K, Kpad, L->r, A->d_tq, A->d_sT);
+    else lq_down_f16_kernel<8><<<blocks, 128, 0, st>>>(Xh, L1, M, K, Kpad, L->r, A->d_tq, A->d_sT);
     if (cudaGetLastError() != cudaSuccess) return LQ_ERR_CUDA;
   }
   return LQ_OK;
