@@ -156,6 +156,16 @@ lq_status lq_linear_forward(const lq_layer* layer, const lq_act* act, void* Y_de
 lq_status lq_linear_forward_host(const lq_layer* layer, lq_act* act, const void* X_f16_host,
                                  int32_t M, void* Y_host, lq_out_dtype dtype, void* cuda_stream);
 
+/* The same without the final wait: returns once everything is queued; Y_host is complete when
+ * `cuda_stream` has been synchronised (the stream is made to wait for the last copy).  X_f16_host
+ * and Y_host must be pinned and must stay valid until then.  Calls for different layers on
+ * different streams (each with its own `act`) overlap their copies in both directions, which a
+ * sequence of waiting calls cannot: one layer's output travels device -> host while the next
+ * layer's input travels host -> device.  Figure 1's data flow; the paper has no counterpart for
+ * the transport itself. */
+lq_status lq_linear_forward_host_async(const lq_layer* layer, lq_act* act, const void* X_f16_host,
+                                       int32_t M, void* Y_host, lq_out_dtype dtype, void* cuda_stream);
+
 /* (The paper has no counterpart for this entry point; it exists for deployment.)
  * Same result as lq_quantize_act followed by lq_linear_forward, for callers that may not
  * allocate device memory when they call: servers whose own pool owns all device memory once

@@ -51,6 +51,7 @@ _SIGNATURES = {
     "lq_quantize_act": [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p],
     "lq_linear_forward": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p],
     "lq_linear_forward_host": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_int, C.c_void_p],
+    "lq_linear_forward_host_async": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_int, C.c_void_p],
     "lq_linear_forward_static": [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_int, C.c_void_p],
     "lq_act_export": [C.c_void_p] * 8,
     "lq_get_device_status": [C.c_int, C.POINTER(C.c_int32), C.POINTER(C.c_int32)],
@@ -183,6 +184,11 @@ def lq_linear_forward(layer, act, Y_dev_ptr: int, dtype: int = OUT_F16, stream: 
 def lq_linear_forward_host(layer, act, X_host_ptr: int, M: int, Y_host_ptr: int, dtype: int = OUT_F16, stream: int = 0):
     _check(lib().lq_linear_forward_host(layer, act, C.c_void_p(X_host_ptr), M, C.c_void_p(Y_host_ptr), dtype,
                                         C.c_void_p(stream)), "lq_linear_forward_host")
+
+
+def lq_linear_forward_host_async(layer, act, X_host_ptr: int, M: int, Y_host_ptr: int, dtype: int = OUT_F16, stream: int = 0):
+    _check(lib().lq_linear_forward_host_async(layer, act, C.c_void_p(X_host_ptr), M, C.c_void_p(Y_host_ptr), dtype,
+                                        C.c_void_p(stream)), "lq_linear_forward_host_async")
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

@@ -437,8 +437,8 @@ extern "C" lq_status lq_linear_forward(const lq_layer* L, const lq_act* A, void*
   return L->mx ? lq_launch_gemm_mx(L, A, Y, dt, (cudaStream_t)stream) : lq_launch_gemm(L, A, Y, dt, (cudaStream_t)stream);
 }
 
-extern "C" lq_status lq_linear_forward_host(const lq_layer* L, lq_act* A, const void* Xh, int32_t M, void* Yh,
-                                            lq_out_dtype dt, void* stream) {
+static lq_status forward_host(const lq_layer* L, lq_act* A, const void* Xh, int32_t M, void* Yh, lq_out_dtype dt, void* stream,
+                              bool wait) {
   if (!L || !A || !Xh || !Yh) return LQ_ERR_INVALID_ARG;
   if (!act_matches(L, A)) return LQ_ERR_INVALID_ARG;
   if (M <= 0 || M > A->M_max) return LQ_ERR_INVALID_ARG;
@@ -502,9 +502,19 @@ extern "C" lq_status lq_linear_forward_host(const lq_layer* L, lq_act* A, const 
   }
   A->M = M;
   CUDA_OK(cudaEventRecord(A->ev_end, A->s_d2h));
-  CUDA_OK(cudaStreamWaitEvent(st, A->ev_end, 0));
-  CUDA_OK(cudaStreamSynchronize(st));
+  CUDA_OK(cudaStreamWaitEvent(st, A->ev_end, 0));              // the caller's stream is done when Y has arrived
+  if (wait) CUDA_OK(cudaStreamSynchronize(st));
   return LQ_OK;
+}
+
+extern "C" lq_status lq_linear_forward_host(const lq_layer* L, lq_act* A, const void* Xh, int32_t M, void* Yh,
+                                            lq_out_dtype dt, void* stream) {
+  return forward_host(L, A, Xh, M, Yh, dt, stream, true);
+}
+
+extern "C" lq_status lq_linear_forward_host_async(const lq_layer* L, lq_act* A, const void* Xh, int32_t M, void* Yh,
+                                                  lq_out_dtype dt, void* stream) {
+  return forward_host(L, A, Xh, M, Yh, dt, stream, false);
 }
 
 static int decode_code(uint8_t b, int kind) {

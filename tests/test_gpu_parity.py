@@ -205,3 +205,38 @@ def test_bounded_wait_reports_timeout_and_device_stays_usable():
     rng = np.random.default_rng(7)
     X = rng.standard_normal((130, 320)).astype(np.float16)
     _check(_random_layer(rng, 320, 72, 16, "w8a8"), X)
+
+
+def test_async_host_entry_point_on_two_streams():
+    """lq_linear_forward_host_async returns before Y has arrived; after the stream is synchronised Y equals the waiting
+    call's result bit for bit.  Two layers on two streams run their copies and kernels concurrently."""
+    import torch
+    from tests.helpers import import_oracle_layer
+    rng = np.random.default_rng(8)
+    M = 1300
+    jobs = []
+    for (K, N, r, br) in ((1152, 392, 32, "w8a8"), (640, 1160, 16, "w6a6")):
+        X = rng.standard_normal((M, K)).astype(np.float16)
+        layer = _random_layer(rng, K, N, r, br)
+        h, _ = import_oracle_layer(layer)
+        B.lq_layer_to_device(h, 0)
+        jobs.append(dict(h=h, act=B.lq_act_create(h, M, 0), Xp=torch.from_numpy(X).pin_memory(), N=N,
+                         ref=O.forward(X, layer)["Y"], stream=torch.cuda.Stream()))
+    try:
+        for j in jobs:                                      # reference: the waiting call
+            j["Yw"] = torch.full((M, j["N"]), float("nan"), dtype=torch.float16).pin_memory()
+            B.lq_linear_forward_host(j["h"], j["act"], j["Xp"].data_ptr(), M, j["Yw"].data_ptr(), B.OUT_F16, j["stream"].cuda_stream)
+        for _ in range(2):
+            for j in jobs:
+                j["Ya"] = torch.full((M, j["N"]), float("nan"), dtype=torch.float16).pin_memory()
+                B.lq_linear_forward_host_async(j["h"], j["act"], j["Xp"].data_ptr(), M, j["Ya"].data_ptr(), B.OUT_F16,
+                                               j["stream"].cuda_stream)
+            for j in jobs:
+                j["stream"].synchronize()
+                assert np.array_equal(j["Ya"].numpy(), j["Yw"].numpy())
+                assert rel_fro(j["Ya"].numpy(), j["ref"]) <= TOL_F16
+        assert B.lq_get_device_status(0)[0] == 0
+    finally:
+        for j in jobs:
+            B.lq_act_free(j["act"])
+            B.lq_layer_free(j["h"])
