@@ -148,7 +148,8 @@ lq_status lq_linear_forward(const lq_layer* layer, const lq_act* act, void* Y_de
 
 /* Whole path from host memory: copies X to the device, runs lq_quantize_act and
  * lq_linear_forward, copies Y back and waits for it.  X_f16_host [M][K], Y_host [M][N].
- * Rows are independent, so for M >= 1024 the call is pipelined over four row chunks: one chunk
+ * Rows are independent, so for M >= 512 the call is pipelined over up to eight row chunks (of at
+ * least 256 rows): one chunk
  * is computed on `cuda_stream` while the next travels host -> device and the previous one
  * device -> host on two internal copy streams (this needs pinned host memory to overlap;
  * pageable memory works but serialises).  Staging buffers, streams and events inside `act`

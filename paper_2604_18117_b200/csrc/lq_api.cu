@@ -465,7 +465,7 @@ static lq_status forward_host(const lq_layer* L, lq_act* A, const void* Xh, int3
     CUDA_OK(cudaEventCreateWithFlags(&A->ev_end, cudaEventDisableTiming));
     A->pipe_ready = true;
   }
-  const int nchunk = M >= LQ_HOST_CHUNKS * 2 * LQ_BM ? LQ_HOST_CHUNKS : 1;
+  const int nchunk = std::max(1, std::min(LQ_HOST_CHUNKS, M / (2 * LQ_BM)));   // chunks of at least 256 rows
   const int rows_per = lq_round_up(lq_ceil_div(M, nchunk), LQ_BM);
   const size_t esz = dt == LQ_OUT_F32 ? 4 : 2;
   CUDA_OK(cudaEventRecord(A->ev_begin, st));                  // copies start after what the caller queued before

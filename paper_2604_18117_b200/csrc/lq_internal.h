@@ -17,7 +17,7 @@
 #define LQ_RCONT 128         // bytes per row of the branch containers (tq, L2q): rank <= 128
 #define LQ_MAX_K 8192
 #define LQ_MAX_RANK 128
-#define LQ_HOST_CHUNKS 4       // row chunks lq_linear_forward_host overlaps (copy in / compute / copy out)
+#define LQ_HOST_CHUNKS 8       // row chunks (at most) lq_linear_forward_host overlaps (copy in / compute / copy out)
 
 // role identifiers reported through the device status word
 enum { LQ_STAGE_NONE = 0, LQ_STAGE_PRODUCER = 1, LQ_STAGE_MMA = 2, LQ_STAGE_DRAIN = 3, LQ_STAGE_TEARDOWN = 4 };

@@ -162,7 +162,7 @@ def test_host_entry_point_pipelines_row_chunks():
     import torch
     from tests.helpers import import_oracle_layer
     rng = np.random.default_rng(6)
-    M, K, N, r = 1300, 1152, 392, 32                       # four chunks, the last one ragged; N not a multiple of 128
+    M, K, N, r = 1300, 1152, 392, 32                       # five chunks, the last one ragged; N not a multiple of 128
     X = rng.standard_normal((M, K)).astype(np.float16)
     layer = _random_layer(rng, K, N, r, "w8a8")
     ref = O.forward(X, layer)
