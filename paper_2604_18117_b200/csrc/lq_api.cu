@@ -11,6 +11,8 @@
 int g_lq_main_kind = LQ_KIND_E4M3;
 int g_lq_gemm_ctas = 0;
 int g_lq_store_qb = 0;
+int g_lq_quant_warps = 0;
+int g_lq_quant_ctas = 0;
 
 static thread_local cudaError_t t_last_cuda_error = cudaSuccess;
 
@@ -55,6 +57,16 @@ extern "C" lq_status lq_set_option(const char* name, int32_t value) {
   }
   if (!strcmp(name, "store_qb")) {
     g_lq_store_qb = value != 0;
+    return LQ_OK;
+  }
+  if (!strcmp(name, "quant_warps")) {
+    if (value < 0 || value > 9) return LQ_ERR_INVALID_ARG;
+    g_lq_quant_warps = value;
+    return LQ_OK;
+  }
+  if (!strcmp(name, "quant_ctas")) {
+    if (value < 0 || value > 4) return LQ_ERR_INVALID_ARG;
+    g_lq_quant_ctas = value;
     return LQ_OK;
   }
   if (!strcmp(name, "gemm_ctas")) {
@@ -211,7 +223,7 @@ static encode_tiled_fn get_encode_fn() {
 }
 
 // 2-D byte tensor [rows][row_bytes], box [box_rows][128 bytes], 128-byte swizzle.
-static lq_status make_tmap_bytes(CUtensorMap* tm, void* base, uint64_t rows, uint64_t row_bytes, uint32_t box_rows) {
+lq_status lq_make_tmap_bytes(CUtensorMap* tm, void* base, uint64_t rows, uint64_t row_bytes, uint32_t box_rows) {
   encode_tiled_fn fn = get_encode_fn();
   if (!fn) return LQ_ERR_CUDA;
   cuuint64_t dims[2] = {row_bytes, rows};
@@ -220,6 +232,19 @@ static lq_status make_tmap_bytes(CUtensorMap* tm, void* base, uint64_t rows, uin
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? LQ_OK : LQ_ERR_CUDA;
+}
+
+lq_status lq_make_tmap_rows16(CUtensorMap* tm, const void* X, uint64_t M, uint64_t K) {
+  encode_tiled_fn fn = get_encode_fn();
+  if (!fn) return LQ_ERR_CUDA;
+  cuuint64_t dims[2] = {K, M};
+  cuuint64_t strides[1] = {K * 2};
+  cuuint32_t box[2] = {64, 16};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? LQ_OK : LQ_ERR_CUDA;
 }
 
@@ -315,19 +340,16 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
     std::vector<float> s1(LQ_MAX_RANK, 1.f), s2((size_t)Npad, 1.f);
     std::vector<uint8_t> l2c((size_t)Npad * LQ_RCONT, 0);
     if (L->integer_branch) {
-      // B fragments of mma.sync.m16n8k32 (s8): lane = 4 * (n % 8) + t holds k = 32 ks + 4 t + {0..3} and + 16
-      const int rpad = lq_round_up(r, 8), ksteps = Kpad / 32, ntiles = rpad / 8;
-      std::vector<uint8_t> l1f((size_t)ksteps * ntiles * 32 * 8, 0);
-      for (int ks = 0; ks < ksteps; ++ks)
+      // B fragments of mma.sync.m16n8k32 (s8) under the k order the quantizer's lanes hold their codes in: per box of
+      // 64 values and 8-column tile, lane 4 c + t carries k = 64 box + 16 t + 0..15 of column 8 tile + c
+      const int ntiles = lq_quant_rank_tiles(r, false), nbox = Kpad / 64;
+      std::vector<uint8_t> l1f((size_t)nbox * ntiles * 32 * 16, 0);
+      for (int b = 0; b < nbox; ++b)
         for (int nt = 0; nt < ntiles; ++nt)
           for (int lane = 0; lane < 32; ++lane) {
-            const int j = nt * 8 + (lane >> 2), kb = ks * 32 + (lane & 3) * 4;
-            uint8_t* dst = &l1f[(((size_t)ks * ntiles + nt) * 32 + lane) * 8];
-            for (int i = 0; i < 4; ++i) {
-              const int k0 = kb + i, k1 = kb + 16 + i;
-              dst[i] = (j < r && k0 < K) ? (uint8_t)L->L1q[(size_t)k0 * r + j] : 0;
-              dst[4 + i] = (j < r && k1 < K) ? (uint8_t)L->L1q[(size_t)k1 * r + j] : 0;
-            }
+            const int j = nt * 8 + (lane >> 2), kb = b * 64 + (lane & 3) * 16;
+            uint8_t* dst = &l1f[(((size_t)b * ntiles + nt) * 32 + lane) * 16];
+            for (int i = 0; i < 16; ++i) dst[i] = (j < r && kb + i < K) ? (uint8_t)L->L1q[(size_t)(kb + i) * r + j] : 0;
           }
       if ((st = upload(&L->d_L1f, l1f)) != LQ_OK) return st;
       for (int j = 0; j < r; ++j) s1[j] = L->sL1[j];
@@ -335,9 +357,16 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
       for (int j = 0; j < r; ++j)
         for (int n = 0; n < N; ++n) l2c[(size_t)n * LQ_RCONT + j] = (uint8_t)L->L2q[(size_t)j * N + n];
     } else if (L->f16_branch) {
-      std::vector<uint16_t> l1t((size_t)r * Kpad, 0);
-      for (int k = 0; k < K; ++k)
-        for (int j = 0; j < r; ++j) l1t[(size_t)j * Kpad + k] = L->L1h[(size_t)k * r + j];
+      // the same fragment order with 16 halves per lane (mma.sync.m16n8k16, four k steps per box)
+      const int ntiles = lq_quant_rank_tiles(r, true), nbox = Kpad / 64;
+      std::vector<uint16_t> l1t((size_t)nbox * ntiles * 32 * 16, 0);
+      for (int b = 0; b < nbox; ++b)
+        for (int nt = 0; nt < ntiles; ++nt)
+          for (int lane = 0; lane < 32; ++lane) {
+            const int j = nt * 8 + (lane >> 2), kb = b * 64 + (lane & 3) * 16;
+            uint16_t* dst = &l1t[(((size_t)b * ntiles + nt) * 32 + lane) * 16];
+            for (int i = 0; i < 16; ++i) dst[i] = (j < r && kb + i < K) ? L->L1h[(size_t)(kb + i) * r + j] : 0;
+          }
       if ((st = upload(&L->d_L1h, l1t)) != LQ_OK) return st;
       uint16_t* c16 = (uint16_t*)l2c.data();
       for (int j = 0; j < r; ++j)
@@ -347,9 +376,9 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
     if ((st = upload(&L->d_sL2, s2)) != LQ_OK) return st;
     if ((st = upload(&L->d_L2c, l2c)) != LQ_OK) return st;
   } catch (const std::bad_alloc&) { return LQ_ERR_ALLOC; }
-  if ((st = make_tmap_bytes(&L->tmB, L->d_Wq8, Npad, Kpad, LQ_BN)) != LQ_OK) return st;
-  if ((st = make_tmap_bytes(&L->tmB2, L->d_Wq8, Npad, Kpad, 2 * LQ_BN)) != LQ_OK) return st;
-  if ((st = make_tmap_bytes(&L->tmL2, L->d_L2c, Npad, LQ_RCONT, LQ_BN)) != LQ_OK) return st;
+  if ((st = lq_make_tmap_bytes(&L->tmB, L->d_Wq8, Npad, Kpad, LQ_BN)) != LQ_OK) return st;
+  if ((st = lq_make_tmap_bytes(&L->tmB2, L->d_Wq8, Npad, Kpad, 2 * LQ_BN)) != LQ_OK) return st;
+  if ((st = lq_make_tmap_bytes(&L->tmL2, L->d_L2c, Npad, LQ_RCONT, LQ_BN)) != LQ_OK) return st;
   if (!lq_device_status_ptr(device)) return LQ_ERR_CUDA;
   if ((st = lq_gemm_prepare(device)) != LQ_OK) return st;
   if (L->mx && (st = lq_gemm_mx_prepare(device)) != LQ_OK) return st;
@@ -393,8 +422,8 @@ extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device,
   cudaMemset(A->d_sT, 0, Mp * sizeof(float));
   if (A->mx) cudaMemset(A->d_sfa, 127, (Mp / 128) * (Kp / 128) * 512);
   lq_status st;
-  if ((st = make_tmap_bytes(&A->tmA, A->d_qx8, Mp, Kp, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
-  if ((st = make_tmap_bytes(&A->tmT, A->d_tq, Mp, LQ_RCONT, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
+  if ((st = lq_make_tmap_bytes(&A->tmA, A->d_qx8, Mp, Kp, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
+  if ((st = lq_make_tmap_bytes(&A->tmT, A->d_tq, Mp, LQ_RCONT, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
   if (cudaDeviceSynchronize() != cudaSuccess) { lq_act_free(A); return LQ_ERR_CUDA; }
   *out = A;
   return LQ_OK;
@@ -492,8 +521,8 @@ static lq_status forward_host(const lq_layer* L, lq_act* A, const void* Xh, int3
     V.d_sT = A->d_sT + m0;
     if (A->mx) V.d_sfa = A->d_sfa + (size_t)(m0 / 128) * (A->Kpad / 128) * 512;
     lq_status s;
-    if ((s = make_tmap_bytes(&V.tmA, V.d_qx8, (uint64_t)(A->Mpad - m0), A->Kpad, LQ_BM)) != LQ_OK) return s;
-    if ((s = make_tmap_bytes(&V.tmT, V.d_tq, (uint64_t)(A->Mpad - m0), LQ_RCONT, LQ_BM)) != LQ_OK) return s;
+    if ((s = lq_make_tmap_bytes(&V.tmA, V.d_qx8, (uint64_t)(A->Mpad - m0), A->Kpad, LQ_BM)) != LQ_OK) return s;
+    if ((s = lq_make_tmap_bytes(&V.tmT, V.d_tq, (uint64_t)(A->Mpad - m0), LQ_RCONT, LQ_BM)) != LQ_OK) return s;
     if ((s = lq_launch_quantize(L, xd, Mc, &V, st)) != LQ_OK) return s;
     if ((s = (L->mx ? lq_launch_gemm_mx(L, &V, yd, dt, st) : lq_launch_gemm(L, &V, yd, dt, st))) != LQ_OK) return s;
     CUDA_OK(cudaEventRecord(A->ev_y[c], st));

@@ -20,7 +20,7 @@
 #define LQ_HOST_CHUNKS 8       // row chunks (at most) lq_linear_forward_host overlaps (copy in / compute / copy out)
 
 // role identifiers reported through the device status word
-enum { LQ_STAGE_NONE = 0, LQ_STAGE_PRODUCER = 1, LQ_STAGE_MMA = 2, LQ_STAGE_DRAIN = 3, LQ_STAGE_TEARDOWN = 4 };
+enum { LQ_STAGE_NONE = 0, LQ_STAGE_PRODUCER = 1, LQ_STAGE_MMA = 2, LQ_STAGE_DRAIN = 3, LQ_STAGE_TEARDOWN = 4, LQ_STAGE_QUANT = 5 };
 
 enum { LQ_KIND_I8 = 0, LQ_KIND_E4M3 = 1 };
 
@@ -64,8 +64,9 @@ struct lq_layer {
   int main_kind;               // LQ_KIND_*: byte encoding of the 4-bit codes in the MMA operands
   uint8_t* d_Wq8;              // [Npad][Kpad] bytes, K contiguous (B operand, K-major)
   float* d_sw;                 // [Gpad][Npad] fp32 (exact images of the fp16 scales)
-  uint8_t* d_L1f;              // [Kpad/32][rpad/8][32 lanes][8 bytes]: first factor in mma.sync B-fragment order (integer branches)
-  uint16_t* d_L1h;             // [r][Kpad] half, K contiguous   (W16A16)
+  uint8_t* d_L1f;              // [Kpad/64][r tiles][32 lanes][16 bytes]: first factor in mma.sync B-fragment order (integer
+                               // branches): lane 4 c + t holds k = 64 box + 16 t + 0..15 of column 8 tile + c
+  uint16_t* d_L1h;             // the same order with 16 halves per lane (W16A16)
   float* d_sL1;                // [LQ_MAX_RANK]
   uint8_t* d_L2c;              // [Npad][LQ_RCONT] bytes: int8 codes (or up to 64 halves) of column n, r contiguous
   float* d_sL2;                // [Npad]  (ones for W16A16)
@@ -111,7 +112,14 @@ lq_status lq_launch_gemm(const lq_layer* L, const lq_act* A, void* Y, lq_out_dty
 lq_status lq_gemm_prepare(int device);
 lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_dtype dt, cudaStream_t st);
 lq_status lq_gemm_mx_prepare(int device);
-lq_status lq_launch_wait_probe(int device, cudaStream_t st);   // bounded-wait self-test kernel   // sets the kernel's shared-memory attribute once per device
+lq_status lq_launch_wait_probe(int device, cudaStream_t st);   // bounded-wait self-test kernel
+int lq_quant_rank_tiles(int r, bool f16);   // 8-column tiles of the rank the quantizer kernels are built for (2, 4, 8 or 16)
+
+// TMA descriptors (lq_api.cu).  lq_make_tmap_bytes: 2-D byte tensor [rows][row_bytes], box [box_rows][128 bytes],
+// 128-byte swizzle.  lq_make_tmap_rows16: fp16 activations [M][K], box 16 rows x 64 values, 128-byte swizzle,
+// zeros outside the tensor.
+lq_status lq_make_tmap_bytes(CUtensorMap* tm, void* base, uint64_t rows, uint64_t row_bytes, uint32_t box_rows);
+lq_status lq_make_tmap_rows16(CUtensorMap* tm, const void* X, uint64_t M, uint64_t K);
 
 // byte an MMA operand carries for a 4-bit code q in [-7, 7]
 static inline uint8_t lq_encode_code_host(int q, int kind) {
@@ -123,4 +131,5 @@ static inline uint8_t lq_encode_code_host(int q, int kind) {
 
 extern int g_lq_main_kind;   // option "main_kind"
 extern int g_lq_gemm_ctas;   // option "gemm_ctas" (0 = one per SM)
+extern int g_lq_quant_warps, g_lq_quant_ctas;   // options "quant_warps", "quant_ctas": 0 = chosen by the launcher
 extern int g_lq_store_qb;    // option "store_qb": also write the branch activation codes to HBM (parity export)

@@ -26,35 +26,6 @@ namespace {
 std::mutex g_mu;
 unsigned char* g_scratch_dev[64] = {nullptr};   // device address of the array, per device
 
-typedef CUresult (*encode_fn_t)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-encode_fn_t encode_fn() {
-  static encode_fn_t fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = (encode_fn_t)p;
-  });
-  return fn;
-}
-
-// [rows][row_bytes] bytes, box [128 rows][128 bytes], 128-byte swizzle (the GEMM's A-side operands)
-bool encode_rows(CUtensorMap* tm, void* base, uint64_t rows, uint64_t row_bytes) {
-  encode_fn_t fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t dims[2] = {row_bytes, rows};
-  cuuint64_t strides[1] = {row_bytes};
-  cuuint32_t box[2] = {128, LQ_BM};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 }  // namespace
@@ -79,13 +50,13 @@ extern "C" lq_status lq_linear_forward_static(const lq_layer* L, const void* X, 
   const size_t o_sT = off; off = align256(off + Mpad * sizeof(float));
   if (off > (size_t)LQ_STATIC_SCRATCH_BYTES) return LQ_ERR_UNSUPPORTED;  // M x K too large for the fixed array
 
-  if (cudaSetDevice(L->device) != cudaSuccess) return LQ_ERR_CUDA;
+  if (lq_note_cuda(cudaSetDevice(L->device)) != cudaSuccess) return LQ_ERR_CUDA;
   unsigned char* base = nullptr;
   {
     std::lock_guard<std::mutex> lk(g_mu);
     if (!g_scratch_dev[L->device]) {
       void* p = nullptr;
-      if (cudaGetSymbolAddress(&p, g_lq_static_scratch) != cudaSuccess || !p) return LQ_ERR_CUDA;
+      if (lq_note_cuda(cudaGetSymbolAddress(&p, g_lq_static_scratch)) != cudaSuccess || !p) return LQ_ERR_CUDA;
       g_scratch_dev[L->device] = (unsigned char*)p;
     }
     base = g_scratch_dev[L->device];
@@ -93,7 +64,7 @@ extern "C" lq_status lq_linear_forward_static(const lq_layer* L, const void* X, 
   cudaStream_t st = (cudaStream_t)stream;
   // The array keeps the previous call's contents; padding columns, padding rows and the tail
   // of the rank-r containers must read as zero codes, so clear the part this call uses.
-  if (cudaMemsetAsync(base, 0, off, st) != cudaSuccess) return LQ_ERR_CUDA;
+  if (lq_note_cuda(cudaMemsetAsync(base, 0, off, st)) != cudaSuccess) return LQ_ERR_CUDA;
 
   lq_act A;
   memset(&A, 0, sizeof(A));
@@ -105,9 +76,9 @@ extern "C" lq_status lq_linear_forward_static(const lq_layer* L, const void* X, 
   A.d_sXb = (float*)(base + o_sXb);
   A.d_tq = base + o_tq;
   A.d_sT = (float*)(base + o_sT);
-  if (!encode_rows(&A.tmA, A.d_qx8, Mpad, Kpad)) return LQ_ERR_CUDA;
-  if (!encode_rows(&A.tmT, A.d_tq, Mpad, LQ_RCONT)) return LQ_ERR_CUDA;
-  lq_status s = lq_launch_quantize(L, X, M, &A, st);
-  if (s != LQ_OK) return s;
+  lq_status s;
+  if ((s = lq_make_tmap_bytes(&A.tmA, A.d_qx8, Mpad, Kpad, LQ_BM)) != LQ_OK) return s;
+  if ((s = lq_make_tmap_bytes(&A.tmT, A.d_tq, Mpad, LQ_RCONT, LQ_BM)) != LQ_OK) return s;
+  if ((s = lq_launch_quantize(L, X, M, &A, st)) != LQ_OK) return s;
   return lq_launch_gemm(L, &A, Y, dt, st);
 }

@@ -1,34 +1,66 @@
-// Activation side of the layer, ONE kernel and one read of X (Figure 1; Appendix A.2: the
-// activations forwarded to both branches are quantized):
-//   a1  SINT4 codes + fp16 scales per token and group of 64 along K          (Appendix A.3)
+// Activation side of the layer, ONE kernel and one read of X from HBM (Figure 1; Appendix A.2: both branches
+// consume quantized X, except the full-precision reference branch of Section 4.2 / Table 2):
+//   a1  4-bit codes + scales per token and group of 64 along K (SINT4, Appendix A.3) or block of 32 (MXINT4)
 //   a2  per-token codes of the low-rank branch (needs the whole row's maximum first)
-//   a3  down-projection I1 = qb L1q, exact int32, on the tensor cores (mma.sync, s8)
+//   a3  down-projection I1 = qb L1q, exact int32, on mma.sync (s8) - or T = X L1 in fp16 x fp16 -> fp32 for the
+//       fp16 reference branch - straight from the registers that hold the freshly made codes
 //   a4  t = fl32(fl32(I1) * fl32(sXb * sL1)), per-token re-quantization of the rank-r row
 //
-// A CTA owns 16 rows (one m16 MMA tile).  A warp holds one row in registers (16-byte loads,
-// X is read from HBM exactly once), finds the row maximum, then walks the row once more and
-// emits both code streams; the CTA then multiplies its 16 x K tile of branch codes, staged in
-// shared memory, with L1q.
+// Shape of the kernel: persistent CTAs walk 16-row tiles.  A tile arrives as TMA boxes of 16 rows x 64 values
+// (128-byte swizzle); W consumer warps each own the boxes g = w, w + W, ... of a tile, and each has a private ring
+// of D shared-memory slots with a full/empty mbarrier pair per slot, fed by one lane of the producer warp (lane w
+// serves warp w: a slot is always filled and drained by the same pair, strictly in order, so a one-bit phase
+// never aliases even though copies complete out of order).  A lane (gid, tig) of a consumer warp
+// holds 16 consecutive values of rows gid and gid + 8 - exactly one operand fragment of the m16 MMA under a
+// k order that A and B share (a sum over k does not care which k sits in which fragment slot), so the branch
+// codes never touch shared memory.  With an integer branch a tile is walked twice (row maxima, then codes);
+// when the ring holds a whole tile the second walk reads the same slots, otherwise the producer streams the
+// tile a second time (served by the L2: DRAM still sees X once).
 //
 // Exactness contract: codes and scales equal the definition evaluated in IEEE binary32 with
-// round-to-nearest-even and true division.  The fast path is division free:
-//   scale   fp16(a / 7) == fp16(a * fl32(1/7)) for every finite fp16 a (checked exhaustively on
-//           the host), because a/7 never comes closer than 2^-15 (relative) to an fp16 midpoint.
-//   main    q' = rint(x * r), r ~ 1/s; e = fma(-q', s, x) is exact (q' has 3 bits, s 11 bits).
-//           x and s are fp16 numbers, so x/s is either exactly k + 1/2 or at least 1e-4 away
-//           from it, while x * r is within 3e-6 of x/s: q' is the correctly rounded code unless
-//           |e| == s/2 exactly (a true tie) - those elements take the exact path.
-//   branch  same with the fp32 per-token scale; an element takes the exact path (IEEE division)
-//           whenever |e| >= 0.4999 s, i.e. whenever the quotient is not safely inside a
-//           rounding cell (the estimate is within 5e-5 of the quotient).
+// round-to-nearest-even and true division.  The kernel is division free:
+//   scale     fp16(a / 7) == fp16(a * fl32(1/7)) for every finite fp16 a (checked exhaustively on the host),
+//             because a/7 never comes closer than 2^-15 (relative) to an fp16 midpoint.
+//   quotient  x / s from the correctly rounded reciprocal by one FMA correction step, which yields the correctly
+//             rounded binary32 quotient (div_rn_by below); rounding to the nearest even integer by adding
+//             1.5 * 2^23.  MXINT4: 1/s is a power of two, so x * (1/s) is already exact.
 #include <cuda_fp16.h>
 
-#include "lq_internal.h"
+#include <algorithm>
+
+#include "lq_device.cuh"
 
 namespace {
 
-constexpr int ROWS = 16;               // rows per CTA
+using namespace lqdev;
+
+constexpr int TR = 16;                 // rows per tile (one m16 MMA tile)
+constexpr int BOX_K = 64;              // values of K per box: one 128-byte swizzle row
+constexpr int BOX_BYTES = TR * BOX_K * 2;
 constexpr float MAGIC = 12582912.0f;   // 1.5 * 2^23: adding it rounds to an integer (ties to even)
+constexpr int MAX_CONSUMER_WARPS = 9;
+enum { BR_NONE = 0, BR_INT = 1, BR_F16 = 2 };
+
+struct QuantParams {
+  int M, K, Kpad, Mpad;
+  int G;                // scales per row that hold data: ceil(K / 64) (SINT4) or ceil(K / 32) (MXINT4)
+  int nbox;             // Kpad / 64 boxes per tile (trailing ones may be all padding: their codes are zeros)
+  int ntiles;           // ceil(M / 16)
+  int depth;            // D: ring slots per consumer warp
+  int refetch;          // 1: a warp's ring is smaller than its share of a tile, the producer streams every tile twice
+  uint8_t* qx8;         // [Mpad][Kpad]
+  float* sx;            // [Gpad][Mpad]
+  uint8_t* sfa;         // MXINT4: E8M0 scale bytes [Mpad/128][Kpad/128][512]
+  int8_t* qb;           // [Mpad][Kpad] or null (not stored)
+  float* sXb;           // [Mpad]
+  const uint4* L1f;     // first factor in fragment order: [nbox][r tiles][32 lanes] x 16 bytes (int8) or 32 bytes (fp16)
+  const float* sL1;     // [LQ_MAX_RANK]
+  uint8_t* tq;          // [Mpad][LQ_RCONT]
+  float* sT;            // [Mpad]
+  int r, rpad;          // rank, rank rounded up to 8
+  float qm;             // largest branch activation code
+  int32_t* status;
+};
 
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
@@ -43,383 +75,547 @@ __device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float hi, float lo) {
   return (uint32_t)r;
 }
 
-__device__ __forceinline__ float rcp_fast(float x) {
-  float r;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-  return r;
-}
-
-__device__ __forceinline__ void mma_s8_16832(int (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void mma_s8_16832(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-
-struct QuantParams {
-  const uint4* X;       // [M][K] halves
-  int M, K, Kpad, Mpad, G;
-  uint8_t* qx8;         // [Mpad][Kpad]
-  float* sx;            // [Gpad][Mpad]
-  uint8_t* sfa;         // MXINT4: E8M0 scale bytes [Mpad/128][Kpad/128][512]
-  int8_t* qb;           // [Mpad][Kpad] or null (not stored)
-  float* sXb;           // [Mpad]
-  const uint2* L1f;     // [Kpad/32][rpad/8][32] fragment-major first factor
-  const float* sL1;     // [LQ_MAX_RANK]
-  uint8_t* tq;          // [Mpad][LQ_RCONT]
-  float* sT;            // [Mpad]
-  int r, rpad;          // rank, rank rounded up to 8
-  int branch_qmax;      // 0: no integer branch
-};
-
-// Shared memory: qb tile [ROWS][Kpad + 16] bytes | sx tile [Gpad][ROWS] floats | I1 [ROWS][rpad] ints | sXb [ROWS]
-// RELOAD: rows too long for the register file are read twice, chunk by chunk - once for the row maximum,
-// once to quantize; the second read is served by the L2 (the row was touched microseconds earlier), so DRAM
-// still sees X once, and the kernel keeps 64 registers per thread and full occupancy.
-template <int NCHUNK, int WARPS, bool RELOAD, bool MX>
-__global__ void __launch_bounds__(WARPS * 32) lq_quant_kernel(const QuantParams p) {
-  extern __shared__ __align__(16) uint8_t qsm[];
-  constexpr int RPW = ROWS / WARPS;    // rows per warp
-  const int qb_stride = p.Kpad + 16;
-  const int Gpad = p.Kpad / LQ_GROUP;
-  uint8_t* qb_s = qsm;
-  float* sx_s = reinterpret_cast<float*>(qsm + (p.branch_qmax > 0 ? ROWS * qb_stride : 0));
-  int* I1_s = reinterpret_cast<int*>(sx_s + Gpad * ROWS);
-  float* sXb_s = reinterpret_cast<float*>(I1_s + ROWS * p.rpad);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * ROWS;
-  const float qm = (float)p.branch_qmax;
-
-  for (int i = threadIdx.x; i < ROWS * p.rpad; i += WARPS * 32) I1_s[i] = 0;
-
-#pragma unroll 1
-  for (int rr = 0; rr < RPW; ++rr) {
-    const int rl = warp * RPW + rr;
-    const int m = m0 + rl;
-    if (m >= p.M) {   // tail rows: zero codes so the MMA tile is defined
-      if (p.branch_qmax > 0)
-        for (int k = lane * 16; k < p.Kpad; k += 512) *reinterpret_cast<uint4*>(qb_s + rl * qb_stride + k) = make_uint4(0, 0, 0, 0);
-      continue;
-    }
-    const uint4* xrow = p.X + (size_t)m * (p.K / 8);
-    constexpr int NKEEP = RELOAD ? 1 : NCHUNK;
-    uint4 v[NKEEP];
-    __half hm[NKEEP];
-    __half hrow = __ushort_as_half((unsigned short)0);
-    // ---- pass A: this lane's maximum per chunk (exact in fp16) and the row maximum
-    auto lane_max = [](const uint4& w) {
-      const __half2* h2 = reinterpret_cast<const __half2*>(&w);
-      const __half2 m2 = __hmax2(__hmax2(__habs2(h2[0]), __habs2(h2[1])), __hmax2(__habs2(h2[2]), __habs2(h2[3])));
-      return __hmax(__low2half(m2), __high2half(m2));
-    };
-    if constexpr (RELOAD) {
-#pragma unroll 6
-      for (int c = 0; c < NCHUNK; ++c) {
-        const int k0 = c * 256 + lane * 8;
-        const uint4 w = (k0 < p.K) ? __ldg(xrow + (k0 >> 3)) : make_uint4(0, 0, 0, 0);
-        hrow = __hmax(hrow, lane_max(w));
-      }
-    } else {
-#pragma unroll
-      for (int c = 0; c < NCHUNK; ++c) {
-        const int k0 = c * 256 + lane * 8;
-        v[c] = (k0 < p.K) ? __ldg(xrow + (k0 >> 3)) : make_uint4(0, 0, 0, 0);
-      }
-#pragma unroll
-      for (int c = 0; c < NCHUNK; ++c) {
-        hm[c] = lane_max(v[c]);
-        hrow = __hmax(hrow, hm[c]);
-      }
-    }
-    float sb = 1.0f, invb = 1.0f, thr = 0.f;
-    if (p.branch_qmax > 0) {
-      const float rowmax = warp_max(__half2float(hrow));
-      sb = (rowmax == 0.f) ? 1.0f : __fdiv_rn(rowmax, qm);
-      invb = __frcp_rn(sb);
-      thr = 0.4999f * sb;
-      if (lane == 0) { sXb_s[rl] = sb; p.sXb[m] = sb; }
-    }
-    // ---- pass B: group scales, 4-bit codes (a1) and branch codes (a2)
-#pragma unroll(RELOAD ? 3 : NCHUNK)
-    for (int c = 0; c < NCHUNK; ++c) {
-      const int k0 = c * 256 + lane * 8;
-      uint4 vc;
-      float a;
-      if constexpr (RELOAD) {
-        vc = (k0 < p.K) ? __ldg(xrow + (k0 >> 3)) : make_uint4(0, 0, 0, 0);
-        a = __half2float(lane_max(vc));
-      } else {
-        vc = v[c];
-        a = __half2float(hm[c]);
-      }
-      a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
-      a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
-      if constexpr (!MX) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 4));   // SINT4: 64 values = 8 lanes; MXINT4: 32 = 4 lanes
-      if (k0 < p.Kpad) {
-        uint32_t w0 = 0, w1 = 0, b0 = 0, b1 = 0;
-        if (k0 < p.K) {
-          __half s16;
-          unsigned short sbits;
-          float s;
-          int mx_e = -127;
-          if constexpr (MX) {
-            // 2^e with e the smallest integer such that 7 * 2^e >= a: a = 1.f * 2^E, e = E - 2 if 1.f <= 1.75 else E - 1
-            const uint32_t ab = __float_as_uint(a);
-            if (a > 0.f) mx_e = (int)(ab >> 23) - 127 - (((ab & 0x7FFFFFu) <= 0x600000u) ? 2 : 1);
-            s = __uint_as_float((uint32_t)(mx_e + 127) << 23);                  // a == 0: 2^-127 is never used (codes are 0)
-            if (a == 0.f) s = 1.0f;
-            sbits = 0x3C00; s16 = __ushort_as_half(sbits);                       // not a subnormal-scale case
-          } else {
-            s16 = __float2half_rn(__fmul_rn(a, 0.142857149243354797f));          // fl32(1/7)
-            sbits = __half_as_ushort(s16);
-            if (sbits == 0) s16 = __ushort_as_half((unsigned short)1);           // floor 2^-24
-            s = __half2float(s16);
-          }
-          const __half2* h2 = reinterpret_cast<const __half2*>(&vc);
-          float x[8], q[8], t[8];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float2 f = __half22float2(h2[i]);
-            x[2 * i] = f.x; x[2 * i + 1] = f.y;
-          }
-          // MXINT4: 1/s = 2^-e is exact, so x * (1/s) is exact and the magic-number rounding is already the definition's
-          const float inv = MX ? __uint_as_float((uint32_t)(127 - (a > 0.f ? mx_e : 0)) << 23) : rcp_fast(s), hs = 0.5f * s;
-          bool exact = sbits < 0x0400;          // subnormal scale: quotient may exceed 7, use the plain definition
-          bool near = false;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            q[i] = __fadd_rn(__fmaf_rn(x[i], inv, MAGIC), -MAGIC);
-            const float e = __fmaf_rn(-q[i], s, x[i]);
-            exact |= (fabsf(e) == hs);
-            t[i] = __fmaf_rn(x[i], invb, MAGIC);                    // low byte of the bit pattern = branch code
-            const float eb = __fmaf_rn(-__fadd_rn(t[i], -MAGIC), sb, x[i]);
-            near |= !(fabsf(eb) < thr);
-          }
-          if constexpr (MX) exact = false;
-          if (exact) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) q[i] = fminf(fmaxf(rintf(__fdiv_rn(x[i], s)), -7.f), 7.f);
-          }
-          if (near) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) t[i] = __fadd_rn(fminf(fmaxf(rintf(__fdiv_rn(x[i], sb)), -qm), qm), MAGIC);
-          }
-          w0 = f32x2_to_e4m3x2(q[1], q[0]) | (f32x2_to_e4m3x2(q[3], q[2]) << 16);
-          w1 = f32x2_to_e4m3x2(q[5], q[4]) | (f32x2_to_e4m3x2(q[7], q[6]) << 16);
-          b0 = __byte_perm(__byte_perm(__float_as_uint(t[0]), __float_as_uint(t[1]), 0x0040),
-                           __byte_perm(__float_as_uint(t[2]), __float_as_uint(t[3]), 0x0040), 0x5410);
-          b1 = __byte_perm(__byte_perm(__float_as_uint(t[4]), __float_as_uint(t[5]), 0x0040),
-                           __byte_perm(__float_as_uint(t[6]), __float_as_uint(t[7]), 0x0040), 0x5410);
-          *reinterpret_cast<uint2*>(p.qx8 + (size_t)m * p.Kpad + k0) = make_uint2(w0, w1);
-          if constexpr (MX) {
-            if ((lane & 3) == 0)
-              p.sfa[((size_t)(m >> 7) * (p.Kpad >> 7) + (k0 >> 7)) * 512 + 16 * (m & 31) + 4 * ((m & 127) >> 5) + ((k0 >> 5) & 3)] =
-                  (uint8_t)(mx_e + 127);
-          } else {
-            if ((lane & 7) == 0) sx_s[(k0 >> 6) * ROWS + rl] = s;
-          }
-          if (p.qb != nullptr && p.branch_qmax > 0) *reinterpret_cast<uint2*>(p.qb + (size_t)m * p.Kpad + k0) = make_uint2(b0, b1);
-        }
-        if (p.branch_qmax > 0) *reinterpret_cast<uint2*>(qb_s + rl * qb_stride + k0) = make_uint2(b0, b1);
-      }
-    }
-  }
-  __syncthreads();
-
-  // group scales, transposed: [g][m0 .. m0+15] are 64-byte segments
-  for (int i = threadIdx.x; !MX && i < p.G * ROWS; i += WARPS * 32) {
-    const int g = i / ROWS, rl = i % ROWS;
-    if (m0 + rl < p.M) p.sx[(size_t)g * p.Mpad + m0 + rl] = sx_s[g * ROWS + rl];
-  }
-  if (p.branch_qmax <= 0) return;
-
-  // ------------------------------------------------------------------ a3: I1 = qb L1q on mma.sync
-  const int ksteps = p.Kpad / 32, ntiles = p.rpad / 8;
-  const int gid = lane >> 2, tig = lane & 3;
-  for (int nt0 = 0; nt0 < ntiles; nt0 += 4) {
-    int acc[4][4];
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-      for (int b = 0; b < 4; ++b) acc[a][b] = 0;
-    for (int ks = warp; ks < ksteps; ks += WARPS) {
-      uint32_t a[4];
-      const uint8_t* ab = qb_s + ks * 32 + tig * 4;
-      a[0] = *reinterpret_cast<const uint32_t*>(ab + gid * qb_stride);
-      a[1] = *reinterpret_cast<const uint32_t*>(ab + (gid + 8) * qb_stride);
-      a[2] = *reinterpret_cast<const uint32_t*>(ab + gid * qb_stride + 16);
-      a[3] = *reinterpret_cast<const uint32_t*>(ab + (gid + 8) * qb_stride + 16);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        if (nt0 + j < ntiles) {
-          const uint2 b = __ldg(p.L1f + ((size_t)ks * ntiles + nt0 + j) * 32 + lane);
-          mma_s8_16832(acc[j], a, b.x, b.y);
-        }
-      }
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (nt0 + j < ntiles) {
-        const int col = (nt0 + j) * 8 + tig * 2;
-        atomicAdd(&I1_s[gid * p.rpad + col], acc[j][0]);
-        atomicAdd(&I1_s[gid * p.rpad + col + 1], acc[j][1]);
-        atomicAdd(&I1_s[(gid + 8) * p.rpad + col], acc[j][2]);
-        atomicAdd(&I1_s[(gid + 8) * p.rpad + col + 1], acc[j][3]);
-      }
-    }
-  }
-  __syncthreads();
-
-  // ------------------------------------------------------------------ a4: re-quantize the rank-r row
-  for (int rr = 0; rr < RPW; ++rr) {
-    const int rl = warp * RPW + rr, m = m0 + rl;
-    if (m >= p.M) continue;
-    const float sb = sXb_s[rl];
-    float t[4], amax = 0.f;
-#pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-      const int j = lane + 32 * jj;
-      t[jj] = 0.f;
-      if (j < p.r) {
-        t[jj] = __fmul_rn(__int2float_rn(I1_s[rl * p.rpad + j]), __fmul_rn(sb, p.sL1[j]));
-        amax = fmaxf(amax, fabsf(t[jj]));
-      }
-    }
-    amax = warp_max(amax);
-    const float st = (amax == 0.f) ? 1.0f : __fdiv_rn(amax, qm);
-    if (lane == 0) p.sT[m] = st;
-#pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-      const int j = lane + 32 * jj;
-      if (j < p.r) {
-        float q = rintf(__fdiv_rn(t[jj], st));
-        q = fminf(fmaxf(q, -qm), qm);
-        p.tq[(size_t)m * LQ_RCONT + j] = (uint8_t)(int8_t)(int)q;
-      }
-    }
-  }
-}
-
-// W16A16 reference branch: T = X L1 accumulated in fp32, rounded once to fp16; no scales.
-// A CTA of four warps owns 16 rows; the warps split K in chunks of 32 (chunk c goes to warp c % 4), multiply with
-// mma.sync m16n8k16 (fp16 x fp16 -> fp32) and add their partial sums in shared memory.  Both operands are fetched with
-// 16-byte loads: lane (g, t) holds elements 8t .. 8t+7 of the chunk for row g (A) or factor column g (B).  A sum over k does
-// not care which k sits in which fragment slot as long as A and B agree, so the lane's first four elements feed one k16 step
-// and its last four the next - no shuffles, and X is read once with full sectors.
-__device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                              uint32_t b1) {
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-template <int NT>   // NT: 8-column tiles of the rank (rank <= 8 NT)
-__global__ void __launch_bounds__(128) lq_down_f16_kernel(const __half* __restrict__ X, const __half* __restrict__ L1h,
-                                                          int M, int K, int Kpad, int r, uint8_t* __restrict__ tq,
-                                                          float* __restrict__ sT) {
-  __shared__ float part[4][16][NT * 8 + 1];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-  const int m0 = blockIdx.x * 16;
-  const int r_lo = m0 + g, r_hi = m0 + g + 8;
-  float acc[NT][4];
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) acc[nt][i] = 0.f;
-  const uint4 zero = make_uint4(0, 0, 0, 0);
-  const int chunks = (K + 31) / 32;
-#pragma unroll 3
-  for (int c = warp; c < chunks; c += 4) {
-    const int k = c * 32 + 8 * t;
-    const bool kin = k < K;                                                        // K is a multiple of 8
-    const uint4 alo = (kin && r_lo < M) ? __ldg(reinterpret_cast<const uint4*>(X + (size_t)r_lo * K + k)) : zero;
-    const uint4 ahi = (kin && r_hi < M) ? __ldg(reinterpret_cast<const uint4*>(X + (size_t)r_hi * K + k)) : zero;
-    uint4 b[NT];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const int j = nt * 8 + g;
-      b[nt] = (j < r) ? __ldg(reinterpret_cast<const uint4*>(L1h + (size_t)j * Kpad + k)) : zero;   // zero-padded up to Kpad
-    }
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      mma_f16_16816(acc[nt], alo.x, ahi.x, alo.y, ahi.y, b[nt].x, b[nt].y);
-      mma_f16_16816(acc[nt], alo.z, ahi.z, alo.w, ahi.w, b[nt].z, b[nt].w);
-    }
-  }
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    part[warp][g][nt * 8 + 2 * t] = acc[nt][0];
-    part[warp][g][nt * 8 + 2 * t + 1] = acc[nt][1];
-    part[warp][g + 8][nt * 8 + 2 * t] = acc[nt][2];
-    part[warp][g + 8][nt * 8 + 2 * t + 1] = acc[nt][3];
-  }
-  __syncthreads();
-  for (int i = threadIdx.x; i < 16 * NT * 8; i += 128) {
-    const int row = i / (NT * 8), j = i % (NT * 8);
-    const int m = m0 + row;
-    if (m < M && j < r) {
-      const float v = (part[0][row][j] + part[1][row][j]) + (part[2][row][j] + part[3][row][j]);
-      reinterpret_cast<__half*>(tq + (size_t)m * LQ_RCONT)[j] = __float2half_rn(v);
-    }
-  }
-  if (threadIdx.x < 16 && m0 + threadIdx.x < M) sT[m0 + threadIdx.x] = 1.0f;
+// largest magnitude of 16 halves (two 16-byte vectors), exact in fp16
+__device__ __forceinline__ __half absmax16(const uint4& a, const uint4& b) {
+  const __half2* p = reinterpret_cast<const __half2*>(&a);
+  const __half2* q = reinterpret_cast<const __half2*>(&b);
+  __half2 m = __hmax2(__hmax2(__habs2(p[0]), __habs2(p[1])), __hmax2(__habs2(p[2]), __habs2(p[3])));
+  m = __hmax2(m, __hmax2(__hmax2(__habs2(q[0]), __habs2(q[1])), __hmax2(__habs2(q[2]), __habs2(q[3]))));
+  return __hmax(__low2half(m), __high2half(m));
 }
 
-template <int NCHUNK, int WARPS, bool RELOAD, bool MX>
-cudaError_t launch_quant(const QuantParams& p, size_t smem, cudaStream_t st) {
+// Correctly rounded quotient a / b in binary32 from the correctly rounded reciprocal y = fl32(1/b), division free:
+// q0 = fl32(a y) is within one ulp of a / b, r = a - b q0 is exact in an FMA, and fl32(q0 + r y) is then the
+// correctly rounded quotient (Markstein's correction step).  Operands here are far from overflow and underflow.
+__device__ __forceinline__ float div_rn_by(float a, float b, float y) {
+  const float q0 = __fmul_rn(a, y);
+  const float r = __fmaf_rn(-q0, b, a);
+  return __fmaf_rn(r, y, q0);
+}
+
+// Scale of one group for a1.  `a` is the maximum magnitude of the whole group (SINT4: 64 values, MXINT4: 32),
+// already reduced over the lanes that share it.
+struct MainScale {
+  float s;       // SINT4: the fp16 scale as a float
+  float inv;     // fl32(1/s) (MXINT4: 2^-e, exact)
+  int e;         // MXINT4: block exponent
+  bool coarse;   // SINT4: subnormal scale, the quotient may exceed 7.5 and has to be clamped
+};
+template <bool MX>
+__device__ __forceinline__ MainScale main_scale(float a) {
+  MainScale m;
+  if constexpr (MX) {
+    // 2^e with e the smallest integer such that 7 * 2^e >= a: a = 1.f * 2^E, e = E - 2 if 1.f <= 1.75 else E - 1
+    const uint32_t ab = __float_as_uint(a);
+    m.e = -127;
+    if (a > 0.f) m.e = (int)(ab >> 23) - 127 - (((ab & 0x7FFFFFu) <= 0x600000u) ? 2 : 1);
+    m.inv = __uint_as_float((uint32_t)(127 - (a > 0.f ? m.e : 0)) << 23);
+    m.s = 0.f;
+    m.coarse = false;
+  } else {
+    __half s16 = __float2half_rn(__fmul_rn(a, 0.142857149243354797f));   // fl32(1/7)
+    const unsigned short sbits = __half_as_ushort(s16);
+    if (sbits == 0) s16 = __ushort_as_half((unsigned short)1);            // floor 2^-24
+    m.s = __half2float(s16);
+    m.inv = __frcp_rn(m.s);
+    m.coarse = sbits < 0x0400;
+    m.e = 0;
+  }
+  return m;
+}
+
+// a1 and a2 for eight consecutive values of one row (one 16-byte vector of halves).
+//   main    SINT4: the correctly rounded quotient x / s, then round-to-nearest-even by the magic constant - the
+//           definition itself; |x| / s <= 7 (1 + 2^-11) for a normal fp16 scale, so only a subnormal (coarse) scale
+//           needs the clamp.  MXINT4: 1/s is a power of two, x * (1/s) is exact.
+//   branch  int8 codes under the row's scale sb, invb = fl32(1/sb); |x| / sb <= qm (1 + 2^-23), so the rounded quotient
+//           never leaves [-qm, qm].  The low byte of (code + MAGIC)'s bit pattern is the code.
+// Returns the 8 operand bytes of the main codes (E4M3 images) and the 8 branch code bytes.
+template <bool MX, bool BRANCH>
+__device__ __forceinline__ void quant8(const uint4& v, const MainScale& ms, float sb, float invb, uint2& w, uint2& b) {
+  const __half2* h2 = reinterpret_cast<const __half2*>(&v);
+  float x[8], q[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __half22float2(h2[i]);
+    x[2 * i] = f.x; x[2 * i + 1] = f.y;
+  }
+  if constexpr (MX) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) q[i] = __fadd_rn(__fmaf_rn(x[i], ms.inv, MAGIC), -MAGIC);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) q[i] = __fadd_rn(__fadd_rn(div_rn_by(x[i], ms.s, ms.inv), MAGIC), -MAGIC);
+    if (ms.coarse) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) q[i] = fminf(fmaxf(q[i], -7.f), 7.f);
+    }
+  }
+  w.x = f32x2_to_e4m3x2(q[1], q[0]) | (f32x2_to_e4m3x2(q[3], q[2]) << 16);
+  w.y = f32x2_to_e4m3x2(q[5], q[4]) | (f32x2_to_e4m3x2(q[7], q[6]) << 16);
+  if constexpr (BRANCH) {
+    uint32_t t[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) t[i] = __float_as_uint(__fadd_rn(div_rn_by(x[i], sb, invb), MAGIC));
+    b.x = __byte_perm(__byte_perm(t[0], t[1], 0x0040), __byte_perm(t[2], t[3], 0x0040), 0x5410);
+    b.y = __byte_perm(__byte_perm(t[4], t[5], 0x0040), __byte_perm(t[6], t[7], 0x0040), 0x5410);
+  }
+}
+
+// CTA-wide rendezvous of the consumer warps on an mbarrier (count = number of consumer warps), bounded like every wait
+__device__ __forceinline__ bool consumers_sync(uint32_t bar, uint32_t parity, int lane, volatile int* abort_flag,
+                                               int32_t* status) {
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar);
+  return mbar_wait(bar, parity, abort_flag, status, LQ_STAGE_QUANT);
+}
+
+// Shared memory (dynamic), from a 1024-byte aligned base:
+//   ring      W x D boxes of 2 KB
+//   bars      full[W D], empty[W D], syncA, syncB, syncC
+//   red       BR_INT: int I1[2][16][rpad]; BR_F16: float part[W][16][rpad]
+//   rowmax    int[2][16] (bit patterns of non-negative floats)
+//   abort     int
+template <bool MX, int BR, int NTR>   // NTR: 8-column tiles of the rank (rank <= 8 NTR)
+__global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_kernel(const __grid_constant__ CUtensorMap tmX,
+                                                                                 const QuantParams p) {
+  extern __shared__ uint8_t qsm_raw[];
+  const uint32_t base = (smem_u32(qsm_raw) + 1023u) & ~1023u;
+  uint8_t* smem = qsm_raw + (base - smem_u32(qsm_raw));
+  const int W = (int)(blockDim.x >> 5) - 1;                 // consumer warps; warp W is the producer
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
+  const int lane = threadIdx.x & 31;
+  const int gid = lane >> 2, tig = lane & 3;
+  const int nslot = W * p.depth;
+  const uint32_t ring = base;
+  const uint32_t bars = base + (uint32_t)nslot * BOX_BYTES;
+  auto bar_full = [&](int s) { return bars + 8u * (uint32_t)s; };
+  auto bar_empty = [&](int s) { return bars + 8u * (uint32_t)(nslot + s); };
+  const uint32_t bar_sync = bars + 16u * (uint32_t)nslot;   // three rendezvous barriers
+  uint8_t* red_ptr = smem + (size_t)nslot * BOX_BYTES + 16 * (size_t)nslot + 32;
+  int* I1_s = reinterpret_cast<int*>(red_ptr);
+  float* part_s = reinterpret_cast<float*>(red_ptr);
+  const size_t red_bytes = BR == BR_INT ? (size_t)2 * TR * p.rpad * 4 : BR == BR_F16 ? (size_t)W * TR * p.rpad * 4 : 0;
+  int* rowmax_s = reinterpret_cast<int*>(red_ptr + red_bytes);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(rowmax_s + 2 * TR);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < nslot; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+    for (int b = 0; b < 3; ++b) mbar_init(bar_sync + 8u * b, (uint32_t)W);
+    *abort_flag = 0;
+    mbar_init_fence();
+  }
+  if constexpr (BR == BR_INT) {
+    for (int i = threadIdx.x; i < 2 * TR * p.rpad; i += blockDim.x) I1_s[i] = 0;
+    if (threadIdx.x < 2 * TR) rowmax_s[threadIdx.x] = 0;
+  }
+  __syncthreads();
+
+  const int passes = (BR == BR_INT && p.refetch) ? 2 : 1;   // how often the producer streams a tile
+
+  if (warp == W) {
+    // ------------------------------------------------------------------ TMA producer: lane w feeds consumer warp w
+    if (lane < W) {
+      const int s0 = lane * p.depth;
+      int idx = 0;
+      uint32_t phase = 0, issued = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.ntiles && ok; tile += gridDim.x) {
+        const int m0 = tile * TR;
+        for (int ps = 0; ps < passes && ok; ++ps) {
+          for (int g = lane; g < p.nbox; g += W) {
+            ok = mbar_wait(bar_empty(s0 + idx), phase ^ 1, abort_flag, p.status, LQ_STAGE_PRODUCER);
+            if (!ok) break;
+            mbar_expect_tx(bar_full(s0 + idx), BOX_BYTES);
+            tma_load_2d(ring + (uint32_t)(s0 + idx) * BOX_BYTES, &tmX, g * BOX_K, m0, bar_full(s0 + idx));
+            ++issued;
+            if (++idx == p.depth) { idx = 0; phase ^= 1; }
+          }
+        }
+      }
+      if (!ok) {
+        // aborting: let the copies already issued land before the CTA's shared memory goes away
+        const uint32_t n = issued < (uint32_t)p.depth ? issued : (uint32_t)p.depth;
+        for (uint32_t i = 0; i < n; ++i) {
+          if (--idx < 0) { idx = p.depth - 1; phase ^= 1; }
+          mbar_settle(bar_full(s0 + idx), phase);
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers
+    // box sequence of this warp: boxes w, w + W, ... of every pass of every tile, through its own ring
+    const int s0 = warp * p.depth;
+    int idx = 0;
+    uint32_t phase = 0;
+    auto advance = [&]() {
+      if (++idx == p.depth) { idx = 0; phase ^= 1; }
+    };
+    // this lane's two 16-byte chunks of a swizzled 128-byte row; rows gid and gid + 8 share the swizzle phase
+    const uint32_t row_off = (uint32_t)gid * 128u;
+    const uint32_t c0 = (uint32_t)((2 * tig) ^ (gid & 7)) << 4, c1 = (uint32_t)((2 * tig + 1) ^ (gid & 7)) << 4;
+    uint32_t sync_par = 0;
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < p.ntiles && ok; tile += gridDim.x, ++tcount) {
+      const int m0 = tile * TR;
+      const int par = (int)(tcount & 1);
+      const int m_lo = m0 + gid, m_hi = m0 + gid + 8;
+      const bool v_lo = m_lo < p.M, v_hi = m_hi < p.M;
+      uint8_t* const qx_lo = p.qx8 + (size_t)m_lo * p.Kpad + 16 * tig;   // this lane's bytes of a row start here
+      uint8_t* const qx_hi = qx_lo + (size_t)8 * p.Kpad;
+      float sb_lo = 1.f, sb_hi = 1.f, invb_lo = 1.f, invb_hi = 1.f;
+      // ---- walk 1 (integer branch only): the rows' maxima
+      if constexpr (BR == BR_INT) {
+        const int idx0 = idx;
+        const uint32_t phase0 = phase;
+        __half2 hm = __float2half2_rn(0.f);                 // (row gid, row gid + 8)
+        for (int g = warp; g < p.nbox; g += W) {
+          ok = mbar_wait(bar_full(s0 + idx), phase, abort_flag, p.status, LQ_STAGE_QUANT);
+          if (!ok) break;
+          const uint8_t* bx = smem + (size_t)(s0 + idx) * BOX_BYTES + row_off;
+          const uint4 l0 = *reinterpret_cast<const uint4*>(bx + c0), l1 = *reinterpret_cast<const uint4*>(bx + c1);
+          const uint4 h0 = *reinterpret_cast<const uint4*>(bx + 1024 + c0), h1 = *reinterpret_cast<const uint4*>(bx + 1024 + c1);
+          hm = __hmax2(hm, __halves2half2(absmax16(l0, l1), absmax16(h0, h1)));
+          if (p.refetch) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty(s0 + idx));
+          }
+          advance();
+        }
+        if (!ok) break;
+        if (!p.refetch) { idx = idx0; phase = phase0; }     // the second walk reads the same slots
+        hm = __hmax2(hm, __shfl_xor_sync(0xffffffffu, hm, 1));
+        hm = __hmax2(hm, __shfl_xor_sync(0xffffffffu, hm, 2));
+        if (tig == 0) {
+          atomicMax(&rowmax_s[par * TR + gid], __float_as_int(__low2float(hm)));
+          atomicMax(&rowmax_s[par * TR + gid + 8], __float_as_int(__high2float(hm)));
+        }
+        ok = consumers_sync(bar_sync, sync_par, lane, abort_flag, p.status);
+        if (!ok) break;
+        if (threadIdx.x < TR) rowmax_s[(par ^ 1) * TR + threadIdx.x] = 0;     // the other buffer: next tile's
+        const float rm_lo = __int_as_float(rowmax_s[par * TR + gid]), rm_hi = __int_as_float(rowmax_s[par * TR + gid + 8]);
+        sb_lo = (rm_lo == 0.f) ? 1.0f : __fdiv_rn(rm_lo, p.qm);
+        sb_hi = (rm_hi == 0.f) ? 1.0f : __fdiv_rn(rm_hi, p.qm);
+        invb_lo = __frcp_rn(sb_lo); invb_hi = __frcp_rn(sb_hi);
+        if (warp == 0 && tig == 0) {
+          if (v_lo) p.sXb[m_lo] = sb_lo;
+          if (v_hi) p.sXb[m_hi] = sb_hi;
+        }
+      }
+      // ---- walk 2: codes, scales, down-projection
+      int acci[BR == BR_INT ? NTR : 1][4];
+      float accf[BR == BR_F16 ? NTR : 1][4];
+#pragma unroll
+      for (int a = 0; a < NTR; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          if constexpr (BR == BR_INT) acci[a][b] = 0;
+          if constexpr (BR == BR_F16) accf[a][b] = 0.f;
+        }
+      {
+        // First-factor fragments (read-only, shared by all CTAs, L2 resident) travel one box ahead of their use: the
+        // load of box g + W is in flight while box g is quantized.  FRAGV: 16-byte vectors per lane and column tile.
+        constexpr int FRAGV = BR == BR_F16 ? 2 : 1;
+        uint4 bfrag[BR == BR_NONE ? 1 : NTR * FRAGV];
+        auto load_frags = [&](int g) {
+          if constexpr (BR != BR_NONE) {
+            const uint4* src = p.L1f + ((size_t)g * NTR * 32 + lane) * FRAGV;
+#pragma unroll
+            for (int i = 0; i < NTR * FRAGV; ++i) bfrag[i] = __ldg(src + (size_t)(i / FRAGV) * 32 * FRAGV + (i % FRAGV));
+          }
+        };
+        if (warp < p.nbox) load_frags(warp);
+        for (int g = warp; g < p.nbox; g += W) {
+          ok = mbar_wait(bar_full(s0 + idx), phase, abort_flag, p.status, LQ_STAGE_QUANT);
+          if (!ok) break;
+          const uint8_t* bx = smem + (size_t)(s0 + idx) * BOX_BYTES + row_off;
+          const uint4 l0 = *reinterpret_cast<const uint4*>(bx + c0), l1 = *reinterpret_cast<const uint4*>(bx + c1);
+          const uint4 h0 = *reinterpret_cast<const uint4*>(bx + 1024 + c0), h1 = *reinterpret_cast<const uint4*>(bx + 1024 + c1);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_empty(s0 + idx));   // the values are in registers: the slot may be refilled
+          advance();
+          const size_t koff = (size_t)(g * BOX_K);             // this box's first value of a row
+          uint4 w_lo, w_hi, b_lo = make_uint4(0, 0, 0, 0), b_hi = make_uint4(0, 0, 0, 0);
+          // group maxima: 64 values = four lanes (SINT4), 32 values = two lanes (MXINT4)
+          float a_lo = __half2float(absmax16(l0, l1)), a_hi = __half2float(absmax16(h0, h1));
+          a_lo = fmaxf(a_lo, __shfl_xor_sync(0xffffffffu, a_lo, 1));
+          a_hi = fmaxf(a_hi, __shfl_xor_sync(0xffffffffu, a_hi, 1));
+          if constexpr (!MX) {
+            a_lo = fmaxf(a_lo, __shfl_xor_sync(0xffffffffu, a_lo, 2));
+            a_hi = fmaxf(a_hi, __shfl_xor_sync(0xffffffffu, a_hi, 2));
+          }
+          const MainScale ms_lo = main_scale<MX>(a_lo), ms_hi = main_scale<MX>(a_hi);
+          {
+            uint2 w, b;
+            quant8<MX, BR == BR_INT>(l0, ms_lo, sb_lo, invb_lo, w, b);
+            w_lo.x = w.x; w_lo.y = w.y; b_lo.x = b.x; b_lo.y = b.y;
+            quant8<MX, BR == BR_INT>(l1, ms_lo, sb_lo, invb_lo, w, b);
+            w_lo.z = w.x; w_lo.w = w.y; b_lo.z = b.x; b_lo.w = b.y;
+          }
+          {
+            uint2 w, b;
+            quant8<MX, BR == BR_INT>(h0, ms_hi, sb_hi, invb_hi, w, b);
+            w_hi.x = w.x; w_hi.y = w.y; b_hi.x = b.x; b_hi.y = b.y;
+            quant8<MX, BR == BR_INT>(h1, ms_hi, sb_hi, invb_hi, w, b);
+            w_hi.z = w.x; w_hi.w = w.y; b_hi.z = b.x; b_hi.w = b.y;
+          }
+          const float s_lo = ms_lo.s, s_hi = ms_hi.s;
+          const int e_lo = ms_lo.e, e_hi = ms_hi.e;
+          // stores: 16 operand bytes per row and lane (64 contiguous bytes per row and box)
+          if (v_lo) {
+            *reinterpret_cast<uint4*>(qx_lo + koff) = w_lo;
+            if (BR == BR_INT && p.qb != nullptr) *reinterpret_cast<uint4*>(p.qb + (qx_lo - p.qx8) + koff) = b_lo;
+          }
+          if (v_hi) {
+            *reinterpret_cast<uint4*>(qx_hi + koff) = w_hi;
+            if (BR == BR_INT && p.qb != nullptr) *reinterpret_cast<uint4*>(p.qb + (qx_hi - p.qx8) + koff) = b_hi;
+          }
+          if constexpr (MX) {
+            const int kb = 2 * g + (tig >> 1);               // block of 32 along K
+            if ((tig & 1) == 0 && kb < p.G) {
+              if (v_lo)
+                p.sfa[((size_t)(m_lo >> 7) * (p.Kpad >> 7) + (kb >> 2)) * 512 + 16 * (m_lo & 31) + 4 * ((m_lo & 127) >> 5) + (kb & 3)] =
+                    (uint8_t)(e_lo + 127);
+              if (v_hi)
+                p.sfa[((size_t)(m_hi >> 7) * (p.Kpad >> 7) + (kb >> 2)) * 512 + 16 * (m_hi & 31) + 4 * ((m_hi & 127) >> 5) + (kb & 3)] =
+                    (uint8_t)(e_hi + 127);
+            }
+          } else {
+            if (tig == 0 && g < p.G) {
+              if (v_lo) p.sx[(size_t)g * p.Mpad + m_lo] = s_lo;
+              if (v_hi) p.sx[(size_t)g * p.Mpad + m_hi] = s_hi;
+            }
+          }
+          // a3 on the fragments just made: bytes 8j .. 8j+7 of a lane's run feed MMA step j
+          if constexpr (BR == BR_INT) {
+#pragma unroll
+            for (int nt = 0; nt < NTR; ++nt) {
+              mma_s8_16832(acci[nt], b_lo.x, b_hi.x, b_lo.y, b_hi.y, bfrag[nt].x, bfrag[nt].y);
+              mma_s8_16832(acci[nt], b_lo.z, b_hi.z, b_lo.w, b_hi.w, bfrag[nt].z, bfrag[nt].w);
+            }
+          }
+          if constexpr (BR == BR_F16) {
+            // rows beyond M and values beyond K are zeros (TMA fill); fp16 x fp16 -> fp32, four k16 steps per box
+#pragma unroll
+            for (int nt = 0; nt < NTR; ++nt) {
+              const uint4 f0 = bfrag[2 * nt], f1 = bfrag[2 * nt + 1];
+              mma_f16_16816(accf[nt], l0.x, h0.x, l0.y, h0.y, f0.x, f0.y);
+              mma_f16_16816(accf[nt], l0.z, h0.z, l0.w, h0.w, f0.z, f0.w);
+              mma_f16_16816(accf[nt], l1.x, h1.x, l1.y, h1.y, f1.x, f1.y);
+              mma_f16_16816(accf[nt], l1.z, h1.z, l1.w, h1.w, f1.z, f1.w);
+            }
+          }
+          if (g + W < p.nbox) load_frags(g + W);
+        }
+        if (!ok) break;
+      }
+      if constexpr (BR == BR_NONE) continue;
+      // ---- the warps' partial products meet in shared memory
+      if constexpr (BR == BR_INT) {
+        int* I1 = I1_s + par * TR * p.rpad;
+#pragma unroll
+        for (int nt = 0; nt < NTR; ++nt) {
+          const int col = nt * 8 + tig * 2;
+          if (col < p.rpad) {
+            atomicAdd(&I1[gid * p.rpad + col], acci[nt][0]);
+            atomicAdd(&I1[gid * p.rpad + col + 1], acci[nt][1]);
+            atomicAdd(&I1[(gid + 8) * p.rpad + col], acci[nt][2]);
+            atomicAdd(&I1[(gid + 8) * p.rpad + col + 1], acci[nt][3]);
+          }
+        }
+      } else {
+        float* mine = part_s + (size_t)warp * TR * p.rpad;
+#pragma unroll
+        for (int nt = 0; nt < NTR; ++nt) {
+          const int col = nt * 8 + tig * 2;
+          if (col < p.rpad) {
+            *reinterpret_cast<float2*>(&mine[gid * p.rpad + col]) = make_float2(accf[nt][0], accf[nt][1]);
+            *reinterpret_cast<float2*>(&mine[(gid + 8) * p.rpad + col]) = make_float2(accf[nt][2], accf[nt][3]);
+          }
+        }
+      }
+      ok = consumers_sync(bar_sync + 8, sync_par, lane, abort_flag, p.status);
+      if (!ok) break;
+      // ---- a4: the rank-r rows of this tile, one warp per row
+      for (int rl = warp; rl < TR; rl += W) {
+        const int m = m0 + rl;
+        if constexpr (BR == BR_INT) {
+          int* I1 = I1_s + par * TR * p.rpad + rl * p.rpad;
+          const float rm = __int_as_float(rowmax_s[par * TR + rl]);
+          const float sb = (rm == 0.f) ? 1.0f : __fdiv_rn(rm, p.qm);
+          float t[4], amax = 0.f;
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) {
+            const int j = lane + 32 * jj;
+            t[jj] = 0.f;
+            if (j < p.rpad) {
+              const int v = I1[j];
+              I1[j] = 0;                                      // ready for the tile after next
+              if (j < p.r) {
+                t[jj] = __fmul_rn(__int2float_rn(v), __fmul_rn(sb, p.sL1[j]));
+                amax = fmaxf(amax, fabsf(t[jj]));
+              }
+            }
+          }
+          amax = warp_max(amax);
+          if (m < p.M) {
+            const float st = (amax == 0.f) ? 1.0f : __fdiv_rn(amax, p.qm);
+            if (lane == 0) p.sT[m] = st;
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+              const int j = lane + 32 * jj;
+              if (j < p.r) {
+                float q = rintf(__fdiv_rn(t[jj], st));
+                q = fminf(fmaxf(q, -p.qm), p.qm);
+                p.tq[(size_t)m * LQ_RCONT + j] = (uint8_t)(int8_t)(int)q;
+              }
+            }
+          }
+        } else {
+          // T = fp16(X L1): the warps' fp32 partial sums are added in warp order (the result does not depend on timing)
+          if (m < p.M) {
+            for (int j = lane; j < p.r; j += 32) {
+              float v = 0.f;
+              for (int w2 = 0; w2 < W; ++w2) v += part_s[((size_t)w2 * TR + rl) * p.rpad + j];
+              reinterpret_cast<__half*>(p.tq + (size_t)m * LQ_RCONT)[j] = __float2half_rn(v);
+            }
+            if (lane == 0) p.sT[m] = 1.0f;
+          }
+        }
+      }
+      if constexpr (BR == BR_F16) {
+        ok = consumers_sync(bar_sync + 16, sync_par, lane, abort_flag, p.status);   // partial sums may be overwritten
+        if (!ok) break;
+      }
+      sync_par ^= 1;
+    }
+  }
+}
+
+struct LaunchPlan {
+  int W, depth, refetch, ctas_per_sm;
+  size_t smem;
+};
+
+// Picks the consumer-warp count, ring depth and residency for a row length.  Budget: 227 KB of shared memory and
+// 64 K registers per SM (allocated per warp in units of 8 registers per thread).  Measured on the PixArt shapes
+// (K = 1152, 4608; all branch kinds): two CTAs per SM with eight or nine consumer warps each is the fastest or within
+// a few percent of it, so that is the default; the options "quant_ctas" / "quant_warps" override it for tuning.
+LaunchPlan plan_launch(int nbox, int br, int rpad, int regs) {
+  const size_t SM_SMEM = 227 * 1024;
+  LaunchPlan best{};
+  double best_score = -1.0;
+  for (int ctas = 4; ctas >= 1; --ctas) {
+    if (g_lq_quant_ctas > 0 ? ctas != g_lq_quant_ctas : ctas > 2) continue;
+    for (int W = 4; W <= MAX_CONSUMER_WARPS; ++W) {
+      if (g_lq_quant_warps > 0 ? W != g_lq_quant_warps : W < 8) continue;
+      const int threads = (W + 1) * 32;
+      if (ctas * threads > 2048 || ctas * threads * ((regs + 7) / 8 * 8) > 65536) continue;
+      const size_t red = br == BR_INT ? (size_t)2 * TR * rpad * 4 : br == BR_F16 ? (size_t)W * TR * rpad * 4 : 0;
+      const size_t fixed = 1024 + 64 + red + 2 * TR * 4 + 64;
+      const size_t budget = std::min(SM_SMEM, SM_SMEM / ctas - 1024);
+      if (budget < fixed + (size_t)W * (BOX_BYTES + 16)) continue;
+      const int per = (nbox + W - 1) / W;                     // boxes of a tile per warp
+      int depth = (int)((budget - fixed) / (BOX_BYTES + 16)) / W;
+      int refetch = 0;
+      if (depth > 2 * per) depth = 2 * per;
+      if (depth < per && br == BR_INT) refetch = 1;
+      // score: resident consumer warps, discounted by the imbalance of boxes over warps; more CTAs and warps win ties
+      const double balance = (double)nbox / (double)(per * W);
+      const double score = ctas * W * balance + 0.01 * ctas + 0.001 * W;
+      if (score > best_score) {
+        best_score = score;
+        best = LaunchPlan{W, depth, refetch, ctas, fixed + (size_t)W * depth * (BOX_BYTES + 16)};
+      }
+    }
+  }
+  return best;
+}
+
+template <bool MX, int BR, int NTR>
+cudaError_t launch_quant(const CUtensorMap& tm, QuantParams& p, int sms, cudaStream_t st) {
   static bool attr_set[64] = {false};
+  static int regs[64] = {0};
   int dev = 0;
   cudaGetDevice(&dev);
-  if (smem > 48 * 1024 && !attr_set[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(lq_quant_kernel<NCHUNK, WARPS, RELOAD, MX>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (!attr_set[dev & 63]) {
+    cudaError_t e = cudaFuncSetAttribute(lq_quant_kernel<MX, BR, NTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
+    cudaFuncAttributes fa;
+    if ((e = cudaFuncGetAttributes(&fa, lq_quant_kernel<MX, BR, NTR>)) != cudaSuccess) return e;
+    regs[dev & 63] = fa.numRegs;
     attr_set[dev & 63] = true;
   }
-  lq_quant_kernel<NCHUNK, WARPS, RELOAD, MX><<<lq_ceil_div(p.M, ROWS), WARPS * 32, smem, st>>>(p);
+  const LaunchPlan pl = plan_launch(p.nbox, BR, p.rpad, regs[dev & 63]);
+  if (pl.W == 0) return cudaErrorInvalidConfiguration;
+  p.depth = pl.depth; p.refetch = pl.refetch;
+  int grid = sms * pl.ctas_per_sm;
+  if (grid > p.ntiles) grid = p.ntiles;
+  lq_quant_kernel<MX, BR, NTR><<<grid, (pl.W + 1) * 32, pl.smem, st>>>(tm, p);
   return cudaGetLastError();
+}
+
+template <bool MX>
+cudaError_t dispatch_quant(int br, int ntr, const CUtensorMap& tm, QuantParams& p, int sms, cudaStream_t st) {
+  if (br == BR_NONE) return launch_quant<MX, BR_NONE, 1>(tm, p, sms, st);
+  if (br == BR_INT) {
+    if (ntr <= 2) return launch_quant<MX, BR_INT, 2>(tm, p, sms, st);
+    if (ntr <= 4) return launch_quant<MX, BR_INT, 4>(tm, p, sms, st);
+    if (ntr <= 8) return launch_quant<MX, BR_INT, 8>(tm, p, sms, st);
+    return launch_quant<MX, BR_INT, 16>(tm, p, sms, st);
+  }
+  if (ntr <= 2) return launch_quant<MX, BR_F16, 2>(tm, p, sms, st);
+  if (ntr <= 4) return launch_quant<MX, BR_F16, 4>(tm, p, sms, st);
+  return launch_quant<MX, BR_F16, 8>(tm, p, sms, st);
 }
 
 }  // namespace
 
+// rank rounded up to the kernels' instantiated widths (8-column tiles: 2, 4, 8, 16)
+int lq_quant_rank_tiles(int r, bool f16) {
+  const int nt = lq_ceil_div(r > 0 ? r : 8, 8);
+  return nt <= 2 ? 2 : nt <= 4 ? 4 : (nt <= 8 || f16) ? 8 : 16;
+}
+
 lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A, cudaStream_t st) {
   if (cudaSetDevice(A->device) != cudaSuccess) return LQ_ERR_CUDA;
-  const int K = L->K, Kpad = L->Kpad;
+  if (A->main_kind != LQ_KIND_E4M3) return LQ_ERR_UNSUPPORTED;
   const int abits = lq_branch_abits(L->cfg.branch);
+  const int br = L->f16_branch ? BR_F16 : (L->integer_branch && abits > 0) ? BR_INT : BR_NONE;
+  const int ntr = lq_quant_rank_tiles(L->r, L->f16_branch);
   QuantParams p;
-  p.X = reinterpret_cast<const uint4*>(X);
-  p.M = M; p.K = K; p.Kpad = Kpad; p.Mpad = A->Mpad; p.G = L->G;
+  p.M = M; p.K = L->K; p.Kpad = L->Kpad; p.Mpad = A->Mpad; p.G = L->G;
+  p.nbox = L->Kpad / BOX_K;
+  p.ntiles = lq_ceil_div(M, TR);
   p.qx8 = A->d_qx8; p.sx = A->d_sx; p.sfa = A->d_sfa;
   p.qb = g_lq_store_qb ? A->d_qb : nullptr;
   p.sXb = A->d_sXb;
-  p.L1f = reinterpret_cast<const uint2*>(L->d_L1f);
+  p.L1f = reinterpret_cast<const uint4*>(L->f16_branch ? (const void*)L->d_L1h : (const void*)L->d_L1f);
   p.sL1 = L->d_sL1; p.tq = A->d_tq; p.sT = A->d_sT;
-  p.r = L->r; p.rpad = lq_round_up(L->r > 0 ? L->r : 8, 8);
-  p.branch_qmax = (L->integer_branch && abits > 0) ? ((1 << (abits - 1)) - 1) : 0;
-  const size_t smem = (p.branch_qmax > 0 ? (size_t)ROWS * (Kpad + 16) : 0) + (size_t)(Kpad / LQ_GROUP) * ROWS * 4 +
-                      (size_t)ROWS * p.rpad * 4 + ROWS * 4;
-  const int nchunk = lq_ceil_div(Kpad, 256);
-  cudaError_t e;
-  if (A->main_kind != LQ_KIND_E4M3) return LQ_ERR_UNSUPPORTED;
-#define LQ_QUANT_DISPATCH(MXF)                                                                                          \
-  if (nchunk <= 2) e = launch_quant<2, 16, false, MXF>(p, smem, st);   /* the row stays in registers (one warp per row) */ \
-  else if (nchunk <= 5) e = launch_quant<5, 16, false, MXF>(p, smem, st);                                               \
-  else if (nchunk <= 9) e = launch_quant<9, 16, true, MXF>(p, smem, st);   /* longer rows: read twice, 2nd time from L2 */ \
-  else if (nchunk <= 12) e = launch_quant<12, 16, true, MXF>(p, smem, st);                                              \
-  else if (nchunk <= 18) e = launch_quant<18, 16, true, MXF>(p, smem, st);                                              \
-  else if (nchunk <= 22) e = launch_quant<22, 16, true, MXF>(p, smem, st);                                              \
-  else if (nchunk <= 32) e = launch_quant<32, 16, true, MXF>(p, smem, st);                                              \
-  else return LQ_ERR_UNSUPPORTED;
-  if (L->mx) { LQ_QUANT_DISPATCH(true) } else { LQ_QUANT_DISPATCH(false) }
-#undef LQ_QUANT_DISPATCH
-  if (lq_note_cuda(e) != cudaSuccess) return LQ_ERR_CUDA;
-  if (L->f16_branch) {
-    const __half* Xh = reinterpret_cast<const __half*>(X);
-    const __half* L1 = reinterpret_cast<const __half*>(L->d_L1h);
-    const int blocks = lq_ceil_div(M, 16);
-    if (L->r <= 16) lq_down_f16_kernel<2><<<blocks, 128, 0, st>>>(Xh, L1, M, K, Kpad, L->r, A->d_tq, A->d_sT);
-    else if (L->r <= 32) lq_down_f16_kernel<4><<<blocks, 128, 0, st>>>(Xh, L1, M, K, Kpad, L->r, A->d_tq, A->d_sT);
-    else lq_down_f16_kernel<8><<<blocks, 128, 0, st>>>(Xh, L1, M, K, Kpad, L->r, A->d_tq, A->d_sT);
-    if (cudaGetLastError() != cudaSuccess) return LQ_ERR_CUDA;
-  }
-  return LQ_OK;
+  p.r = L->r; p.rpad = ntr * 8;
+  p.qm = br == BR_INT ? (float)((1 << (abits - 1)) - 1) : 0.f;
+  p.status = lq_device_status_ptr(A->device);
+  if (!p.status) return LQ_ERR_CUDA;
+  CUtensorMap tm;
+  lq_status s = lq_make_tmap_rows16(&tm, X, (uint64_t)M, (uint64_t)L->K);
+  if (s != LQ_OK) return s;
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, A->device) != cudaSuccess) return LQ_ERR_CUDA;
+  const cudaError_t e = L->mx ? dispatch_quant<true>(br, ntr, tm, p, sms, st) : dispatch_quant<false>(br, ntr, tm, p, sms, st);
+  return lq_note_cuda(e) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
 }

@@ -1,5 +1,7 @@
-"""Host-side checks of the arithmetic identities the CUDA quantizer's division-free fast path
-relies on, against the oracle's plain definition (Appendix A.3: SINT4, fp16 scale, RTN)."""
+"""Host-side checks of the arithmetic identities the CUDA quantizer's division-free arithmetic
+relies on, against the plain definition (Appendix A.3: SINT4, fp16 scale, RTN)."""
+from fractions import Fraction
+
 import numpy as np
 
 from oracle import lq_oracle as O
@@ -16,21 +18,50 @@ def test_scale_by_reciprocal_equals_division_for_every_fp16_maximum():
     assert np.array_equal(s_def[:, 0].view(np.uint16), s_fast.view(np.uint16))
 
 
-def test_exact_remainder_flags_exactly_the_ties():
-    """Main-branch fast path: q' = rint(x * r) with r ~ 1/s, remainder e = x - q' s; the code is
-    q' unless |e| == s/2.  Emulated in fl32 on random fp16 rows plus planted ties; the flagged
-    elements re-done with true division must give the oracle's codes everywhere."""
+def _rn32(v: Fraction) -> Fraction:
+    """v rounded to the nearest binary32 number, ties to even (normal range), in exact rational arithmetic."""
+    if v == 0:
+        return Fraction(0)
+    sign, a = (-1 if v < 0 else 1), abs(v)
+    e = a.numerator.bit_length() - a.denominator.bit_length() - 23
+    while a / Fraction(2) ** e >= 2 ** 24:
+        e += 1
+    while a / Fraction(2) ** e < 2 ** 23:
+        e -= 1
+    t = a / Fraction(2) ** e
+    n = t.numerator // t.denominator
+    rem = t - n
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and n % 2 == 1):
+        n += 1
+    return sign * n * Fraction(2) ** e
+
+
+def test_fma_corrected_quotient_is_the_correctly_rounded_division():
+    """The kernel never divides: with y = fl32(1/b) it forms q0 = fl32(a y), r = a - b q0 (exact in an FMA) and
+    q1 = fl32(q0 + r y).  q1 must be fl32(a / b), the definition's quotient (Appendix A.3: RTN of the scaled value),
+    for fp16 numerators over fp16 scales (main branch) and over fp32 per-token scales (low-rank branch), including
+    quotients that sit exactly on k + 1/2.  Everything here is exact rational arithmetic."""
     rng = np.random.default_rng(0)
-    X = rng.standard_normal((64, 1024)).astype(np.float16)
-    X[:8] = (rng.integers(-14, 15, size=(8, 1024)) * 0.5).astype(np.float16); X[:8, ::64] = 7   # ties k + 1/2, s = 1
-    codes, scales = O.qgrp(X.astype(np.float32))
-    s = np.repeat(scales.astype(np.float32), 64, axis=1)
-    x = X.astype(np.float32)
-    r = (np.float32(1.0) / s).astype(np.float32) * np.float32(1.0 + 2.0 ** -22)          # a reciprocal 2 ulp off
-    q = np.rint((x * r).astype(np.float32)).astype(np.float32)
-    e = (x.astype(np.float64) - q.astype(np.float64) * s.astype(np.float64)).astype(np.float32)  # exact in fl32
-    tie = np.abs(e) == np.float32(0.5) * s
-    q_exact = np.clip(np.rint(x / s), -7, 7)
-    q = np.where(tie, q_exact, q)
-    assert tie.any()
-    assert np.array_equal(q.astype(np.int8), codes)
+    cases = []
+    x16 = rng.standard_normal(6000).astype(np.float16)
+    s16 = (np.abs(rng.standard_normal(6000)) * 0.3 + 2.0 ** -10).astype(np.float16)
+    cases += [(Fraction(float(a)), Fraction(float(b))) for a, b in zip(x16, s16)]
+    for k in range(0, 8):                                    # exact ties x = (k + 1/2) s
+        for b in s16[:60]:
+            a = np.float16((k + 0.5) * float(b))
+            cases.append((Fraction(float(a)), Fraction(float(b))))
+    xb = (rng.standard_normal(6000) * 3).astype(np.float16)
+    rowmax = np.abs(xb).max()
+    for qm in (127.0, 31.0, 7.0):
+        sb = np.float32(np.float32(rowmax) / np.float32(qm))
+        cases += [(Fraction(float(a)), Fraction(float(sb))) for a in xb[:2000]]
+    ties = 0
+    for a, b in cases:
+        y = _rn32(1 / b)
+        q0 = _rn32(a * y)
+        r = a - b * q0
+        assert _rn32(r) == r, "the remainder must be a binary32 number (exact FMA)"
+        q1 = _rn32(q0 + r * y)
+        assert q1 == _rn32(a / b), (float(a), float(b))
+        ties += (2 * a / b).denominator == 1 and (a / b).denominator == 2
+    assert ties > 100
