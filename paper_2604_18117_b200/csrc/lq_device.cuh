@@ -38,6 +38,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// Non-blocking poll: mbarrier.try_wait may suspend the thread for a system-defined time when the phase is still
+// open, test_wait never does.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
 // Bounded wait.  Returns false when the CTA is aborting or the deadline passed (then it raises the abort flag
 // and records who gave up in the device status word {code, stage}).
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
@@ -205,5 +219,34 @@ constexpr uint32_t IDESC_F16 = (1u << 4) | (0u << 7) | (0u << 10);   // F16 x F1
 __device__ __forceinline__ constexpr uint32_t idesc_mx(int n, int sf_id) {
   return ((uint32_t)sf_id << 4) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(LQ_BM >> 4) << 24) | ((uint32_t)sf_id << 29);
 }
+
+// ---- timeline build (-DLQ_TIMELINE): per-role clock stamps of CTA 0 ----------------------
+// A stamp is one 8-byte store by lane 0 of the stamping warp: (event id << 48) | (tag << 40) | (clock64 & 2^40-1),
+// appended to that warp's list g_lq_timeline[list][...] (a zero word ends a list).  The regular build compiles
+// every LQ_TL_* macro to nothing.
+#ifdef LQ_TIMELINE
+constexpr int TL_LISTS = 4, TL_CAP = 8192;
+enum { TL_PRODUCER = 0, TL_MMA = 1, TL_DRAIN_FIRST = 2, TL_DRAIN_LAST = 3 };
+enum {
+  EV_P_SLOT_FREE = 1, EV_P_ISSUED = 2,                          // producer: stage free / copies issued
+  EV_M_STAGE_FULL = 3, EV_M_ACC_FREE = 4, EV_M_ISSUED = 5,      // MMA warp: operands landed / accumulator free / MMAs + commit issued
+  EV_D_OPEN = 6, EV_D_ACC_FULL = 7, EV_D_LOADED = 8, EV_D_DONE = 9,   // drain: starts waiting / accumulator ready / slice in registers / arithmetic done
+  EV_D_EPI_BEGIN = 10, EV_D_EPI_END = 11, EV_TILE = 12, EV_D_HALF = 13, EV_D_LD_ISSUED = 14, EV_D_WAITED = 15
+};
+}  // namespace lqdev
+static __device__ unsigned long long g_lq_timeline[lqdev::TL_LISTS][lqdev::TL_CAP];   // one per translation unit
+namespace lqdev {
+struct TlCursor { int list; unsigned n; };
+__device__ __forceinline__ void tl_stamp(TlCursor& c, int ev, int tag) {
+  if (c.list >= 0 && c.n + 1 < (unsigned)TL_CAP)
+    g_lq_timeline[c.list][c.n++] = ((unsigned long long)ev << 48) | ((unsigned long long)(tag & 0xFF) << 40) |
+                                   ((unsigned long long)clock64() & 0xFFFFFFFFFFull);
+}
+#define LQ_TL_DECL(LIST_EXPR) lqdev::TlCursor tl_cur{(LIST_EXPR), 0u}
+#define LQ_TL(EV, TAG) lqdev::tl_stamp(tl_cur, (EV), (TAG))
+#else
+#define LQ_TL_DECL(LIST_EXPR)
+#define LQ_TL(EV, TAG)
+#endif
 
 }  // namespace lqdev

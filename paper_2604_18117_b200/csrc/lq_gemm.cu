@@ -11,17 +11,21 @@
 //   warp 0      TMA producer: operand tiles (two groups = 128 bytes of K per stage row) and
 //               the two groups' scale vectors, all signalled on the stage's "full" barrier
 //   warp 1      owns tensor memory; issues tcgen05.mma: each group of 64 codes is two K=32
-//               MMAs into a FRESH 128 x 256 accumulator (ring of 2 in tensor memory).  The
-//               loop is warp-uniform (operands live in uniform registers) and one elected
-//               lane issues; N = 256 keeps the tensor pipe at its full rate per instruction
-//   warps 2-17  drain: each warp owns 32 rows x a quarter of the tile's columns; tcgen05.ld one
-//               32 x 16 slice at a time, acc += P * (sx * sw) with packed f32x2 arithmetic
-//               in fp32 registers; after the last group: bias, convert, stage the warp's
-//               rows in shared memory, read them back with lanes along the row and store
-//               whole 64/128-byte row segments
-// Work is cut in units of 128 x 128 outputs; every CTA takes a contiguous run of units
-// (balanced to one unit) and walks it as 128 x 256 tiles, with a 128 x 128 tile where the
-// run or the row block ends.
+//               MMAs into a FRESH 128 x 128 accumulator.  The (up to) two groups of an operand
+//               stage fill one PAIR of accumulators that is handed over with one commit; two
+//               pairs alternate, so the issuer works a stage ahead of the drain.  The loop is
+//               warp-uniform (operands live in uniform registers) and one elected lane issues
+//   warps 2-17  drain: each warp owns 32 rows x 32 columns of the tile.  A group's accumulator
+//               slice is fetched as two tcgen05.ld.16x256b (256 bits per lane and access), ONE
+//               wait, and the accumulator is handed back at once; the next group's halves are
+//               requested as the registers of the current one are consumed, so the fetch runs
+//               under the arithmetic: acc += P * (sx * sw), packed f32x2, fp32 registers.  After
+//               the last group: bias is already in (it is the start value), convert, exchange
+//               inside each quad so that a lane holds 16 contiguous bytes of a row, store
+// The per-group arithmetic is the bound: 2 fp32 operations per output and group on 128 lanes
+// per SM, against 8192 MACs per clock on the tensor pipe - 256 clocks of drain for 128 clocks
+// of tensor work per 128 x 128 x 64 block.  Work is cut in 128 x 128 tiles; every CTA takes a
+// contiguous, balanced run of them, row block major.
 // The 4-bit codes ride in E4M3 operands (integers up to 7 are exact, fp32 accumulation of
 // |sum| <= 3136 is exact); the branch's 8-bit codes use kind::i8 (exact int32), the fp16
 // reference branch kind::f16.
@@ -29,30 +33,40 @@
 // raises a CTA-wide abort flag and all roles leave through the common teardown.
 #include <cuda_fp16.h>
 
-#include "lq_internal.h"
+#include "lq_device.cuh"
+
+#ifdef LQ_TIMELINE
+// Timeline build only: copies the stamp lists of the last launch to the host ([TL_LISTS][TL_CAP] words) and clears them.
+extern "C" int lq_debug_timeline(unsigned long long* host_out) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return 1;
+  if (cudaMemcpyFromSymbol(host_out, g_lq_timeline, sizeof(unsigned long long) * lqdev::TL_LISTS * lqdev::TL_CAP) != cudaSuccess) return 1;
+  static unsigned long long zeros[lqdev::TL_LISTS][lqdev::TL_CAP];
+  return cudaMemcpyToSymbol(g_lq_timeline, zeros, sizeof(zeros)) == cudaSuccess ? 0 : 1;
+}
+#endif
 
 namespace {
 
-constexpr int UNIT = LQ_BN;                        // 128 output columns
-constexpr int NSTAGE = 3;                          // operand ring depth
-constexpr int NTBUF = 2;                           // accumulator ring in tensor memory (2 x 256 columns)
-constexpr int TCOLS = 256;                         // columns per accumulator
+using namespace lqdev;
+
+constexpr int UNIT = LQ_BN;                        // 128 output columns per tile
+constexpr int NSTAGE = 4;                          // operand ring depth (a power of two: ring positions are masks)
+constexpr int NTBUF = 2;                           // ring of accumulator PAIRS in tensor memory: a pair = the (up to) two groups of one operand stage, 2 x 128 columns
+constexpr int TCOLS = 128;                         // columns per accumulator
 constexpr int STAGE_A_BYTES = LQ_BM * LQ_KSTAGE;   // 16 KB
-constexpr int STAGE_B_BYTES = 2 * UNIT * LQ_KSTAGE;   // 32 KB (two 128-row boxes)
+constexpr int STAGE_B_BYTES = UNIT * LQ_KSTAGE;    // 16 KB
 constexpr int STAGE_BYTES = STAGE_A_BYTES + STAGE_B_BYTES;
-constexpr int SC_GROUP_FLOATS = LQ_BM + 2 * UNIT;  // sx[128] then sw[256]
+constexpr int SC_GROUP_FLOATS = LQ_BM + UNIT;      // sx[128] then sw[128]
 constexpr int SC_STAGE_BYTES = 2 * SC_GROUP_FLOATS * 4;   // two groups
 constexpr int NUM_DRAIN_WARPS = 16;
 constexpr int FIRST_DRAIN_WARP = 2;
 constexpr int GEMM_THREADS = (FIRST_DRAIN_WARP + NUM_DRAIN_WARPS) * 32;
-constexpr int OUT_ROW_BYTES = 128;                 // output bytes staged per row and pass
-constexpr int OUT_ROW_STRIDE = OUT_ROW_BYTES + 16; // +16: rows start 4 banks apart, 16-byte stores do not conflict
-constexpr int OUT_WARP_BYTES = 32 * OUT_ROW_STRIDE;
+constexpr int WCOLS = 32;                          // columns per drain warp
 constexpr int SMEM_BAR_BYTES = 256;
-constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + NSTAGE * STAGE_BYTES + NSTAGE * SC_STAGE_BYTES +
-                           NUM_DRAIN_WARPS * OUT_WARP_BYTES + SMEM_BAR_BYTES;
+constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + NSTAGE * STAGE_BYTES + NSTAGE * SC_STAGE_BYTES + SMEM_BAR_BYTES;
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s at 2 GHz
+static_assert(STAGE_BYTES % 1024 == 0, "stages must keep the 1024-byte alignment of the swizzled tiles");
+static_assert((NSTAGE & (NSTAGE - 1)) == 0 && (NTBUF & (NTBUF - 1)) == 0, "ring sizes must be powers of two");
 
 struct GemmParams {
   int M, N, Mpad, Npad, G;
@@ -70,157 +84,41 @@ struct GemmParams {
   int32_t* status;
 };
 
-// ---- PTX wrappers -------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.b32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
-// Bounded wait.  Returns false when the CTA is aborting or the deadline passed (then it
-// raises the abort flag and records who gave up).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                            int role, long long limit = WAIT_LIMIT_CYCLES) {
-  const long long t0 = clock64();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 0xFF) == 0) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > limit) {
-        *abort_flag = 1;
-        if (atomicCAS(status, 0, (int)LQ_ERR_TIMEOUT) == 0) status[1] = role;
-        return false;
-      }
-    }
-  }
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                          int role) {
-  if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, status, role);
-}
-// The same wait for a whole warp whose control flow must stay provably uniform (the producer
-// and the MMA warp keep their loop state in uniform registers).
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                               int role) {
-  const bool ok = mbar_wait(bar, parity, abort_flag, status, role);
-  return __all_sync(0xffffffffu, ok);
-}
-
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.b32 %0, 1, 0, P;\n\t}" : "=r"(pred));
-  return pred != 0;
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
-               : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-template <int KIND>   // 0: i8, 1: f8f6f4, 2: f16
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  if constexpr (KIND == 0) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-  } else if constexpr (KIND == 1) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-  } else {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-  }
-}
-
-// 32 lanes x 16 consecutive 32-bit columns: thread t of the warp receives row (lane base + t).
-__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
-// 8-row atoms 1024 bytes apart.  Adding (bytes >> 4) steps along K inside the swizzled row.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
-  const uint32_t lo = ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16);          // start address, LBO = 1 (unused)
-  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);              // SBO = 1024 B, version 1, SWIZZLE_128B
-  return ((uint64_t)hi << 32) | lo;
-}
-
-// instruction descriptor: accumulator format, operand formats, N >> 3 at bit 17, M >> 4 at bit 24
-__device__ __forceinline__ constexpr uint32_t idesc_shape(int n) { return ((uint32_t)(n >> 3) << 17) | ((uint32_t)(LQ_BM >> 4) << 24); }
-constexpr uint32_t IDESC_I8 = (2u << 4) | (1u << 7) | (1u << 10);    // S8 x S8 -> S32
-constexpr uint32_t IDESC_F8 = (1u << 4) | (0u << 7) | (0u << 10);    // E4M3 x E4M3 -> F32
-constexpr uint32_t IDESC_F16 = (1u << 4) | (0u << 7) | (0u << 10);   // F16 x F16 -> F32
-
-// One accumulator slice of 32 rows x 16 columns: acc += P * (sx * sw).  INT: the accumulator
-// holds int32 (kind::i8); |P| < 2^22, so adding 1.5 * 2^23 in the integer domain and
-// subtracting it in fp32 converts exactly without the conversion pipe.
+// One accumulator slice of 16 rows x 32 columns in the layout of tcgen05.ld.16x256b (the accumulator-fragment layout
+// of mma.sync m16n8: with g = lane / 4 and t = lane % 4, registers 4j .. 4j+3 hold row g, columns 8j + 2t and
+// 8j + 2t + 1, then row g + 8, the same columns): acc += P * (sx * sw).  This shape moves 256 bits per lane and access;
+// the one-row-per-thread shape (32x32b) moves 32 and was measured at 60-80 bytes per clock and SM, which capped the
+// whole kernel.  INT: the accumulator holds int32 (kind::i8); |P| < 2^22, so adding 1.5 * 2^23 in the integer domain
+// and subtracting it in fp32 converts exactly without the conversion pipe.
 template <bool INT>
-__device__ __forceinline__ void drain_chunk(const uint32_t (&v)[16], float2 (&acc)[8], float sxv, const float* sw) {
-  const float2 sx2 = make_float2(sxv, sxv);
+__device__ __forceinline__ void drain_frag(const uint32_t (&v)[16], float2* acc, float sx_lo, float sx_hi, const float2 (&sw)[4]) {
+  const float2 sl = make_float2(sx_lo, sx_lo), sh = make_float2(sx_hi, sx_hi);
 #pragma unroll
-  for (int c4 = 0; c4 < 4; ++c4) {
-    const float4 w = *reinterpret_cast<const float4*>(sw + c4 * 4);
+  for (int j = 0; j < 4; ++j) {
     float2 p0, p1;
     if constexpr (INT) {
-      p0 = make_float2(__int_as_float((int)v[c4 * 4 + 0] + 0x4B400000) - 12582912.0f,
-                       __int_as_float((int)v[c4 * 4 + 1] + 0x4B400000) - 12582912.0f);
-      p1 = make_float2(__int_as_float((int)v[c4 * 4 + 2] + 0x4B400000) - 12582912.0f,
-                       __int_as_float((int)v[c4 * 4 + 3] + 0x4B400000) - 12582912.0f);
+      p0 = make_float2(__int_as_float((int)v[4 * j + 0] + 0x4B400000) - 12582912.0f,
+                       __int_as_float((int)v[4 * j + 1] + 0x4B400000) - 12582912.0f);
+      p1 = make_float2(__int_as_float((int)v[4 * j + 2] + 0x4B400000) - 12582912.0f,
+                       __int_as_float((int)v[4 * j + 3] + 0x4B400000) - 12582912.0f);
     } else {
-      p0 = make_float2(__uint_as_float(v[c4 * 4 + 0]), __uint_as_float(v[c4 * 4 + 1]));
-      p1 = make_float2(__uint_as_float(v[c4 * 4 + 2]), __uint_as_float(v[c4 * 4 + 3]));
+      p0 = make_float2(__uint_as_float(v[4 * j + 0]), __uint_as_float(v[4 * j + 1]));
+      p1 = make_float2(__uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
     }
-    const float2 s0 = __fmul2_rn(sx2, make_float2(w.x, w.y));
-    const float2 s1 = __fmul2_rn(sx2, make_float2(w.z, w.w));
-    acc[c4 * 2 + 0] = __ffma2_rn(p0, s0, acc[c4 * 2 + 0]);
-    acc[c4 * 2 + 1] = __ffma2_rn(p1, s1, acc[c4 * 2 + 1]);
+    acc[2 * j + 0] = __ffma2_rn(p0, __fmul2_rn(sl, sw[j]), acc[2 * j + 0]);
+    acc[2 * j + 1] = __ffma2_rn(p1, __fmul2_rn(sh, sw[j]), acc[2 * j + 1]);
   }
+}
+
+// 4 x 4 transpose across the four lanes of a quad: afterwards v[s] of lane t is what v[t] of lane s was.
+__device__ __forceinline__ void quad_transpose(uint32_t (&v)[4], int t) {
+  const bool hi2 = (t & 2) != 0, hi1 = (t & 1) != 0;
+  uint32_t y0 = __shfl_xor_sync(0xffffffffu, hi2 ? v[0] : v[2], 2);
+  uint32_t y1 = __shfl_xor_sync(0xffffffffu, hi2 ? v[1] : v[3], 2);
+  if (hi2) { v[0] = y0; v[1] = y1; } else { v[2] = y0; v[3] = y1; }
+  y0 = __shfl_xor_sync(0xffffffffu, hi1 ? v[0] : v[1], 1);
+  y1 = __shfl_xor_sync(0xffffffffu, hi1 ? v[2] : v[3], 1);
+  if (hi1) { v[0] = y0; v[2] = y1; } else { v[1] = y0; v[3] = y1; }
 }
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
@@ -233,9 +131,8 @@ lq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const uint32_t sm_stage = base;
   const uint32_t sm_sc = base + NSTAGE * STAGE_BYTES;
   const float* sc_ptr = reinterpret_cast<const float*>(smem + NSTAGE * STAGE_BYTES);
-  uint8_t* out_ptr = smem + NSTAGE * STAGE_BYTES + NSTAGE * SC_STAGE_BYTES;
-  const uint32_t sm_bar = sm_sc + NSTAGE * SC_STAGE_BYTES + NUM_DRAIN_WARPS * OUT_WARP_BYTES;
-  uint8_t* bar_ptr = out_ptr + NUM_DRAIN_WARPS * OUT_WARP_BYTES;
+  const uint32_t sm_bar = sm_sc + NSTAGE * SC_STAGE_BYTES;
+  uint8_t* bar_ptr = smem + NSTAGE * STAGE_BYTES + NSTAGE * SC_STAGE_BYTES;
   // barrier map (8 bytes each)
   auto bar_full = [&](int s) { return sm_bar + 8u * (uint32_t)s; };                        // operands + scales landed
   auto bar_empty = [&](int s) { return sm_bar + 8u * (uint32_t)(NSTAGE + s); };           // MMAs of the stage retired
@@ -250,7 +147,7 @@ lq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // provably warp-uniform
   const int lane = threadIdx.x & 31;
   const int stages_per_tile = p.n_stages_main + (p.branch_mmas > 0 ? 1 : 0);
-  // this CTA's contiguous run of 128 x 128 units, row block major
+  // this CTA's contiguous run of 128 x 128 tiles, row block major
   const long long units = (long long)p.tiles_m * p.units_n;
   const int u_begin = (int)((units * blockIdx.x) / gridDim.x);
   const int u_end = (int)((units * (blockIdx.x + 1)) / gridDim.x);
@@ -263,233 +160,246 @@ lq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int b = 0; b < NTBUF; ++b) { mbar_init(bar_tfull(b), 1); mbar_init(bar_tempty(b), NUM_DRAIN_WARPS); }
     *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_init_fence();
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
 
+  LQ_TL_DECL((blockIdx.x == 0 && lane == 0)
+                 ? (warp == 0 ? (int)TL_PRODUCER : warp == 1 ? (int)TL_MMA : warp == FIRST_DRAIN_WARP ? (int)TL_DRAIN_FIRST
+                    : warp == FIRST_DRAIN_WARP + NUM_DRAIN_WARPS - 1 ? (int)TL_DRAIN_LAST : -1)
+                 : -1);
+
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    uint32_t it = 0;
+    uint32_t it = 0, armed = 0;
     bool ok = true;
-    for (int u = u_begin; u < u_end && ok;) {
+    for (int u = u_begin; u < u_end && ok; ++u) {
       const int mb = u / p.units_n, nu = u - mb * p.units_n;
-      const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
       const int m0 = mb * LQ_BM, n0 = nu * UNIT;
       for (int s = 0; s < stages_per_tile && ok; ++s, ++it) {
-        const int st = it % NSTAGE;
+        const int st = it & (NSTAGE - 1);
         const uint32_t par = ((it / NSTAGE) & 1) ^ 1;
         ok = mbar_wait_warp(bar_empty(st), par, abort_flag, p.status, LQ_STAGE_PRODUCER);
         if (!ok) break;
         ok = mbar_wait_warp(bar_sempty(st), par, abort_flag, p.status, LQ_STAGE_PRODUCER);
         if (!ok) break;
+        LQ_TL(EV_P_SLOT_FREE, s);
         const uint32_t a_dst = sm_stage + st * STAGE_BYTES, b_dst = a_dst + STAGE_A_BYTES;
         const uint32_t sc_dst = sm_sc + st * SC_STAGE_BYTES;
         const uint32_t full = bar_full(st);
         const bool is_main = s < p.n_stages_main;
         const int ngroups = is_main ? ((2 * s + 1 < p.G) ? 2 : 1) : 1;
-        const uint32_t tx = STAGE_A_BYTES + width * (UNIT * LQ_KSTAGE) + ngroups * (LQ_BM + width * UNIT) * 4;
+        const uint32_t tx = STAGE_BYTES + ngroups * SC_GROUP_FLOATS * 4;
         if (elect_one()) {
           mbar_expect_tx(full, tx);
           if (is_main) {
             tma_load_2d(a_dst, &tmA, s * LQ_KSTAGE, m0, full);
             tma_load_2d(b_dst, &tmB, s * LQ_KSTAGE, n0, full);
-            if (width == 2) tma_load_2d(b_dst + UNIT * LQ_KSTAGE, &tmB, s * LQ_KSTAGE, n0 + UNIT, full);
             for (int q = 0; q < ngroups; ++q) {
               const size_t g = (size_t)(2 * s + q);
               bulk_load(sc_dst + q * SC_GROUP_FLOATS * 4, p.sx + g * p.Mpad + m0, LQ_BM * 4, full);
-              bulk_load(sc_dst + q * SC_GROUP_FLOATS * 4 + LQ_BM * 4, p.sw + g * p.Npad + n0, width * UNIT * 4, full);
+              bulk_load(sc_dst + q * SC_GROUP_FLOATS * 4 + LQ_BM * 4, p.sw + g * p.Npad + n0, UNIT * 4, full);
             }
           } else {
             tma_load_2d(a_dst, &tmT, 0, m0, full);
             tma_load_2d(b_dst, &tmL2, 0, n0, full);
-            if (width == 2) tma_load_2d(b_dst + UNIT * LQ_KSTAGE, &tmL2, 0, n0 + UNIT, full);
             bulk_load(sc_dst, p.sT + m0, LQ_BM * 4, full);
-            bulk_load(sc_dst + LQ_BM * 4, p.sL2 + n0, width * UNIT * 4, full);
+            bulk_load(sc_dst + LQ_BM * 4, p.sL2 + n0, UNIT * 4, full);
           }
         }
         __syncwarp();
+        ++armed;
+        LQ_TL(EV_P_ISSUED, s);
       }
-      u += width;
     }
-    if (!ok) {   // let copies in flight land before the CTA's shared memory goes away
-      const long long t0 = clock64();
-      while (clock64() - t0 < 2000000ll) { }
+    if (!ok && lane == 0) {
+      // aborting: give the copies already issued a bounded time to land before the CTA's shared memory goes away
+      const uint32_t n = armed < (uint32_t)NSTAGE ? armed : (uint32_t)NSTAGE;
+      for (uint32_t i = 1; i <= n; ++i) {
+        const uint32_t j = armed - i;
+        mbar_settle(bar_full(j % NSTAGE), (j / NSTAGE) & 1);
+      }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    uint32_t it = 0, slot = 0;
+    uint32_t it = 0;
     bool ok = true;
-    for (int u = u_begin; u < u_end && ok;) {
-      const int mb = u / p.units_n, nu = u - mb * p.units_n;
-      const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
-      const uint32_t shape = idesc_shape(width * UNIT);
+    const uint32_t shape = idesc_shape(UNIT);
+    for (int u = u_begin; u < u_end && ok; ++u) {
       for (int s = 0; s < stages_per_tile && ok; ++s, ++it) {
-        const int st = it % NSTAGE;
+        const int st = it & (NSTAGE - 1);
         ok = mbar_wait_warp(bar_full(st), (it / NSTAGE) & 1, abort_flag, p.status, LQ_STAGE_MMA);
         if (!ok) break;
         tc_fence_after();
+        LQ_TL(EV_M_STAGE_FULL, s);
         const uint32_t a_addr = sm_stage + st * STAGE_BYTES, b_addr = a_addr + STAGE_A_BYTES;
         const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
         const bool is_main = s < p.n_stages_main;
         const int ngroups = is_main ? ((2 * s + 1 < p.G) ? 2 : 1) : 1;
-        for (int q = 0; q < ngroups && ok; ++q, ++slot) {
-          const int buf = slot % NTBUF;
-          ok = mbar_wait_warp(bar_tempty(buf), ((slot / NTBUF) & 1) ^ 1, abort_flag, p.status, LQ_STAGE_MMA);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t d = tmem_base + buf * TCOLS;
+        // the stage's (up to) two groups go to the two accumulators of one pair; ONE commit hands the pair over
+        const int pb = it & (NTBUF - 1);
+        ok = mbar_wait_warp(bar_tempty(pb), ((it / NTBUF) & 1) ^ 1, abort_flag, p.status, LQ_STAGE_MMA);
+        if (!ok) break;
+        tc_fence_after();
+        LQ_TL(EV_M_ACC_FREE, s);
+        const uint32_t d = tmem_base + pb * (2 * TCOLS);
+        if (elect_one()) {
           if (is_main) {
-            const uint64_t off = (uint64_t)((q * 64) >> 4);
-            if (elect_one()) {
-              tc_mma<1>(d, adesc + off, bdesc + off, IDESC_F8 | shape, 0u);
-              tc_mma<1>(d, adesc + off + 2, bdesc + off + 2, IDESC_F8 | shape, 1u);
-              tc_commit(bar_tfull(buf));
+            for (int q = 0; q < ngroups; ++q) {
+              const uint64_t off = (uint64_t)((q * 64) >> 4);
+              tc_mma<TC_F8>(d + q * TCOLS, adesc + off, bdesc + off, IDESC_F8 | shape, 0u);
+              tc_mma<TC_F8>(d + q * TCOLS, adesc + off + 2, bdesc + off + 2, IDESC_F8 | shape, 1u);
             }
           } else {
-            if (elect_one()) {
-              for (int j = 0; j < p.branch_mmas; ++j) {
-                const uint64_t off = (uint64_t)((j * 32) >> 4);
-                if (p.branch_f16) tc_mma<2>(d, adesc + off, bdesc + off, IDESC_F16 | shape, (uint32_t)j);
-                else tc_mma<0>(d, adesc + off, bdesc + off, IDESC_I8 | shape, (uint32_t)j);
-              }
-              tc_commit(bar_tfull(buf));
+            for (int j = 0; j < p.branch_mmas; ++j) {
+              const uint64_t off = (uint64_t)((j * 32) >> 4);
+              if (p.branch_f16) tc_mma<TC_F16>(d, adesc + off, bdesc + off, IDESC_F16 | shape, (uint32_t)j);
+              else tc_mma<TC_I8>(d, adesc + off, bdesc + off, IDESC_I8 | shape, (uint32_t)j);
             }
           }
-          __syncwarp();
+          tc_commit(bar_tfull(pb));
+          tc_commit(bar_empty(st));
         }
-        if (elect_one()) tc_commit(bar_empty(st));
         __syncwarp();
+        LQ_TL(EV_M_ISSUED, s);
       }
-      u += width;
     }
   } else {
     // ------------------------------------------------------------------ drain + epilogue
     const int quad = warp & 3;                          // tensor-memory lanes 32*quad .. 32*quad+31
     const int cgi = (warp - FIRST_DRAIN_WARP) >> 2;     // which quarter of the tile's columns
-    const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16);
-    uint8_t* out_row = out_ptr + (warp - FIRST_DRAIN_WARP) * OUT_WARP_BYTES + lane * OUT_ROW_STRIDE;
-    uint32_t it = 0, slot = 0;
+    const int coff = cgi * WCOLS;
+    const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)coff;
+    const int fg = lane >> 2, ft = lane & 3;            // fragment coordinates: rows fg + 8 i, column pair ft
+    uint32_t it = 0;
     bool ok = true;
-    for (int u = u_begin; u < u_end && ok;) {
+    for (int u = u_begin; u < u_end && ok; ++u) {
       const int mb = u / p.units_n, nu = u - mb * p.units_n;
-      const int width = (nu + 1 < p.units_n && u + 1 < u_end) ? 2 : 1;
       const int m0 = mb * LQ_BM, n0 = nu * UNIT;
-      const int coff = cgi * width * 32;                // first of this warp's width*32 columns
-      float2 acc[4][8];                                 // [16-column chunk][column pair], starts from the bias
+      LQ_TL(EV_TILE, 0);
+      // this thread's 4 rows x 8 columns: acc[8 h + 2 j + i] = rows 16 h + fg + 8 i, columns 8 j + 2 ft, + 1; starts from the bias
+      float2 acc[16];
 #pragma unroll
-      for (int a = 0; a < 4; ++a) {
-        if (a < 2 * width) {
-          const float4* b4 = reinterpret_cast<const float4*>(p.bias + n0 + coff + a * 16);
-#pragma unroll
-          for (int b = 0; b < 4; ++b) {
-            const float4 bv = __ldg(b4 + b);
-            acc[a][2 * b] = make_float2(bv.x, bv.y);
-            acc[a][2 * b + 1] = make_float2(bv.z, bv.w);
-          }
-        }
+      for (int j = 0; j < 4; ++j) {
+        const float2 bv = __ldg(reinterpret_cast<const float2*>(p.bias + n0 + coff + 8 * j + 2 * ft));
+        acc[2 * j] = bv; acc[2 * j + 1] = bv; acc[8 + 2 * j] = bv; acc[8 + 2 * j + 1] = bv;
+      }
+      // Groups g = 0 .. G-1 come two per operand stage, then the branch has a stage of its own.  `it` counts operand
+      // stages since the kernel began: stage ring position it & (NSTAGE-1), accumulator pair it & (NTBUF-1).  All
+      // hand-shakes are per stage: the scale vectors and the accumulator pair are awaited once, the pair is handed back
+      // when its last group sits in registers.  The group being consumed sits in (vlo, vhi): rows 0-15 and 16-31 of
+      // this warp's quarter, 32 columns each; the next group's halves are requested as soon as a half is consumed.
+      uint32_t vlo[16], vhi[16];
+      // waits for stage `IT_`'s scale vectors and accumulator pair
+#define LQ_AWAIT_STAGE(IT_)                                                                                              \
+      {                                                                                                                  \
+        const uint32_t i_ = (IT_);                                                                                       \
+        ok = mbar_wait(bar_full(i_ & (NSTAGE - 1)), (i_ / NSTAGE) & 1, abort_flag, p.status, LQ_STAGE_DRAIN);            \
+        if (ok) ok = mbar_wait(bar_tfull(i_ & (NTBUF - 1)), (i_ / NTBUF) & 1, abort_flag, p.status, LQ_STAGE_DRAIN);     \
+        tc_fence_after();                                                                                                \
+      }
+      // one group: arithmetic on (vlo, vhi) with the scales at SCG_; the next group's halves (if HAS_NEXT_) are at TNEXT_
+#define LQ_DRAIN_GROUP(SCG_, IS_INT_, HAS_NEXT_, TNEXT_)                                                                 \
+      {                                                                                                                  \
+        const float* sxp_ = (SCG_) + quad * 32 + fg;                                                                     \
+        const float* swp_ = (SCG_) + LQ_BM + coff + 2 * ft;                                                              \
+        const float sx0 = sxp_[0], sx1 = sxp_[8], sx2 = sxp_[16], sx3 = sxp_[24];                                        \
+        float2 sw2[4];                                                                                                   \
+        _Pragma("unroll") for (int j_ = 0; j_ < 4; ++j_) sw2[j_] = *reinterpret_cast<const float2*>(swp_ + 8 * j_);      \
+        if (IS_INT_) drain_frag<true>(vlo, &acc[0], sx0, sx1, sw2);                                                      \
+        else drain_frag<false>(vlo, &acc[0], sx0, sx1, sw2);                                                             \
+        if (HAS_NEXT_) tmem_ld_16x256b_x4((TNEXT_), vlo);                                                                \
+        if (IS_INT_) drain_frag<true>(vhi, &acc[8], sx2, sx3, sw2);                                                      \
+        else drain_frag<false>(vhi, &acc[8], sx2, sx3, sw2);                                                             \
+        if (HAS_NEXT_) tmem_ld_16x256b_x4((TNEXT_) + (16u << 16), vhi);                                                  \
+      }
+      LQ_AWAIT_STAGE(it)
+      if (!ok) break;
+      {
+        const uint32_t t0_ = tlane + (it & (NTBUF - 1)) * (2 * TCOLS);
+        tmem_ld_16x256b_x4(t0_, vlo);
+        tmem_ld_16x256b_x4(t0_ + (16u << 16), vhi);
       }
       for (int s = 0; s < stages_per_tile && ok; ++s, ++it) {
-        const int st = it % NSTAGE;
-        ok = mbar_wait(bar_full(st), (it / NSTAGE) & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
-        if (!ok) break;
         const bool is_main = s < p.n_stages_main;
-        const int ngroups = is_main ? ((2 * s + 1 < p.G) ? 2 : 1) : 1;
+        const bool two = is_main && (2 * s + 1 < p.G);
         const bool is_int = !is_main && p.branch_f16 == 0;
-        for (int q = 0; q < ngroups && ok; ++q, ++slot) {
-          const int buf = slot % NTBUF;
-          ok = mbar_wait(bar_tfull(buf), (slot / NTBUF) & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
-          if (!ok) break;
-          tc_fence_after();
-          const float* scg = sc_ptr + (size_t)st * (SC_STAGE_BYTES / 4) + q * SC_GROUP_FLOATS;
-          const float sxv = scg[quad * 32 + lane];
-          const float* swp = scg + LQ_BM + coff;
-          const uint32_t taddr = tlane + (uint32_t)(buf * TCOLS + coff);
-#pragma unroll
-          for (int ch = 0; ch < 4; ++ch) {
-            if (ch < 2 * width) {
-              uint32_t v[16];
-              tmem_ld_32x16(taddr + ch * 16, v);
-              tmem_ld_wait();
-              if (ch == 2 * width - 1) {     // the accumulator may be overwritten once every warp has read its part
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_tempty(buf));
-              }
-              if (is_int) drain_chunk<true>(v, acc[ch], sxv, swp + ch * 16);
-              else drain_chunk<false>(v, acc[ch], sxv, swp + ch * 16);
-            }
-          }
+        const bool last_stage = s + 1 == stages_per_tile;
+        const int st = it & (NSTAGE - 1);
+        const float* scg = sc_ptr + st * (SC_STAGE_BYTES / 4);
+        const uint32_t tpair = tlane + (it & (NTBUF - 1)) * (2 * TCOLS);
+        const uint32_t tpair_next = tlane + ((it + 1) & (NTBUF - 1)) * (2 * TCOLS);
+        LQ_TL(EV_D_OPEN, s);
+        if (two) {
+          tmem_ld_wait();                               // the stage's first group is in registers
+          LQ_TL(EV_D_WAITED, s);
+          LQ_DRAIN_GROUP(scg, false, true, tpair + TCOLS)
+          LQ_TL(EV_D_HALF, s);
         }
+        tmem_ld_wait();                                 // the stage's last group is in registers:
+        tc_fence_before();                              // the accumulator pair goes back to the MMA warp
         __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty(it & (NTBUF - 1)));
+        LQ_TL(EV_D_LOADED, s);
+        if (!last_stage) LQ_AWAIT_STAGE(it + 1)
+        LQ_TL(EV_D_ACC_FULL, s);
+        {
+          const float* scg2 = scg + (two ? SC_GROUP_FLOATS : 0);
+          const bool has_next = !last_stage && ok;
+          LQ_DRAIN_GROUP(scg2, is_int, has_next, tpair_next)
+        }
+        LQ_TL(EV_D_DONE, s);
+        __syncwarp();                                   // done with this stage's scale vectors
         if (lane == 0) mbar_arrive(bar_sempty(st));
       }
+#undef LQ_DRAIN_GROUP
+#undef LQ_AWAIT_STAGE
       if (!ok) break;
-      // epilogue: convert, stage this thread's row segment in the warp's shared-memory rows, read it back
-      // with lanes along the row and store whole 64/128-byte row segments
-      const int rbase = m0 + quad * 32;
-      const int col0 = n0 + coff;
-      const int esize = p.out_f32 ? 4 : 2;
-      const int cols_per_pass = OUT_ROW_BYTES / esize;                  // 64 halves or 32 floats
-      const int npass = (width * 32 + cols_per_pass - 1) / cols_per_pass;
+      LQ_TL(EV_D_EPI_BEGIN, 0);
+      // epilogue straight from registers: rows m0 + 32 quad + 16 h + fg (+ 8), columns n0 + coff + 8 j + 2 ft (+ 1)
+      const int row_w = m0 + quad * 32;
+      if (p.out_f32) {
+        float* Y = reinterpret_cast<float*>(p.Y);
 #pragma unroll
-      for (int pass = 0; pass < 2; ++pass) {
-        if (pass < npass) {
-          __syncwarp();                                                 // previous pass has been read back
-          if (p.out_f32) {
+        for (int h = 0; h < 2; ++h) {
+          const int r_lo = row_w + 16 * h + fg, r_hi = r_lo + 8;
 #pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-              const int ch = pass * 2 + cc;
-              if (ch < 2 * width) {
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4)
-                  *reinterpret_cast<float4*>(out_row + cc * 64 + c4 * 16) =
-                      make_float4(acc[ch][c4 * 2].x, acc[ch][c4 * 2].y, acc[ch][c4 * 2 + 1].x, acc[ch][c4 * 2 + 1].y);
-              }
-            }
-          } else {
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-              if (ch < 2 * width) {
-#pragma unroll
-                for (int c8 = 0; c8 < 2; ++c8) {
-                  __half2 h[4];
-                  h[0] = __floats2half2_rn(acc[ch][c8 * 4 + 0].x, acc[ch][c8 * 4 + 0].y);
-                  h[1] = __floats2half2_rn(acc[ch][c8 * 4 + 1].x, acc[ch][c8 * 4 + 1].y);
-                  h[2] = __floats2half2_rn(acc[ch][c8 * 4 + 2].x, acc[ch][c8 * 4 + 2].y);
-                  h[3] = __floats2half2_rn(acc[ch][c8 * 4 + 3].x, acc[ch][c8 * 4 + 3].y);
-                  *reinterpret_cast<uint4*>(out_row + ch * 32 + c8 * 16) = *reinterpret_cast<uint4*>(h);
-                }
-              }
-            }
-          }
-          __syncwarp();
-          int ncols = width * 32 - pass * cols_per_pass;                // columns of this pass
-          if (ncols > cols_per_pass) ncols = cols_per_pass;
-          const int lpr = ncols * esize / 16;                           // lanes per row: 4 or 8
-          const int rpi = 32 / lpr;                                     // rows per instruction
-          const int cpl = 16 / esize;                                   // columns per lane
-          const int lcol = col0 + pass * cols_per_pass + (lane % lpr) * cpl;
-          const uint8_t* wbase = out_ptr + (warp - FIRST_DRAIN_WARP) * OUT_WARP_BYTES + (lane % lpr) * 16;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            if (i * rpi < 32) {
-              const int rl = i * rpi + lane / lpr;
-              const uint4 val = *reinterpret_cast<const uint4*>(wbase + rl * OUT_ROW_STRIDE);
-              if (rbase + rl < p.M && lcol < p.N)
-                *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(p.Y) + ((size_t)(rbase + rl) * p.N + lcol) * esize) = val;
+          for (int j = 0; j < 4; ++j) {
+            const int c = n0 + coff + 8 * j + 2 * ft;                  // four lanes write the 32 bytes of one row's sector
+            if (c < p.N) {
+              if (r_lo < p.M) *reinterpret_cast<float2*>(Y + (size_t)r_lo * p.N + c) = acc[8 * h + 2 * j];
+              if (r_hi < p.M) *reinterpret_cast<float2*>(Y + (size_t)r_hi * p.N + c) = acc[8 * h + 2 * j + 1];
             }
           }
         }
+      } else {
+        __half* Y = reinterpret_cast<__half*>(p.Y);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          // pack to fp16, then exchange inside the quad: lane ft ends up with columns 8 ft .. 8 ft + 7 of both rows
+          uint32_t lo[4], hi[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const __half2 l2 = __floats2half2_rn(acc[8 * h + 2 * j].x, acc[8 * h + 2 * j].y);
+            const __half2 h2 = __floats2half2_rn(acc[8 * h + 2 * j + 1].x, acc[8 * h + 2 * j + 1].y);
+            lo[j] = *reinterpret_cast<const uint32_t*>(&l2);
+            hi[j] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+          quad_transpose(lo, ft);
+          quad_transpose(hi, ft);
+          const int c = n0 + coff + 8 * ft;                            // 16 contiguous bytes of a row per lane
+          const int r_lo = row_w + 16 * h + fg, r_hi = r_lo + 8;
+          if (c < p.N) {
+            if (r_lo < p.M) *reinterpret_cast<uint4*>(Y + (size_t)r_lo * p.N + c) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            if (r_hi < p.M) *reinterpret_cast<uint4*>(Y + (size_t)r_hi * p.N + c) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          }
+        }
       }
-      u += width;
+      LQ_TL(EV_D_EPI_END, 0);
     }
   }
 
@@ -498,7 +408,7 @@ lq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    tmem_dealloc(tmem_base, 512);
   }
 }
 
@@ -510,7 +420,7 @@ __global__ void lq_wait_probe_kernel(int32_t* status, long long limit) {
   if (threadIdx.x == 0) {
     mbar_init(bar, 1);
     abort_word = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_init_fence();
   }
   __syncwarp();
   mbar_wait_slow(bar, 0, &abort_word, status, LQ_STAGE_TEARDOWN, limit);
