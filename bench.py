@@ -11,10 +11,14 @@ stand in for the paper's PixArt-Sigma activations and weights.
 
 Prints ONE JSON line.  `value` is TOPS (2MKN + 2Mr(K+N) algorithmic ops per layer) with inputs
 resident in HBM; `e2e` is the same metric through lq_linear_forward_host_async (pinned host X in,
-host Y out, one stream per layer, all synchronised at the end of the step: copies inside the timed region); `roofline` describes the GEMM kernel against the
-8-bit-operand tensor peak (2 x the measured bf16 cuBLAS peak); `cpu_baseline` is the CPU oracle
-timed on a 256-row sample of the same layers.  With N > 1 (torchrun) every rank runs the same
-rows-sharded workload independently (rows are independent: no collective on the data path).
+host Y out, one stream per layer, all synchronised at the end of the step: copies inside the timed region);
+`roofline` describes the GEMM kernel against the 8-bit-operand tensor peak (2 x the measured bf16 cuBLAS burst peak),
+with the fractions against the nominal and the sustained peak and against the composite bound
+max(t_tensor, t_drain, t_HBM) per layer beside it; `mxint4` (default run only) is the same step with the MXINT4 main
+branch; `cpu_baseline` is the CPU oracle timed on a 256-row sample of the same layers.  `--config 4` runs the whole
+PixArt-class stack (28 blocks x 4 linears back to back, M = 32768, no L2 flush) and reports tokens/s.  With N > 1
+(torchrun) every rank runs the same rows-sharded workload independently (rows are independent: no collective on the
+data path).
 """
 from __future__ import annotations
 
@@ -42,6 +46,28 @@ def layer_ops(M, K, N, r):
 
 def gemm_ops(M, K, N, r):
     return 2.0 * M * K * N + 2.0 * M * r * N
+
+
+NOMINAL_8BIT_TOPS = 4500.0      # dense 8-bit-operand class figure of the part (context, not the denominator of `frac`)
+SMS, FP32_LANES, SM_MAX_HZ = 148, 128, 1.965e9
+STACK_BLOCKS = 28
+
+
+def layer_bounds(M, K, N, r, main, peaks):
+    """Lower bounds (seconds) of one layer's two kernels from the algorithmic figures:
+    K2 tensor: ops / (2 x bf16 burst); K2 drain (SINT4 only): 2 fp32 operations per output and group (G groups + the
+    branch) on 128 lanes per SM at the maximum SM clock; K2 HBM: packed 4-bit codes, scales, branch codes in, fp16 Y
+    out, weights once; K1 HBM: X in, codes and scales out."""
+    G = -(-K // (32 if main == "mxint4" else 64))
+    sc = G if main == "mxint4" else 2 * G
+    t_tensor = gemm_ops(M, K, N, r) / (2.0 * peaks["bf16_tflops"] * 1e12)
+    t_drain = 0.0 if main == "mxint4" else 2.0 * M * N * (-(-K // 64) + (1 if r else 0)) / (SMS * FP32_LANES * SM_MAX_HZ)
+    k2_bytes = M * (K // 2 + sc + r + 4) + 2 * M * N + (K * N // 2 + sc * N + r * N + 4 * N)
+    k1_bytes = M * (2 * K + K // 2 + K + sc + 4 + r + 4)
+    t_hbm2 = k2_bytes / (peaks["hbm_gbs"] * 1e9)
+    t_hbm1 = k1_bytes / (peaks["hbm_gbs"] * 1e9)
+    return {"t_tensor_us": t_tensor * 1e6, "t_drain_us": t_drain * 1e6, "t_hbm_gemm_us": t_hbm2 * 1e6,
+            "t_hbm_quant_us": t_hbm1 * 1e6, "gemm_bound_us": max(t_tensor, t_drain, t_hbm2) * 1e6, "k1_bytes": k1_bytes}
 
 
 def measured_peaks():
@@ -170,12 +196,26 @@ MAIN_NAMES = {"sint4": "SINT4 group 64 (fp16 scales)", "mxint4": "MXINT4 block 3
 
 
 def workload_config(wl, args):
-    return {"workload": f"config{wl.config}: PixArt-class block linears (qkv 1152->3456, attn-out 1152->1152, "
-                        f"fc1 1152->4608, fc2 4608->1152), M={wl.M} rows (4096 tokens x batch 2), rank {wl.rank}, "
-                        f"main W4A4 {MAIN_NAMES[args.main]}, branch {wl.branch}" if wl.config in (1, 2) else f"config{wl.config}",
+    if wl.config in (1, 2):
+        desc = (f"config{wl.config}: PixArt-class block linears (qkv 1152->3456, attn-out 1152->1152, fc1 1152->4608, "
+                f"fc2 4608->1152), M={wl.M} rows (4096 tokens x batch 2), rank {wl.rank}, main W4A4 {MAIN_NAMES[args.main]}, "
+                f"branch {wl.branch}")
+    elif wl.config == 4:
+        desc = (f"config4: full PixArt-class stack, {STACK_BLOCKS} blocks x (qkv, attn-out, fc1, fc2) run back to back, "
+                f"M={wl.M} rows (batch 8 x 4096 tokens; the 2048px case, 16384 tokens x batch 2, has the same row count and "
+                f"the same launches), rank {wl.rank}, main W4A4 {MAIN_NAMES[args.main]}, branch {wl.branch}; one calibrated "
+                f"layer and one X / Y buffer per distinct shape, reused by all blocks; no L2 flush inside the stack")
+    elif wl.config == 3:
+        desc = (f"config3: SANA-class block linears (qkv 2240->6720, out 2240->2240, up 2240->5600, down 5600->2240), "
+                f"M={wl.M} rows, rank {wl.rank}, main W4A4 {MAIN_NAMES[args.main]}, branch {wl.branch}")
+    else:
+        desc = f"config{wl.config}"
+    return {"workload": desc,
             "main": args.main, "rows": wl.M, "rank": wl.rank, "branch": wl.branch, "layers": [s.name for s in wl.layers],
             "calibration_steps": args.calib_steps,
-            "l2": ("L2 flushed (256 MiB write) before every timed step; layers inside a step run back to back"
+            "l2": ("no flush: one pass of the stack touches 112 x (X + codes + Y) = far more than the 126 MB L2; per-launch "
+                   "times are those of the first block of each pass" if wl.config == 4 else
+                   "L2 flushed (256 MiB write) before every timed step; layers inside a step run back to back"
                    if args.l2 == "flush" else
                    "no explicit flush: one step reads 132 MB of X and writes 170 MB of Y plus 66 MB of codes, the L2 holds 126 MB"),
             "parallelism": f"rows sharded x{args.gpus}, no collective"}
@@ -202,8 +242,8 @@ def cpu_baseline(wl, I, args):
         if dt > 10.0 or n >= 200:
             break
     return {"value": ops * n / dt / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-            "sample": f"{SAMPLE_ROWS} seeded rows of each of the {len(layers)} layers, {n} passes in {dt:.1f} s "
-                      f"(numpy/BLAS threads as configured on the box)"}
+            "sample": f"{SAMPLE_ROWS} seeded rows of each of the {len(layers)} layers, {n} passes in {dt:.1f} s; the oracle is "
+                      f"numpy: its matrix products run on `cores` BLAS threads, everything else (quantizers, scaling) on one"}
 
 
 def run_ours(args):
@@ -220,168 +260,222 @@ def run_ours(args):
     dev = torch.device(f"cuda:{local}")
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    BUILD.build()
+    # one process per node builds (a stale library would otherwise be rebuilt by every rank at once into the same files)
+    if local == 0:
+        BUILD.build()
+    if world > 1:
+        dist.barrier()
     I, wl = build_workload(args)
     M, r = wl.M, wl.rank
     st = torch.cuda.current_stream().cuda_stream
-
-    layers = []
-    for spec in wl.layers:
-        Xh, W, bias = I.layer_inputs(wl, spec, seed=D.shard_seed(0, rank), with_bias=True)
-        cfg = B.lq_config_default(spec.K, spec.N, r, wl.branch)
-        cfg.steps = args.calib_steps
-        if args.main == "mxint4":
-            cfg.group = 32
-        h, _ = B.lq_calibrate(cfg, W, bias)
-        B.lq_layer_to_device(h, local)
-        act = B.lq_act_create(h, M, local)
-        Xd = torch.from_numpy(Xh).to(dev)
-        Yd = torch.empty((M, spec.N), dtype=torch.float16, device=dev)
-        Xp = torch.from_numpy(Xh).pin_memory()
-        Yp = torch.empty((M, spec.N), dtype=torch.float16).pin_memory()
-        layers.append(dict(spec=spec, h=h, act=act, Xd=Xd, Yd=Yd, Xp=Xp, Yp=Yp))
-    ops_step = sum(layer_ops(M, L["spec"].K, L["spec"].N, r) for L in layers)
-    gops_step = sum(gemm_ops(M, L["spec"].K, L["spec"].N, r) for L in layers)
+    stack = wl.config == 4
+    repeats = STACK_BLOCKS if stack else 1           # the stack runs its four distinct layers 28 times back to back
+    peaks = measured_peaks()
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
-
-    def step(timed=None):
-        if args.l2 == "flush":
-            flush.zero_()
-        if timed is not None:
-            timed["s"].record()
-        for i, L in enumerate(layers):
-            if timed is not None:
-                timed["q0"][i].record()
-            B.lq_quantize_act(L["h"], L["Xd"].data_ptr(), M, L["act"], st)
-            if timed is not None:
-                timed["g0"][i].record()
-            B.lq_linear_forward(L["h"], L["act"], L["Yd"].data_ptr(), B.OUT_F16, st)
-            if timed is not None:
-                timed["g1"][i].record()
-        if timed is not None:
-            timed["e"].record()
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        step()
-    ev = lambda: torch.cuda.Event(enable_timing=True)
-    timers = [dict(s=ev(), e=ev(), q0=[ev() for _ in layers], g0=[ev() for _ in layers], g1=[ev() for _ in layers])
-              for _ in range(args.steps)]
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-        t_wait = time.perf_counter()          # nvidia-smi needs a moment before its first line: keep the GPU busy meanwhile
-        while not sampler.rows and time.perf_counter() - t_wait < 3.0:
+    def setup(main):
+        layers = []
+        for spec in wl.layers:
+            Xh, W, bias = I.layer_inputs(wl, spec, seed=D.shard_seed(0, rank), with_bias=True)
+            cfg = B.lq_config_default(spec.K, spec.N, r, wl.branch)
+            cfg.steps = args.calib_steps
+            if main == "mxint4":
+                cfg.group = 32
+            h, _ = B.lq_calibrate(cfg, W, bias)
+            B.lq_layer_to_device(h, local)
+            act = B.lq_act_create(h, M, local)
+            Xd = torch.from_numpy(Xh).to(dev)
+            Yd = torch.empty((M, spec.N), dtype=torch.float16, device=dev)
+            layers.append(dict(spec=spec, h=h, act=act, Xd=Xd, Yd=Yd, Xh=Xh))
+        return layers
+
+    def teardown(layers):
+        for L in layers:
+            B.lq_act_free(L["act"])
+            B.lq_layer_free(L["h"])
+
+    def measure(main, layers, steps, sample_clocks):
+        """Device-resident timing of `steps` steps; returns per-step and per-launch CUDA-event times."""
+        def step(timed=None):
+            if args.l2 == "flush" and not stack:
+                flush.zero_()
+            if timed is not None:
+                timed["s"].record()
+            for rep in range(repeats):
+                for i, L in enumerate(layers):
+                    ev = timed is not None and rep == 0
+                    if ev:
+                        timed["q0"][i].record()
+                    B.lq_quantize_act(L["h"], L["Xd"].data_ptr(), M, L["act"], st)
+                    if ev:
+                        timed["g0"][i].record()
+                    B.lq_linear_forward(L["h"], L["act"], L["Yd"].data_ptr(), B.OUT_F16, st)
+                    if ev:
+                        timed["g1"][i].record()
+            if timed is not None:
+                timed["e"].record()
+
+        for _ in range(max(args.warmup, 3)):
             step()
-            torch.cuda.synchronize()
-    barrier()
-    n_before = len(sampler.rows)
-    t_timed = time.perf_counter()
-    for t in timers:
-        step(t)
-    barrier()
-    timed_wall = time.perf_counter() - t_timed
-    clocks = None
-    if rank == 0:
-        # The timed region of a short run is over before nvidia-smi (one line per 100 ms) reports: repeat the same
-        # steps, untimed, until at least 1.5 s of this load have been sampled.
-        extended = False
-        while time.perf_counter() - t_timed < 1.5:
-            extended = True
-            step()
-            torch.cuda.synchronize()
-        sampler.rows = sampler.rows[n_before:]
-        clocks = sampler.stop()
-        clocks["window"] = (f"timed region of {timed_wall * 1e3:.0f} ms" +
-                            (" plus untimed repeats of the same steps up to 1.5 s" if extended else ""))
-    barrier()
-    step_ms = [t["s"].elapsed_time(t["e"]) for t in timers]
-    gemm_ms = [sum(a.elapsed_time(b) for a, b in zip(t["g0"], t["g1"])) for t in timers]
-    quant_ms = [sum(a.elapsed_time(b) for a, b in zip(t["q0"], t["g0"])) for t in timers]
-    per_layer = []
-    for i, L in enumerate(layers):
-        q = float(np.mean([t["q0"][i].elapsed_time(t["g0"][i]) for t in timers]))
-        g = float(np.mean([t["g0"][i].elapsed_time(t["g1"][i]) for t in timers]))
-        sp = L["spec"]
-        per_layer.append({"layer": sp.name, "K": sp.K, "N": sp.N, "quantize_us": q * 1e3, "gemm_us": g * 1e3,
-                          "gemm_tops": gemm_ops(M, sp.K, sp.N, r) / (g * 1e-3) / 1e12,
-                          "pair_tops": layer_ops(M, sp.K, sp.N, r) / ((q + g) * 1e-3) / 1e12})
-    total_ms = float(sum(step_ms))
-    code, stage = B.lq_get_device_status(local)
-    if code != 0:
-        raise SystemExit(f"device status {code} (stage {stage}) after the timed region")
-    total_ms_max = D.max_over_ranks(total_ms, world, dev)
+        ev = lambda: torch.cuda.Event(enable_timing=True)
+        timers = [dict(s=ev(), e=ev(), q0=[ev() for _ in layers], g0=[ev() for _ in layers], g1=[ev() for _ in layers])
+                  for _ in range(steps)]
+        sampler = ClockSampler(local)
+        if rank == 0 and sample_clocks:
+            sampler.start()
+            t_wait = time.perf_counter()          # nvidia-smi needs a moment before its first line: keep the GPU busy meanwhile
+            while not sampler.rows and time.perf_counter() - t_wait < 3.0:
+                step()
+                torch.cuda.synchronize()
+        barrier()
+        n_before = len(sampler.rows)
+        t_timed = time.perf_counter()
+        for t in timers:
+            step(t)
+        barrier()
+        timed_wall = time.perf_counter() - t_timed
+        clocks = None
+        if rank == 0 and sample_clocks:
+            # The timed region of a short run is over before nvidia-smi (one line per 100 ms) reports: repeat the same
+            # steps, untimed, until at least 1.5 s of this load have been sampled.
+            extended = False
+            while time.perf_counter() - t_timed < 1.5:
+                extended = True
+                step()
+                torch.cuda.synchronize()
+            sampler.rows = sampler.rows[n_before:]
+            clocks = sampler.stop()
+            clocks["window"] = (f"timed region of {timed_wall * 1e3:.0f} ms" +
+                                (" plus untimed repeats of the same steps up to 1.5 s" if extended else ""))
+        barrier()
+        code, stage = B.lq_get_device_status(local)
+        if code != 0:
+            raise SystemExit(f"device status {code} (stage {stage}) after the timed region")
+        step_ms = [t["s"].elapsed_time(t["e"]) for t in timers]
+        per_layer = []
+        for i, L in enumerate(layers):
+            q = float(np.mean([t["q0"][i].elapsed_time(t["g0"][i]) for t in timers]))
+            g = float(np.mean([t["g0"][i].elapsed_time(t["g1"][i]) for t in timers]))
+            sp = L["spec"]
+            bd = layer_bounds(M, sp.K, sp.N, r, main, peaks)
+            per_layer.append({"layer": sp.name, "K": sp.K, "N": sp.N, "quantize_us": q * 1e3, "gemm_us": g * 1e3,
+                              "gemm_tops": gemm_ops(M, sp.K, sp.N, r) / (g * 1e-3) / 1e12,
+                              "pair_tops": layer_ops(M, sp.K, sp.N, r) / ((q + g) * 1e-3) / 1e12,
+                              "bounds_us": {k: round(v, 2) for k, v in bd.items() if k.endswith("_us")},
+                              "k1_bytes": bd["k1_bytes"]})
+        total_ms_max = D.max_over_ranks(float(sum(step_ms)), world, dev)
+        return {"total_ms": total_ms_max, "steps": steps, "layers": per_layer, "clocks": clocks}
+
+    def summarise(main, res):
+        """value / roofline records of one measured format."""
+        ops_step = repeats * sum(layer_ops(M, L["K"], L["N"], r) for L in res["layers"])
+        gops_block = sum(gemm_ops(M, L["K"], L["N"], r) for L in res["layers"])
+        gemm_ms = sum(L["gemm_us"] for L in res["layers"]) * 1e-3
+        quant_ms = sum(L["quantize_us"] for L in res["layers"]) * 1e-3
+        achieved = gops_block / (gemm_ms * 1e-3) / 1e12
+        burst, sust = 2.0 * peaks["bf16_tflops"], 2.0 * (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"])
+        bound_gemm_ms = sum(L["bounds_us"]["gemm_bound_us"] for L in res["layers"]) * 1e-3
+        bound_quant_ms = sum(L["bounds_us"]["t_hbm_quant_us"] for L in res["layers"]) * 1e-3
+        k1_bytes = sum(L["k1_bytes"] for L in res["layers"])
+        kname = "lq_gemm_mx_kernel" if main == "mxint4" else "lq_gemm_kernel"
+        roof = {"kernel": kname + " (one launch per layer)", "bound": "tensor",
+                "achieved": achieved, "peak": burst, "unit": "TOP/s", "frac": achieved / burst,
+                "traffic": gemm_traffic_bytes(main),
+                "traffic_note": "DRAM read + write bytes of the four GEMM launches of one block from one ncu capture; null when "
+                                "the kernel source changed since",
+                "peak_source": f"2 x bf16_tflops ({peaks['bf16_tflops']}) of {peaks['source']}: 8-bit operands, nominal "
+                               f"ratio 2 to bf16",
+                "frac_of_nominal_4500": achieved / NOMINAL_8BIT_TOPS,
+                "frac_of_2x_bf16_sustained": achieved / sust,
+                "composite_bound": {"what": "sum over layers of max(t_tensor at 2 x bf16 burst, t_drain: 2 fp32 ops per output "
+                                            "and group on 148 x 128 lanes at 1965 MHz (SINT4 only), t_HBM of the GEMM)",
+                                    "bound_ms": bound_gemm_ms, "measured_ms": gemm_ms, "frac": bound_gemm_ms / gemm_ms},
+                "pair_sum_of_bounds": {"what": "quantizer HBM bound + GEMM composite bound (the two kernels run one after "
+                                               "the other)", "bound_ms": bound_gemm_ms + bound_quant_ms,
+                                       "measured_ms": gemm_ms + quant_ms,
+                                       "frac": (bound_gemm_ms + bound_quant_ms) / (gemm_ms + quant_ms)},
+                "avg_launch_ms_sum": gemm_ms}
+        roofq = {"kernel": "lq_quant_kernel (activation quantizer + down-projection, one launch per layer)", "bound": "hbm",
+                 "achieved": k1_bytes / (quant_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                 "frac": k1_bytes / (quant_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "avg_ms_sum": quant_ms}
+        return {"value": D.job_throughput(ops_step, res["steps"], res["total_ms"], world) / 1e12,
+                "ms_per_step": res["total_ms"] / res["steps"],
+                "tokens_per_s": D.job_throughput(M, res["steps"], res["total_ms"], world),
+                "roofline": roof, "roofline_quantizer": roofq}
+
+    layers = setup(args.main)
+    res = measure(args.main, layers, args.steps, True)
+    summ = summarise(args.main, res)
 
     # end to end: pinned host X -> device -> K1 -> K2 -> pinned host Y, every step
     # one stream per layer: a layer's output travels to the host while the next layer's input travels to the device
+    for L in layers:
+        L["Xp"] = torch.from_numpy(L["Xh"]).pin_memory()
+        L["Yp"] = torch.empty((M, L["spec"].N), dtype=torch.float16).pin_memory()
     e2e_streams = [torch.cuda.Stream(device=dev) for _ in layers]
 
     def e2e_step():
-        for L, es in zip(layers, e2e_streams):
-            B.lq_linear_forward_host_async(L["h"], L["act"], L["Xp"].data_ptr(), M, L["Yp"].data_ptr(), B.OUT_F16, es.cuda_stream)
+        for rep in range(repeats):
+            for L, es in zip(layers, e2e_streams):
+                B.lq_linear_forward_host_async(L["h"], L["act"], L["Xp"].data_ptr(), M, L["Yp"].data_ptr(), B.OUT_F16, es.cuda_stream)
         for es in e2e_streams:
             es.synchronize()
 
-    for _ in range(2):
+    for _ in range(1 if stack else 2):
         e2e_step()
     barrier()
-    e2e_steps = max(3, min(args.steps, 10))
+    e2e_steps = 2 if stack else max(3, min(args.steps, 10))
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
         e2e_step()
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     e2e_s = D.max_over_ranks(e2e_s, world, dev)
+    ops_step = repeats * sum(layer_ops(M, L["spec"].K, L["spec"].N, r) for L in layers)
+    specs = [L["spec"] for L in layers]
+    teardown(layers)
+
+    mx = None
+    if args.main == "sint4" and wl.config == 1 and not args.no_mxint4:
+        # the same step with the MXINT4 main branch (Table 2's format), whose block scales the tensor core applies itself
+        mx_layers = setup("mxint4")
+        mx_res = measure("mxint4", mx_layers, args.steps, True)
+        mx_s = summarise("mxint4", mx_res)
+        mx = {"what": "the same step with the MXINT4 main branch (blocks of 32, power-of-two scales, tcgen05 block-scaled MMA)",
+              "value": mx_s["value"], "unit": UNIT, "ms_per_step": mx_s["ms_per_step"], "tokens_per_s": mx_s["tokens_per_s"],
+              "roofline": mx_s["roofline"], "roofline_quantizer": mx_s["roofline_quantizer"], "layers": mx_res["layers"],
+              "clocks": mx_res["clocks"]}
+        teardown(mx_layers)
 
     if rank == 0:
-        peaks = measured_peaks()
-        peak_tops = 2.0 * peaks["bf16_tflops"]
-        gemm_avg_ms = float(np.mean(gemm_ms))
-        achieved = gops_step / (gemm_avg_ms * 1e-3) / 1e12
-        # algorithmic bytes per row of the quantizer: X read once (2K); packed 4-bit codes (K/2), 8-bit branch
-        # codes (K), fp16 group scales (2G), the per-token scale (4), r intermediate codes and their scale (4)
-        # (MXINT4: one scale byte per block of 32 instead)
-        sc_bytes = (lambda K: -(-K // 32)) if args.main == "mxint4" else (lambda K: 2 * (-(-K // 64)))
-        k1_bytes = sum(M * (2 * L["spec"].K + L["spec"].K // 2 + L["spec"].K + sc_bytes(L["spec"].K) + 4 + r + 4)
-                       for L in layers)
-        quant_avg_ms = float(np.mean(quant_ms))
+        nl = len(specs)
         line = {
-            "metric": METRIC, "value": D.job_throughput(ops_step, args.steps, total_ms_max, world) / 1e12, "unit": UNIT,
+            "metric": METRIC, "value": summ["value"], "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": total_ms_max / args.steps, "higher_is_better": True, "scaling": "weak",
+            "ms_per_step": summ["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "e4m3 (exact int4 codes) / int8 operands, fp32 accumulate", "data": "synthetic",
             "config": workload_config(wl, args),
-            "tokens_per_s": D.job_throughput(M, args.steps, total_ms_max, world),
+            "tokens_per_s": summ["tokens_per_s"],
             "e2e": {"value": D.job_throughput(ops_step, e2e_steps, e2e_s * 1e3, world) / 1e12, "unit": UNIT,
-                    "h2d_bytes_per_step": int(sum(M * L["spec"].K * 2 for L in layers)),
-                    "d2h_bytes_per_step": int(sum(M * L["spec"].N * 2 for L in layers)),
+                    "h2d_bytes_per_step": int(repeats * sum(M * sp.K * 2 for sp in specs)),
+                    "d2h_bytes_per_step": int(repeats * sum(M * sp.N * 2 for sp in specs)),
                     "ms_per_step": e2e_s / e2e_steps * 1e3},
-            "gpu_launches": args.steps * len(layers) * (3 if wl.branch == "w16a16" else 2),
-            "roofline": {"kernel": ("lq_gemm_mx_kernel" if args.main == "mxint4" else "lq_gemm_kernel") +
-                                   " (4 launches per step, one per layer)", "bound": "tensor",
-                         "achieved": achieved, "peak": peak_tops, "unit": "TOP/s", "frac": achieved / peak_tops,
-                         "traffic": gemm_traffic_bytes(args.main), "traffic_note": "DRAM read + write bytes of the four GEMM "
-                         "launches of one step from one ncu capture; null when the kernel source changed since",
-                         "peak_source": f"2 x bf16_tflops ({peaks['bf16_tflops']}) of {peaks['source']}: 8-bit operands, "
-                                        f"nominal ratio 2 to bf16",
-                         "avg_launch_ms_sum": gemm_avg_ms},
-            "roofline_quantizer": {"kernel": "lq_quant_kernel + down-projection", "bound": "hbm",
-                                   "achieved": k1_bytes / (quant_avg_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
-                                   "unit": "GB/s", "frac": k1_bytes / (quant_avg_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                                   "avg_ms_sum": quant_avg_ms},
-            "layers": per_layer,
-            "clocks": clocks,
+            "gpu_launches": args.steps * repeats * nl * 2 * (2 if mx is not None else 1),
+            "roofline": summ["roofline"],
+            "roofline_quantizer": summ["roofline_quantizer"],
+            "layers": res["layers"],
+            "clocks": res["clocks"],
         }
+        if mx is not None:
+            line["mxint4"] = mx
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(wl, I, args)
         print(json.dumps(line))
-    for L in layers:
-        B.lq_act_free(L["act"])
-        B.lq_layer_free(L["h"])
     if world > 1:
         dist.destroy_process_group()
 
@@ -400,6 +494,8 @@ def main():
                          "mxint4 = blocks of 32 with power-of-two scales applied by the tensor core")
     ap.add_argument("--calib-steps", type=int, default=2, dest="calib_steps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-mxint4", action="store_true", dest="no_mxint4",
+                    help="leave out the MXINT4 sub-record that the default (config 1, sint4) run adds")
     ap.add_argument("--l2", default="flush", choices=["flush", "working-set"],
                     help="flush: write 256 MiB before every step; working-set: rely on one step touching more than the L2 holds")
     args = ap.parse_args()

@@ -57,7 +57,8 @@ typedef enum { LQ_OUT_F16 = 0, LQ_OUT_F32 = 1 } lq_out_dtype;
 
 /* One layer's shape and calibration settings. */
 typedef struct {
-  int32_t K, N, rank; /* d, n and rho of Sections 3.1-3.2; rank in [0, 128], N even, K <= 8192    */
+  int32_t K, N, rank; /* d, n and rho of Sections 3.1-3.2; rank in [0, 128]; K and N multiples of 8,
+                         K <= 8192 (anything else: LQ_ERR_UNSUPPORTED)                              */
   int32_t group;      /* 64 = SINT4 (default), 32 = MXINT4: block length of the 4-bit main format  */
   int32_t branch;     /* an lq_branch_fmt                                                         */
   int32_t steps;      /* Adam steps on (L, R); 1000 in Appendix A "Optimization"                  */
@@ -124,7 +125,7 @@ lq_status lq_act_create(const lq_layer* layer, int32_t M_max, int device, lq_act
 lq_status lq_act_free(lq_act* act);
 
 /* Dynamic activation quantization fused with the branch's down-projection (Figure 1;
- * Appendix A.2 "Quantization": the activations forwarded to both branches are quantized).
+ * Appendix A.2 "Quantization": both the residual and the low-rank branch consume quantized X).
  * One read of X produces
  *   qx, sx   4-bit codes / scales per token and block along K (Appendix A.3): fp16 scales per
  *            block of 64 (SINT4) or one exponent byte per block of 32 (MXINT4)
@@ -132,6 +133,9 @@ lq_status lq_act_free(lq_act* act);
  *   tq, sT   per-token codes / scale of the rank-r intermediate T = deq(qb) deq(L1)
  *   X_f16_dev  [M][K] row-major half, device, 16-byte aligned
  *   M          1 <= M <= M_max of `out`
+ * X must be finite: the kernel does not look for infinities or NaNs (a row that holds one gets an
+ * undefined scale and codes; nothing is flagged).  LQ_ERR_NUMERIC is raised only by the host-side
+ * calls, for non-finite weights or scales.
  * Asynchronous on `cuda_stream` (a cudaStream_t). */
 lq_status lq_quantize_act(const lq_layer* layer, const void* X_f16_dev, int32_t M, lq_act* out,
                           void* cuda_stream);
@@ -216,8 +220,14 @@ lq_status lq_get_device_status(int device, int32_t* code, int32_t* stage);
  * Asynchronous on `cuda_stream`. */
 lq_status lq_selftest_wait_timeout(int device, void* cuda_stream);
 
-/* Tuning knobs for experiments, e.g. "main_kind" (0 = int8 operands, 1 = E4M3-carried
- * codes).  Returns INVALID_ARG for an unknown name.  Affects layers uploaded afterwards. */
+/* Process-wide switches, read when a call is made; they are plain globals, so set them while no other
+ * thread is inside the library (distinct handles may otherwise be used from distinct threads).
+ *   "store_qb"     1: lq_quantize_act also writes the branch activation codes to HBM so that lq_act_export can
+ *                  return them (parity tests); 0 (default): they stay on chip
+ *   "gemm_ctas"    CTAs of the GEMM kernels; 0 (default) = one per SM
+ *   "quant_ctas", "quant_warps"   residency and consumer warps of the quantizer kernel; 0 = chosen by the library
+ *   "main_kind"    byte format that carries the 4-bit codes into the tensor cores; only 1 (E4M3) exists
+ * Returns INVALID_ARG for an unknown name or value. */
 lq_status lq_set_option(const char* name, int32_t value);
 
 const char* lq_status_string(lq_status s);

@@ -337,6 +337,16 @@ def optimize_rotation(L, R, bits, steps: int = 500, lr: float = 0.5):
     return best[1], trace
 
 
+def adam_update(x, g, m, v, k: int, lr: float, beta1: float, beta2: float, eps: float):
+    """One Adam step (Kingma & Ba, Algorithm 1; Appendix A "Optimization" names the optimiser and the learning rate):
+    m <- b1 m + (1-b1) g,  v <- b2 v + (1-b2) g^2,  x <- x - lr (m / (1-b1^k)) / (sqrt(v / (1-b2^k)) + eps), k = 1, 2, ...
+    Returns (x, m, v)."""
+    m = beta1 * m + (1 - beta1) * g
+    v = beta2 * v + (1 - beta2) * g * g
+    x = x - lr * (m / (1 - beta1 ** k)) / (np.sqrt(v / (1 - beta2 ** k)) + eps)
+    return x, m, v
+
+
 def calibrate(W16, rank: int, branch: str = "w8a8", steps: int = 1000, lr: float = 1e-4,
               beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, bias=None, main: str = "sint4",
               rot_steps: int = 0, rot_lr: float = 0.5):
@@ -375,12 +385,8 @@ def calibrate(W16, rank: int, branch: str = "w8a8", steps: int = 1000, lr: float
             best = (loss, L.copy(), R.copy())
         if t == steps:
             break
-        k = t + 1
-        mL = beta1 * mL + (1 - beta1) * gL; vL = beta2 * vL + (1 - beta2) * gL * gL
-        mR = beta1 * mR + (1 - beta1) * gR; vR = beta2 * vR + (1 - beta2) * gR * gR
-        c1, c2 = 1 - beta1 ** k, 1 - beta2 ** k
-        L = L - lr * (mL / c1) / (np.sqrt(vL / c2) + eps)
-        R = R - lr * (mR / c1) / (np.sqrt(vR / c2) + eps)
+        L, mL, vL = adam_update(L, gL, mL, vL, t + 1, lr, beta1, beta2, eps)
+        R, mR, vR = adam_update(R, gR, mR, vR, t + 1, lr, beta1, beta2, eps)
 
     # Figure 1 sign: W ~ P + L1 L2 with L1 = -L*, L2 = R*
     L1, L2 = -best[1], best[2]

@@ -51,7 +51,7 @@ extern "C" int lq_version(void) { return 100; }
 extern "C" lq_status lq_set_option(const char* name, int32_t value) {
   if (!name) return LQ_ERR_INVALID_ARG;
   if (!strcmp(name, "main_kind")) {
-    if (value != LQ_KIND_I8 && value != LQ_KIND_E4M3) return LQ_ERR_INVALID_ARG;
+    if (value != LQ_KIND_E4M3) return LQ_ERR_INVALID_ARG;   // the only operand format the kernels are built for
     g_lq_main_kind = value;
     return LQ_OK;
   }
@@ -475,9 +475,10 @@ static lq_status forward_host(const lq_layer* L, lq_act* A, const void* Xh, int3
   cudaStream_t st = (cudaStream_t)stream;
   CUDA_OK(cudaSetDevice(A->device));
   if (!A->d_Xstage && cudaMalloc(&A->d_Xstage, (size_t)A->M_max * A->K * 2) != cudaSuccess) return LQ_ERR_ALLOC;
-  const size_t ybytes = (size_t)A->M_max * A->N * (dt == LQ_OUT_F32 ? 4 : 2);
-  if (A->ystage_bytes < ybytes) {
-    cudaFree(A->d_Ystage); A->d_Ystage = nullptr; A->ystage_bytes = 0;
+  // sized once, for the wider output type: it is never freed or re-allocated while an earlier call's copies
+  // may still be queued
+  const size_t ybytes = (size_t)A->M_max * A->N * 4;
+  if (!A->d_Ystage) {
     if (cudaMalloc(&A->d_Ystage, ybytes) != cudaSuccess) return LQ_ERR_ALLOC;
     A->ystage_bytes = ybytes;
   }

@@ -16,6 +16,7 @@
 
 #include <algorithm>
 #include <new>
+#include <memory>
 #include <vector>
 
 #include <cuda_fp16.h>
@@ -440,13 +441,14 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
   if (cfg->rank > std::min(cfg->K, cfg->N)) return LQ_ERR_INVALID_ARG;
   const int K = cfg->K, N = cfg->N;
   try {
-    lq_layer* Lr = lq_layer_new(cfg);
+    std::unique_ptr<lq_layer> owner(lq_layer_new(cfg));   // freed on every early return and on std::bad_alloc
+    lq_layer* Lr = owner.get();
     if (!Lr) return LQ_ERR_ALLOC;
     const int r = Lr->r, G = Lr->G;
     std::vector<double> W((size_t)K * N);
     for (size_t i = 0; i < W.size(); ++i) {
       const float f = half_bits_to_float(W16[i]);
-      if (!isfinite(f)) { delete Lr; return LQ_ERR_NUMERIC; }
+      if (!isfinite(f)) return LQ_ERR_NUMERIC;
       W[i] = (double)f;
     }
     if (bias16) { Lr->bias.assign(bias16, bias16 + N); Lr->has_bias = true; }
@@ -461,7 +463,7 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
         for (size_t i = 0; i < W.size(); ++i) loss += (Dq[i] - W[i]) * (Dq[i] - W[i]);
         trace[0] = loss * inv_size;
       }
-      *out = Lr;
+      *out = owner.release();
       return LQ_OK;
     }
     std::vector<double> L, R;
@@ -542,7 +544,7 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
     matmul_LR(L1d, L2d, K, N, r, D);
     for (size_t i = 0; i < A.size(); ++i) A[i] = W[i] - D[i];     // P = W - Q2(L1) Q2(L2)
     quant_main(A, K, N, Lr->Wq.data(), Lr->sw.data(), nullptr, cfg->group);
-    *out = Lr;
+    *out = owner.release();
     return LQ_OK;
   } catch (const std::bad_alloc&) {
     return LQ_ERR_ALLOC;

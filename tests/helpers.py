@@ -56,6 +56,24 @@ def rel_fro(Y, Yref) -> float:
     return float(np.linalg.norm(Y - Yref) / max(np.linalg.norm(Yref), 1e-300))
 
 
+def elementwise_excess(Y, Yref, out_f32: bool, tol: float = 1e-5) -> float:
+    """Largest |Y - Yref| in units of the element-wise bound  tol * (|y| + row scale)  (+ 2^-10 |y| when the output was
+    rounded to fp16), row scale = the largest magnitude in the reference row.  The Frobenius figure alone would hide one
+    wrong element, a missing bias or a mis-scaled column pair among 10^5 good ones; this does not.  <= 1 passes.
+    tol: 1e-5 for integer branches with SINT4 (a length-(G+1) fp32 sum of exact terms), larger where the tensor core
+    sums thousands of exact products in its own order (MXINT4) or T is rounded to fp16 on the way (W16A16)."""
+    Y = np.asarray(Y, dtype=np.float64)
+    Yref = np.asarray(Yref, dtype=np.float64)
+    scale = np.abs(Yref).max(axis=1, keepdims=True)
+    bound = tol * (np.abs(Yref) + scale) + (0.0 if out_f32 else 2.0 ** -10 * np.abs(Yref) + 2.0 ** -24)
+    return float((np.abs(Y - Yref) / np.maximum(bound, 1e-300)).max())
+
+
+def assert_y_close(Y, Yref, out_f32: bool, tol: float = 1e-5, what: str = "Y"):
+    ex = elementwise_excess(Y, Yref, out_f32, tol)
+    assert ex <= 1.0, f"{what}: element-wise bound exceeded {ex:.2f}x (tol {tol}, {'fp32' if out_f32 else 'fp16'} output)"
+
+
 def assert_codes_equal(ex: dict, ref: dict, branch: str, with_qb: bool = True):
     assert np.array_equal(ex["qx"], ref["qx"]), "qx differs"
     if "ex" in ref:                                        # MXINT4: the library exports the block exponents

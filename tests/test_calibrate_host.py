@@ -151,3 +151,25 @@ def test_rotation_aware_step_on_the_host():
     _, tr = O.optimize_rotation(L1, L2, 4, steps=60, lr=0.5)
     loss_host_0 = np.mean((O.q2_dequant(L1, 4) - L1) ** 2) + np.mean((O.q2_dequant(L2, 4) - L2) ** 2)
     assert abs(loss_host_0 - tr[0]) <= 1e-12 * tr[0] and tr.min() < tr[0]
+
+
+def test_first_adam_steps_match_the_oracle_trajectory():
+    """Two Adam steps on a small weight with well separated singular values.  The SVD start is then unique up to the
+    sign of each factor pair, a sign flip of (L_i, R_i) flips both gradients and leaves the product and the objective
+    unchanged, and two steps are far from the chaotic regime: the library's objective trace must follow the oracle's
+    (whose Adam step is pinned to its closed form in test_oracle_pins_branch_and_adam.py).  A library step without bias
+    correction, with swapped betas or with eps under the root lands on a different point and fails this."""
+    rng = np.random.default_rng(11)
+    K, N, r = 64, 32, 3
+    U, _ = np.linalg.qr(rng.standard_normal((K, N)))
+    V, _ = np.linalg.qr(rng.standard_normal((N, N)))
+    sig = np.concatenate([[0.9, 0.6, 0.35], np.linspace(0.05, 0.01, N - 3)])
+    W = ((U * sig[None, :]) @ V.T).astype(np.float16)
+    for main, group in (("sint4", 64), ("mxint4", 32)):
+        cfg = B.lq_config_default(K, N, r, "w8a8")
+        cfg.steps, cfg.group = 2, group
+        h, trace = B.lq_calibrate(cfg, W, want_trace=True)
+        _, tr_o = O.calibrate(W, r, "w8a8", steps=2, main=main)
+        assert np.allclose(trace, tr_o, rtol=1e-7, atol=0), (main, trace, tr_o)
+        assert abs(tr_o[1] - tr_o[0]) > 1e-4 * tr_o[0]     # the step is visible in the objective
+        B.lq_layer_free(h)
