@@ -33,9 +33,11 @@
 // Every wait is bounded as in lq_gemm.cu.
 #include <cuda_fp16.h>
 
-#include "lq_internal.h"
+#include "lq_device.cuh"
 
 namespace {
+
+using namespace lqdev;
 
 constexpr int UNIT = LQ_BN;                        // 128 output columns
 constexpr int NSTAGE = 4;                          // operand ring depth
@@ -53,7 +55,6 @@ constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + NSTAGE * STAGE_BYTES + NST
                            SMEM_BAR_BYTES;
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 static_assert(STAGE_BYTES % 1024 == 0, "stages must keep the 1024-byte alignment of the swizzled tiles");
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s at 2 GHz
 // tensor-memory columns: main accumulator [0, 256), branch accumulator [256, 512); 4 columns of A scales and 8 of B
 // scales alias the start of the branch accumulator (disjoint lifetimes, see the top of the file)
 constexpr int TM_BR = 256, TM_SFA = 256, TM_SFB = TM_SFA + 4, TM_SF_ALIASED = 16;
@@ -75,128 +76,6 @@ struct MxParams {
   int32_t* status;
 };
 
-// ---- PTX wrappers -------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.b32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
-// Bounded wait.  Returns false when the CTA is aborting or the deadline passed (then it
-// raises the abort flag and records who gave up).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                            int role, long long limit = WAIT_LIMIT_CYCLES) {
-  const long long t0 = clock64();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 0xFF) == 0) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > limit) {
-        *abort_flag = 1;
-        if (atomicCAS(status, 0, (int)LQ_ERR_TIMEOUT) == 0) status[1] = role;
-        return false;
-      }
-    }
-  }
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                          int role) {
-  if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, status, role);
-}
-// Wait of a role that is idle for a long time (the drain during a tile's main loop): polling at full speed would take
-// issue slots from the producer and the MMA issuer that share its scheduler, so it sleeps between polls.
-__device__ __forceinline__ bool mbar_wait_idle(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                               int role) {
-  for (int i = 0; i < 64; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    __nanosleep(200);
-  }
-  return mbar_wait_slow(bar, parity, abort_flag, status, role);
-}
-// The same wait for a whole warp whose control flow must stay provably uniform (the producer
-// and the MMA warp keep their loop state in uniform registers).
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                               int role) {
-  const bool ok = mbar_wait(bar, parity, abort_flag, status, role);
-  return __all_sync(0xffffffffu, ok);
-}
-
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.b32 %0, 1, 0, P;\n\t}" : "=r"(pred));
-  return pred != 0;
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
-               : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-template <int KIND>   // 0: i8, 1: f8f6f4, 2: f16
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  if constexpr (KIND == 0) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-  } else if constexpr (KIND == 1) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-  } else {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-  }
-}
-
-// 16 lanes x 32 consecutive 32-bit columns in the accumulator-fragment layout of mma.sync m16n8: with g = lane / 4 and
-// t = lane % 4, registers 4j .. 4j+3 hold (row g, columns 8j + 2t, 8j + 2t + 1) and (row g + 8, the same columns).
-__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&v)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr)
-      : "memory");
-}
 // 4 x 4 transpose across the four lanes of a quad: afterwards v[s] of lane t is what v[t] of lane s was.
 __device__ __forceinline__ void quad_transpose(uint32_t (&v)[4], int t) {
   const bool hi2 = (t & 2) != 0, hi1 = (t & 1) != 0;
@@ -207,53 +86,6 @@ __device__ __forceinline__ void quad_transpose(uint32_t (&v)[4], int t) {
   y1 = __shfl_xor_sync(0xffffffffu, hi1 ? v[2] : v[3], 1);
   if (hi1) { v[0] = y0; v[2] = y1; } else { v[1] = y0; v[3] = y1; }
 }
-__device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, uint32_t (&v)[8]) {
-  asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
-               : "r"(taddr)
-               : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
-// 8-row atoms 1024 bytes apart.  Adding (bytes >> 4) steps along K inside the swizzled row.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
-  const uint32_t lo = ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16);          // start address, LBO = 1 (unused)
-  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);              // SBO = 1024 B, version 1, SWIZZLE_128B
-  return ((uint64_t)hi << 32) | lo;
-}
-
-// instruction descriptor: accumulator format, operand formats, N >> 3 at bit 17, M >> 4 at bit 24
-__device__ __forceinline__ constexpr uint32_t idesc_shape(int n) { return ((uint32_t)(n >> 3) << 17) | ((uint32_t)(LQ_BM >> 4) << 24); }
-constexpr uint32_t IDESC_I8 = (2u << 4) | (1u << 7) | (1u << 10);    // S8 x S8 -> S32
-constexpr uint32_t IDESC_F8 = (1u << 4) | (0u << 7) | (0u << 10);    // E4M3 x E4M3 -> F32
-constexpr uint32_t IDESC_F16 = (1u << 4) | (0u << 7) | (0u << 10);   // F16 x F16 -> F32
-
-
-// Shared-memory matrix descriptor without swizzle (K-major, 8-row x 16-byte core matrices stored contiguously).
-__device__ __forceinline__ uint64_t make_smem_desc_plain(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
-  const uint32_t lo = ((smem_addr & 0x3FFFFu) >> 4) | ((lbo >> 4) << 16);
-  const uint32_t hi = (sbo >> 4) | (1u << 14);                             // version 1, no swizzle
-  return ((uint64_t)hi << 32) | lo;
-}
-// 32 rows x 16 bytes of shared memory -> 4 tensor-memory columns, replicated into the four 32-lane quarters
-__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
-  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
-}
-// block-scaled MMA: E4M3 operands, E8M0 scales (one per row and 32-deep K block) read from tensor memory
-__device__ __forceinline__ void tc_mma_mx(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t tsfa,
-                                          uint32_t tsfb, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
-      : "memory");
-}
-// instruction descriptor of the block-scaled kind: E4M3 x E4M3, E8M0 scales, K-major operands, scale-byte ids
-__device__ __forceinline__ constexpr uint32_t idesc_mx(int n, int sf_id) {
-  return ((uint32_t)sf_id << 4) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(LQ_BM >> 4) << 24) | ((uint32_t)sf_id << 29);
-}
-
 // y = main + U sT sL2 + bias for one n8 fragment (registers: row g columns 2t, 2t+1, then row g + 8 the same columns).
 // U is an exact int32 with |U| < 2^22: converted exactly with the 1.5 * 2^23 trick.
 __device__ __forceinline__ void combine_fragment(float (&a)[4], const uint32_t* u, bool has_branch, float st_lo, float st_hi,
@@ -324,12 +156,10 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     for (int b = 0; b < 2; ++b) { mbar_init(bar(B_RFULL + b), 1); mbar_init(bar(B_REMPTY + b), NUM_DRAIN_WARPS); }
     mbar_init(bar(B_BEMPTY), NUM_DRAIN_WARPS);
     *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_init_fence();
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    tmem_alloc(smem_u32(tmem_slot), 512);
   }
   tc_fence_before();
   __syncthreads();
@@ -441,8 +271,8 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
         if (elect_one()) {
           for (int j = 0; j < p.branch_steps; ++j) {
-            if (branch_acc) tc_mma<0>(tmem_base + TM_BR, adesc + 2 * j, bdesc + 2 * j, IDESC_I8 | idesc_shape(ncols), (uint32_t)j);
-            else tc_mma<2>(tmem_base, adesc + 2 * j, bdesc + 2 * j, IDESC_F16 | idesc_shape(ncols), 1u);   // 16 halves each
+            if (branch_acc) tc_mma<TC_I8>(tmem_base + TM_BR, adesc + 2 * j, bdesc + 2 * j, IDESC_I8 | idesc_shape(ncols), (uint32_t)j);
+            else tc_mma<TC_F16>(tmem_base, adesc + 2 * j, bdesc + 2 * j, IDESC_F16 | idesc_shape(ncols), 1u);   // 16 halves each
           }
           tc_commit(bar(B_EMPTY + st));
         }
@@ -585,7 +415,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    tmem_dealloc(tmem_base, 512);
   }
 }
 
