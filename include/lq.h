@@ -50,8 +50,21 @@ typedef enum {
   LQ_BRANCH_W16A16 = 1, /* fp16 factors, fp16 activations (reference variant)  */
   LQ_BRANCH_W8A8 = 2,
   LQ_BRANCH_W6A6 = 3,
-  LQ_BRANCH_W4A8 = 4
+  LQ_BRANCH_W4A8 = 4,
+  /* MX branches of the mixed-precision study (Section 4.3, Tables 3-4; Appendix A.3 "MX Formats"): factors in
+   * blocks of 32 with a power-of-two scale and e4m3 / e2m3 / e2m1 elements; the activations of BOTH branches and
+   * the rank-r intermediate are MXFP8e4.  Only with main_fmt = LQ_MAIN_MXFP4. */
+  LQ_BRANCH_MXFP8 = 5,
+  LQ_BRANCH_MXFP6 = 6,
+  LQ_BRANCH_MXFP4 = 7
 } lq_branch_fmt;
+
+/* 4-bit format of the residual (main) branch, Appendix A.3. */
+typedef enum {
+  LQ_MAIN_AUTO = 0,    /* from `group`: 64 -> SINT4 (integer codes, fp16 scale per 64), 32 -> MXINT4           */
+  LQ_MAIN_MXFP4 = 2    /* MXFP4e2 weights (e2m1 elements, power-of-two scale per 32; group must be 32) times
+                          MXFP8e4 activations, all scales applied by the tensor core (Tables 3-4)              */
+} lq_main_fmt;
 
 typedef enum { LQ_OUT_F16 = 0, LQ_OUT_F32 = 1 } lq_out_dtype;
 
@@ -67,6 +80,8 @@ typedef struct {
   int32_t rot_steps;  /* steps of the rotation-aware optimisation of Section 3.3; 0 (default) = none,  */
   float rot_lr;       /* 500 steps at 0.5 (0.1 for the mixed-precision study) in Appendix A           */
   uint64_t seed;      /* start vectors of the host SVD iteration                                  */
+  int32_t main_fmt;   /* an lq_main_fmt; 0 (default) = SINT4 / MXINT4 as `group` says                */
+  int32_t reserved;   /* 0                                                                          */
 } lq_config;
 
 typedef struct lq_layer lq_layer; /* opaque: Q1(P) codes+scales, Q2(L1), Q2(L2), bias (Figure 1)  */
@@ -101,7 +116,14 @@ lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W_f16_host,
  *   L1, L2    integer branches: int8 codes [K][rank] and [rank][N]; W16A16: half bits, same shapes
  *   sL1, sL2  fp32 per-column scales [rank] and [N]; NULL for W16A16
  *   bias      [N] half bits or NULL
- * With rank == 0 or LQ_BRANCH_NONE the branch pointers are ignored. */
+ * With rank == 0 or LQ_BRANCH_NONE the branch pointers are ignored.
+ * MXFP layers (main_fmt = LQ_MAIN_MXFP4; the library has no host calibration for them: calibrate elsewhere, import
+ * here; lq_calibrate returns UNSUPPORTED):
+ *   Wq_packed [K][N/2] bytes: e2m1 bit patterns (sign, two exponent bits, one mantissa bit) as nibbles, same order
+ *   sw        [ceil(K/32)][N] half bits: the block's power-of-two scale 2^e, e in [-24, 15]
+ *   L1, L2    [K][rank] and [rank][N] bytes: e4m3 bit patterns of the elements (every e2m3 and e2m1 value is an
+ *             e4m3 value, so the three MXFP branch formats arrive in one encoding)
+ *   sL1, sL2  fp32 powers of two: [ceil(K/32)][rank] (blocks of L1 along K) and [ceil(rank/32)][N] (of L2 along rank) */
 lq_status lq_layer_import(const lq_config* cfg, const uint8_t* Wq_packed, const uint16_t* sw,
                           const void* L1, const float* sL1, const void* L2, const float* sL2,
                           const uint16_t* bias, lq_layer** out);

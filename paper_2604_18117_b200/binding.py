@@ -15,7 +15,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liblq.so")
 
 LQ_OK = 0
-BRANCH = {"none": 0, "w16a16": 1, "w8a8": 2, "w6a6": 3, "w4a8": 4}
+BRANCH = {"none": 0, "w16a16": 1, "w8a8": 2, "w6a6": 3, "w4a8": 4, "mxfp8": 5, "mxfp6": 6, "mxfp4": 7}
+MAIN_AUTO, MAIN_MXFP4 = 0, 2
 BRANCH_NAME = {v: k for k, v in BRANCH.items()}
 OUT_F16, OUT_F32 = 0, 1
 GROUP = 64
@@ -25,7 +26,7 @@ class LqConfig(C.Structure):
     _fields_ = [("K", C.c_int32), ("N", C.c_int32), ("rank", C.c_int32), ("group", C.c_int32),
                 ("branch", C.c_int32), ("steps", C.c_int32), ("lr", C.c_float), ("beta1", C.c_float),
                 ("beta2", C.c_float), ("eps", C.c_float), ("rot_steps", C.c_int32), ("rot_lr", C.c_float),
-                ("seed", C.c_uint64)]
+                ("seed", C.c_uint64), ("main_fmt", C.c_int32), ("reserved", C.c_int32)]
 
 
 class LqError(RuntimeError):
@@ -124,6 +125,48 @@ def unpack_nibbles(P: np.ndarray) -> np.ndarray:
     return out
 
 
+# ---- e4m3 / e2m1 byte formats (layout only: the bit patterns of the OCP element formats; no method arithmetic) ----
+def _e4m3_table() -> np.ndarray:
+    """Value of each of the 256 e4m3 bit patterns (bias 7, subnormals, no infinities; 0x7F / 0xFF are NaN)."""
+    t = np.zeros(256, dtype=np.float32)
+    for b in range(256):
+        e, m = (b >> 3) & 0xF, b & 7
+        v = m / 8.0 * 2.0 ** -6 if e == 0 else (1 + m / 8.0) * 2.0 ** (e - 7)
+        t[b] = np.nan if (b & 0x7F) == 0x7F else (-v if b & 0x80 else v)
+    return t
+
+
+E4M3_VALUES = _e4m3_table()
+
+
+def e4m3_decode(codes: np.ndarray) -> np.ndarray:
+    """uint8 / int8 e4m3 bit patterns -> float32 values."""
+    return E4M3_VALUES[np.asarray(codes).view(np.uint8)]
+
+
+def e4m3_encode(values: np.ndarray) -> np.ndarray:
+    """float values that are exactly representable in e4m3 -> their bit patterns (uint8); raises otherwise."""
+    v = np.asarray(values, dtype=np.float32)
+    pos = E4M3_VALUES[:0x7F]                                   # ascending non-negative values
+    idx = np.searchsorted(pos, np.abs(v))
+    idx = np.minimum(idx, 0x7E)
+    if not np.array_equal(pos[idx], np.abs(v)):
+        raise ValueError("value not representable in e4m3")
+    return (idx.astype(np.uint8) | np.where(np.signbit(v), 0x80, 0).astype(np.uint8)).astype(np.uint8)
+
+
+def pack_e2m1(values: np.ndarray) -> np.ndarray:
+    """e2m1 element values [K, N] -> nibbles [K, N/2] (sign, two exponent bits, one mantissa bit), column 2j low."""
+    grid = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6], dtype=np.float32)
+    v = np.asarray(values, dtype=np.float32)
+    idx = np.searchsorted(grid, np.abs(v))
+    idx = np.minimum(idx, 7)
+    if not np.array_equal(grid[idx], np.abs(v)):
+        raise ValueError("value not representable in e2m1")
+    nib = (idx | np.where(np.signbit(v) & (v != 0), 8, 0)).astype(np.uint8)
+    return np.ascontiguousarray(nib[:, 0::2] | (nib[:, 1::2] << 4))
+
+
 def lq_layer_import(cfg: LqConfig, Wq_packed, sw, L1=None, sL1=None, L2=None, sL2=None, bias=None):
     """All arguments are host numpy arrays in the layouts include/lq.h documents."""
     arrs = [np.ascontiguousarray(a) if a is not None else None for a in (Wq_packed, sw, L1, sL1, L2, sL2, bias)]
@@ -144,7 +187,10 @@ def lq_layer_export(layer) -> dict:
     out = {"Wq_packed": np.zeros((K, N // 2), np.uint8), "sw": np.zeros((G, N), np.float16),
            "bias": np.zeros(N, np.float16), "branch": BRANCH_NAME[cfg.branch], "rank": r, "K": K, "N": N}
     L1 = L2 = sL1 = sL2 = None
-    if r > 0 and cfg.branch == BRANCH["w16a16"]:
+    if cfg.main_fmt == MAIN_MXFP4 and r > 0:
+        L1, L2 = np.zeros((K, r), np.uint8), np.zeros((r, N), np.uint8)               # e4m3 bit patterns
+        sL1, sL2 = np.zeros((G, r), np.float32), np.zeros((-(-r // 32), N), np.float32)
+    elif r > 0 and cfg.branch == BRANCH["w16a16"]:
         L1, L2 = np.zeros((K, r), np.float16), np.zeros((r, N), np.float16)
     elif r > 0:
         L1, L2 = np.zeros((K, r), np.int8), np.zeros((r, N), np.int8)
@@ -204,6 +250,16 @@ def lq_linear_forward_static(layer, X_dev_ptr: int, M: int, Y_dev_ptr: int, dtyp
 
 def lq_act_export(act, M: int, cfg: LqConfig, stream: int = 0) -> dict:
     K, r, G = cfg.K, cfg.rank, -(-cfg.K // cfg.group)
+    if cfg.main_fmt == MAIN_MXFP4:
+        # MXFP: qx / tq are e4m3 bit patterns (decode with e4m3_decode), sx the int16 block exponents of X,
+        # sT the block exponents of the rank-r intermediate as floats [M, ceil(r/32)]
+        out = {"qx": np.zeros((M, K), np.int8), "sx": np.zeros((M, G), np.int16), "qb": None, "sXb": None, "tq": None, "sT": None}
+        if r > 0 and cfg.branch != BRANCH["none"]:
+            out["tq"] = np.zeros((M, r), np.int8)
+            out["sT"] = np.zeros((M, -(-r // 32)), np.float32)
+        _check(lib().lq_act_export(act, _np_ptr(out["qx"]), _np_ptr(out["sx"]), None, None, _np_ptr(out["tq"]),
+                                   _np_ptr(out["sT"]), C.c_void_p(stream)), "lq_act_export")
+        return out
     # SINT4: fp16 group scales; MXINT4 (group 32): int16 block exponents e (scale 2^e)
     out = {"qx": np.zeros((M, K), np.int8), "sx": np.zeros((M, G), np.int16 if cfg.group == 32 else np.float16)}
     qb = sXb = tq = sT = None

@@ -83,14 +83,21 @@ extern "C" lq_status lq_config_default(lq_config* cfg, int32_t K, int32_t N, int
   cfg->K = K; cfg->N = N; cfg->rank = rank; cfg->group = LQ_GROUP; cfg->branch = branch;
   cfg->steps = 1000; cfg->lr = 1e-4f; cfg->beta1 = 0.9f; cfg->beta2 = 0.999f; cfg->eps = 1e-8f;
   cfg->rot_steps = 0; cfg->rot_lr = 0.5f; cfg->seed = 0;
+  cfg->main_fmt = LQ_MAIN_AUTO; cfg->reserved = 0;
+  if (lq_branch_is_mxfp(branch)) { cfg->main_fmt = LQ_MAIN_MXFP4; cfg->group = LQ_MX_BLOCK; cfg->lr = 1e-3f; }
   return LQ_OK;
 }
 
 static lq_status check_config(const lq_config* c) {
   if (!c) return LQ_ERR_INVALID_ARG;
   if (c->K <= 0 || c->N <= 0 || c->rank < 0) return LQ_ERR_INVALID_ARG;
-  if (c->branch < LQ_BRANCH_NONE || c->branch > LQ_BRANCH_W4A8) return LQ_ERR_INVALID_ARG;
+  if (c->branch < LQ_BRANCH_NONE || c->branch > LQ_BRANCH_MXFP4) return LQ_ERR_INVALID_ARG;
   if (c->group != LQ_GROUP && c->group != LQ_MX_BLOCK) return LQ_ERR_UNSUPPORTED;
+  if (c->main_fmt != LQ_MAIN_AUTO && c->main_fmt != LQ_MAIN_MXFP4) return LQ_ERR_INVALID_ARG;
+  // MXFP4 weights go with blocks of 32 and an MXFP (or no) branch; MXFP branches go with nothing else
+  if (c->main_fmt == LQ_MAIN_MXFP4 && (c->group != LQ_MX_BLOCK || !(c->branch == LQ_BRANCH_NONE || lq_branch_is_mxfp(c->branch))))
+    return LQ_ERR_UNSUPPORTED;
+  if (c->main_fmt != LQ_MAIN_MXFP4 && lq_branch_is_mxfp(c->branch)) return LQ_ERR_UNSUPPORTED;
   if (c->K > LQ_MAX_K || (c->K % 8) != 0) return LQ_ERR_UNSUPPORTED;
   if ((c->N % 8) != 0) return LQ_ERR_UNSUPPORTED;
   if (c->rank > LQ_MAX_RANK) return LQ_ERR_UNSUPPORTED;
@@ -109,18 +116,39 @@ lq_layer* lq_layer_new(const lq_config* cfg) {
   if (L->r == 0) L->cfg.branch = LQ_BRANCH_NONE;
   L->cfg.rank = L->r;
   L->mx = cfg->group == LQ_MX_BLOCK;
+  L->mxfp = cfg->main_fmt == LQ_MAIN_MXFP4;
   L->G = lq_ceil_div(L->K, cfg->group);
   L->Kpad = lq_round_up(L->K, LQ_KSTAGE);
   L->Gpad = L->Kpad / LQ_GROUP;
   L->Npad = lq_round_up(L->N, LQ_BN);
-  L->integer_branch = L->r > 0 && L->cfg.branch != LQ_BRANCH_W16A16;
+  L->integer_branch = L->r > 0 && L->cfg.branch != LQ_BRANCH_W16A16 && !lq_branch_is_mxfp(L->cfg.branch);
   L->f16_branch = L->r > 0 && L->cfg.branch == LQ_BRANCH_W16A16;
   L->has_bias = false;
   L->device = -1;
   L->main_kind = g_lq_main_kind;
   L->d_Wq8 = nullptr; L->d_sw = nullptr; L->d_L1f = nullptr; L->d_L1h = nullptr; L->d_sL1 = nullptr;
   L->d_L2c = nullptr; L->d_sL2 = nullptr; L->d_bias = nullptr; L->d_sfb = nullptr;
+  L->d_s1b = nullptr; L->d_sfl2 = nullptr;
   return L;
+}
+
+// e2m1 bit pattern (sign, two exponent bits, one mantissa bit) -> the e4m3 byte of the same value
+static inline uint8_t e2m1_to_e4m3(int nib) {
+  static const uint8_t mag[8] = {0x00, 0x30, 0x38, 0x3C, 0x40, 0x44, 0x48, 0x4C};   // 0, 0.5, 1, 1.5, 2, 3, 4, 6
+  return (uint8_t)(mag[nib & 7] | ((nib & 8) ? 0x80 : 0));
+}
+static inline int e4m3_to_e2m1(uint8_t b) {
+  static const uint8_t mag[8] = {0x00, 0x30, 0x38, 0x3C, 0x40, 0x44, 0x48, 0x4C};
+  for (int i = 0; i < 8; ++i)
+    if ((b & 0x7F) == mag[i]) return i | ((b & 0x80) ? 8 : 0);
+  return -1;
+}
+// power of two held in a float -> its exponent (false if the value is not a positive power of two)
+static inline bool pow2_exponent(float v, int* e) {
+  int x = 0;
+  if (!(v > 0.f) || !isfinite(v) || frexpf(v, &x) != 0.5f) return false;
+  *e = x - 1;
+  return true;
 }
 
 extern "C" lq_status lq_layer_import(const lq_config* cfg, const uint8_t* Wq_packed, const uint16_t* sw,
@@ -134,6 +162,39 @@ extern "C" lq_status lq_layer_import(const lq_config* cfg, const uint8_t* Wq_pac
   const int K = L->K, N = L->N, r = L->r, G = L->G;
   if (r > 0 && (!L1 || !L2)) { delete L; return LQ_ERR_INVALID_ARG; }
   if (L->integer_branch && (!sL1 || !sL2)) { delete L; return LQ_ERR_INVALID_ARG; }
+  if (L->mxfp) {
+    const int nbK = lq_ceil_div(K, LQ_MX_BLOCK), nbR = lq_ceil_div(r > 0 ? r : 1, LQ_MX_BLOCK);
+    if (r > 0 && (!sL1 || !sL2)) { delete L; return LQ_ERR_INVALID_ARG; }
+    try {
+      L->Wq8h.resize((size_t)K * N);
+      for (int k = 0; k < K; ++k)
+        for (int j = 0; j < N / 2; ++j) {
+          const uint8_t b = Wq_packed[(size_t)k * (N / 2) + j];
+          L->Wq8h[(size_t)k * N + 2 * j] = e2m1_to_e4m3(b & 0xF);
+          L->Wq8h[(size_t)k * N + 2 * j + 1] = e2m1_to_e4m3(b >> 4);
+        }
+      L->sw.assign(sw, sw + (size_t)G * N);
+      for (size_t i = 0; i < L->sw.size(); ++i) {
+        int e = 0;
+        if (!pow2_exponent(h2f(L->sw[i]), &e)) { delete L; return LQ_ERR_INVALID_ARG; }
+      }
+      if (r > 0) {
+        const uint8_t* a = (const uint8_t*)L1; const uint8_t* b = (const uint8_t*)L2;
+        L->L1e.assign(a, a + (size_t)K * r);
+        L->L2e.assign(b, b + (size_t)r * N);
+        for (uint8_t v : L->L1e) if ((v & 0x7F) == 0x7F) { delete L; return LQ_ERR_NUMERIC; }   // e4m3 NaN
+        for (uint8_t v : L->L2e) if ((v & 0x7F) == 0x7F) { delete L; return LQ_ERR_NUMERIC; }
+        L->s1b.assign(sL1, sL1 + (size_t)nbK * r);
+        L->s2b.assign(sL2, sL2 + (size_t)nbR * N);
+        int e = 0;
+        for (float v : L->s1b) if (!pow2_exponent(v, &e)) { delete L; return LQ_ERR_INVALID_ARG; }
+        for (float v : L->s2b) if (!pow2_exponent(v, &e) || e < -127 || e > 127) { delete L; return LQ_ERR_INVALID_ARG; }
+      }
+      if (bias) { L->bias.assign(bias, bias + N); L->has_bias = true; }
+    } catch (const std::bad_alloc&) { delete L; return LQ_ERR_ALLOC; }
+    *out = L;
+    return LQ_OK;
+  }
   try {
     L->Wq.resize((size_t)K * N);
     for (int k = 0; k < K; ++k)
@@ -178,6 +239,22 @@ extern "C" lq_status lq_layer_export(const lq_layer* L, uint8_t* Wq_packed, uint
                                      float* sL1, void* L2, float* sL2, uint16_t* bias) {
   if (!L) return LQ_ERR_INVALID_ARG;
   const int K = L->K, N = L->N, r = L->r;
+  if (L->mxfp) {
+    if (Wq_packed)
+      for (int k = 0; k < K; ++k)
+        for (int j = 0; j < N / 2; ++j)
+          Wq_packed[(size_t)k * (N / 2) + j] = (uint8_t)(e4m3_to_e2m1(L->Wq8h[(size_t)k * N + 2 * j]) |
+                                                         (e4m3_to_e2m1(L->Wq8h[(size_t)k * N + 2 * j + 1]) << 4));
+    if (sw) memcpy(sw, L->sw.data(), L->sw.size() * sizeof(uint16_t));
+    if (r > 0) {
+      if (L1) memcpy(L1, L->L1e.data(), L->L1e.size());
+      if (L2) memcpy(L2, L->L2e.data(), L->L2e.size());
+      if (sL1) memcpy(sL1, L->s1b.data(), L->s1b.size() * sizeof(float));
+      if (sL2) memcpy(sL2, L->s2b.data(), L->s2b.size() * sizeof(float));
+    }
+    if (bias && L->has_bias) memcpy(bias, L->bias.data(), N * sizeof(uint16_t));
+    return LQ_OK;
+  }
   if (Wq_packed)
     for (int k = 0; k < K; ++k)
       for (int j = 0; j < N / 2; ++j) {
@@ -291,6 +368,8 @@ static void layer_free_device(lq_layer* L) {
   cudaSetDevice(L->device);
   cudaFree(L->d_Wq8); cudaFree(L->d_sw); cudaFree(L->d_L1f); cudaFree(L->d_L1h); cudaFree(L->d_sL1);
   cudaFree(L->d_L2c); cudaFree(L->d_sL2); cudaFree(L->d_bias); cudaFree(L->d_sfb);
+  cudaFree(L->d_s1b); cudaFree(L->d_sfl2);
+  L->d_s1b = nullptr; L->d_sfl2 = nullptr;
   L->d_Wq8 = nullptr; L->d_sw = nullptr; L->d_L1f = nullptr; L->d_L1h = nullptr; L->d_sL1 = nullptr;
   L->d_L2c = nullptr; L->d_sL2 = nullptr; L->d_bias = nullptr; L->d_sfb = nullptr;
   L->device = -1;
@@ -316,7 +395,8 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
   try {
     std::vector<uint8_t> w8((size_t)Npad * Kpad, lq_encode_code_host(0, L->main_kind));
     for (int k = 0; k < K; ++k)
-      for (int n = 0; n < N; ++n) w8[(size_t)n * Kpad + k] = lq_encode_code_host(L->Wq[(size_t)k * N + n], L->main_kind);
+      for (int n = 0; n < N; ++n)
+        w8[(size_t)n * Kpad + k] = L->mxfp ? L->Wq8h[(size_t)k * N + n] : lq_encode_code_host(L->Wq[(size_t)k * N + n], L->main_kind);
     if ((st = upload(&L->d_Wq8, w8)) != LQ_OK) return st;
     if (L->mx) {
       // E8M0 bytes (exponent + 127) in the layout the block-scaled MMA reads from tensor memory; 127 = 2^0 for padding
@@ -356,6 +436,38 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
       for (int n = 0; n < N; ++n) s2[n] = L->sL2[n];
       for (int j = 0; j < r; ++j)
         for (int n = 0; n < N; ++n) l2c[(size_t)n * LQ_RCONT + j] = (uint8_t)L->L2q[(size_t)j * N + n];
+    } else if (L->mxfp && r > 0) {
+      // B fragments of mma.sync.m16n8k32 (e4m3) for the MXFP quantizer, whose lanes hold two runs of eight values per
+      // box (one per block of 32): lane 4 c + t carries k = 64 box + 32 j + 8 t + 0..7 of column 8 tile + c, j = 0, 1
+      const int ntiles = lq_quant_rank_tiles(r, false), nbox = Kpad / 64, rpad = ntiles * 8;
+      std::vector<uint8_t> l1f((size_t)nbox * ntiles * 32 * 16, 0);
+      for (int b = 0; b < nbox; ++b)
+        for (int nt = 0; nt < ntiles; ++nt)
+          for (int lane = 0; lane < 32; ++lane) {
+            const int j = nt * 8 + (lane >> 2);
+            uint8_t* dst = &l1f[(((size_t)b * ntiles + nt) * 32 + lane) * 16];
+            for (int blk = 0; blk < 2; ++blk)
+              for (int i = 0; i < 8; ++i) {
+                const int k = b * 64 + 32 * blk + 8 * (lane & 3) + i;
+                dst[8 * blk + i] = (j < r && k < K) ? L->L1e[(size_t)k * r + j] : 0;
+              }
+          }
+      if ((st = upload(&L->d_L1f, l1f)) != LQ_OK) return st;
+      std::vector<float> s1b((size_t)(Kpad / 32) * rpad, 0.f);
+      for (int b = 0; b < lq_ceil_div(K, 32); ++b)
+        for (int j = 0; j < r; ++j) s1b[(size_t)b * rpad + j] = L->s1b[(size_t)b * r + j];
+      if ((st = upload(&L->d_s1b, s1b)) != LQ_OK) return st;
+      for (int j = 0; j < r; ++j)
+        for (int n = 0; n < N; ++n) l2c[(size_t)n * LQ_RCONT + j] = L->L2e[(size_t)j * N + n];
+      // E8M0 bytes of L2's block scales along the rank, one 128-byte-of-rank stage: [1][Npad/128][512]
+      std::vector<uint8_t> sfl2((size_t)(Npad / 128) * 512, 127);
+      for (int c = 0; c < lq_ceil_div(r, 32); ++c)
+        for (int n = 0; n < N; ++n) {
+          int e = 0;
+          pow2_exponent(L->s2b[(size_t)c * N + n], &e);
+          sfl2[lq_sfb_offset(n, c, Npad)] = (uint8_t)(e + 127);
+        }
+      if ((st = upload(&L->d_sfl2, sfl2)) != LQ_OK) return st;
     } else if (L->f16_branch) {
       // the same fragment order with 16 halves per lane (mma.sync.m16n8k16, four k steps per box)
       const int ntiles = lq_quant_rank_tiles(r, true), nbox = Kpad / 64;
@@ -400,7 +512,7 @@ extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device,
   if (!A) return LQ_ERR_ALLOC;
   memset(A, 0, sizeof(*A));
   A->K = L->K; A->N = L->N; A->r = L->r; A->G = L->G; A->Kpad = L->Kpad; A->Gpad = L->Gpad;
-  A->mx = L->mx;
+  A->mx = L->mx; A->mxfp = L->mxfp;
   A->branch = L->cfg.branch; A->M_max = M_max; A->Mpad = lq_round_up(M_max, LQ_BM);
   A->device = device; A->main_kind = L->main_kind; A->M = 0;
   if (cudaSetDevice(device) != cudaSuccess) { delete A; return LQ_ERR_CUDA; }
@@ -411,7 +523,8 @@ extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device,
             cudaMalloc((void**)&A->d_sXb, Mp * sizeof(float)) == cudaSuccess &&
             cudaMalloc((void**)&A->d_tq, Mp * LQ_RCONT) == cudaSuccess &&
             cudaMalloc((void**)&A->d_sT, Mp * sizeof(float)) == cudaSuccess &&
-            (!A->mx || cudaMalloc((void**)&A->d_sfa, (Mp / 128) * (Kp / 128) * 512) == cudaSuccess);
+            (!A->mx || cudaMalloc((void**)&A->d_sfa, (Mp / 128) * (Kp / 128) * 512) == cudaSuccess) &&
+            (!A->mxfp || cudaMalloc((void**)&A->d_sft, (Mp / 128) * 512) == cudaSuccess);
   if (!ok) { lq_act_free(A); return LQ_ERR_ALLOC; }
   // padding rows/columns are read by the GEMM's tiles: start from defined contents
   cudaMemset(A->d_qx8, 0, Mp * Kp);
@@ -421,6 +534,7 @@ extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device,
   cudaMemset(A->d_tq, 0, Mp * LQ_RCONT);
   cudaMemset(A->d_sT, 0, Mp * sizeof(float));
   if (A->mx) cudaMemset(A->d_sfa, 127, (Mp / 128) * (Kp / 128) * 512);
+  if (A->mxfp) cudaMemset(A->d_sft, 127, (Mp / 128) * 512);
   lq_status st;
   if ((st = lq_make_tmap_bytes(&A->tmA, A->d_qx8, Mp, Kp, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
   if ((st = lq_make_tmap_bytes(&A->tmT, A->d_tq, Mp, LQ_RCONT, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
@@ -432,7 +546,7 @@ extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device,
 extern "C" lq_status lq_act_free(lq_act* A) {
   if (!A) return LQ_ERR_INVALID_ARG;
   cudaSetDevice(A->device);
-  cudaFree(A->d_qx8); cudaFree(A->d_sx); cudaFree(A->d_qb); cudaFree(A->d_sXb); cudaFree(A->d_tq); cudaFree(A->d_sT); cudaFree(A->d_sfa);
+  cudaFree(A->d_qx8); cudaFree(A->d_sx); cudaFree(A->d_qb); cudaFree(A->d_sXb); cudaFree(A->d_tq); cudaFree(A->d_sT); cudaFree(A->d_sfa); cudaFree(A->d_sft);
   cudaFree(A->d_Xstage); cudaFree(A->d_Ystage);
   if (A->pipe_ready) {
     cudaStreamDestroy(A->s_h2d); cudaStreamDestroy(A->s_d2h);
@@ -445,7 +559,7 @@ extern "C" lq_status lq_act_free(lq_act* A) {
 
 static bool act_matches(const lq_layer* L, const lq_act* A) {
   return L && A && L->device == A->device && L->device >= 0 && L->K == A->K && L->N == A->N && L->r == A->r &&
-         L->cfg.branch == A->branch && L->main_kind == A->main_kind && L->mx == A->mx;
+         L->cfg.branch == A->branch && L->main_kind == A->main_kind && L->mx == A->mx && L->mxfp == A->mxfp;
 }
 
 extern "C" lq_status lq_quantize_act(const lq_layer* L, const void* X, int32_t M, lq_act* A, void* stream) {
@@ -521,6 +635,7 @@ static lq_status forward_host(const lq_layer* L, lq_act* A, const void* Xh, int3
     V.d_tq = A->d_tq + (size_t)m0 * LQ_RCONT;
     V.d_sT = A->d_sT + m0;
     if (A->mx) V.d_sfa = A->d_sfa + (size_t)(m0 / 128) * (A->Kpad / 128) * 512;
+    if (A->mxfp) V.d_sft = A->d_sft + (size_t)(m0 / 128) * 512;
     lq_status s;
     if ((s = lq_make_tmap_bytes(&V.tmA, V.d_qx8, (uint64_t)(A->Mpad - m0), A->Kpad, LQ_BM)) != LQ_OK) return s;
     if ((s = lq_make_tmap_bytes(&V.tmT, V.d_tq, (uint64_t)(A->Mpad - m0), LQ_RCONT, LQ_BM)) != LQ_OK) return s;
@@ -571,7 +686,8 @@ extern "C" lq_status lq_act_export(const lq_act* A, int8_t* qx, uint16_t* sx, in
       std::vector<uint8_t> h((size_t)M * Kp);
       CUDA_OK(cudaMemcpy(h.data(), A->d_qx8, h.size(), cudaMemcpyDeviceToHost));
       for (int m = 0; m < M; ++m)
-        for (int k = 0; k < K; ++k) qx[(size_t)m * K + k] = (int8_t)decode_code(h[m * Kp + k], A->main_kind);
+        for (int k = 0; k < K; ++k)   // MXFP: the e4m3 bytes themselves
+          qx[(size_t)m * K + k] = A->mxfp ? (int8_t)h[m * Kp + k] : (int8_t)decode_code(h[m * Kp + k], A->main_kind);
     }
     if (sx && A->mx) {
       std::vector<uint8_t> h((Mp / 128) * (Kp / 128) * 512);
@@ -590,19 +706,26 @@ extern "C" lq_status lq_act_export(const lq_act* A, int8_t* qx, uint16_t* sx, in
           sx[(size_t)m * G + g] = __half_raw(v).x;
         }
     }
-    if (qb && A->branch != LQ_BRANCH_NONE && A->branch != LQ_BRANCH_W16A16) {
+    if (qb && A->branch != LQ_BRANCH_NONE && A->branch != LQ_BRANCH_W16A16 && !A->mxfp) {
       std::vector<int8_t> h((size_t)M * Kp);
       CUDA_OK(cudaMemcpy(h.data(), A->d_qb, h.size(), cudaMemcpyDeviceToHost));
       for (int m = 0; m < M; ++m) memcpy(qb + (size_t)m * K, h.data() + m * Kp, K);
     }
-    if (sXb && r > 0) CUDA_OK(cudaMemcpy(sXb, A->d_sXb, M * sizeof(float), cudaMemcpyDeviceToHost));
+    if (sXb && r > 0 && !A->mxfp) CUDA_OK(cudaMemcpy(sXb, A->d_sXb, M * sizeof(float), cudaMemcpyDeviceToHost));
     if (tq && r > 0) {
       std::vector<uint8_t> h((size_t)M * LQ_RCONT);
       CUDA_OK(cudaMemcpy(h.data(), A->d_tq, h.size(), cudaMemcpyDeviceToHost));
       const int eb = A->branch == LQ_BRANCH_W16A16 ? 2 : 1;
       for (int m = 0; m < M; ++m) memcpy((uint8_t*)tq + (size_t)m * r * eb, h.data() + (size_t)m * LQ_RCONT, (size_t)r * eb);
     }
-    if (sT && r > 0) CUDA_OK(cudaMemcpy(sT, A->d_sT, M * sizeof(float), cudaMemcpyDeviceToHost));
+    if (sT && r > 0 && A->mxfp) {
+      // MXFP: the block exponents of the rank-r intermediate as floats, [M][ceil(r/32)]
+      std::vector<uint8_t> h((Mp / 128) * 512);
+      CUDA_OK(cudaMemcpy(h.data(), A->d_sft, h.size(), cudaMemcpyDeviceToHost));
+      const int nbR = lq_ceil_div(r, LQ_MX_BLOCK);
+      for (int m = 0; m < M; ++m)
+        for (int c = 0; c < nbR; ++c) sT[(size_t)m * nbR + c] = (float)((int)h[lq_sf_offset(m, c, 128)] - 127);
+    } else if (sT && r > 0) CUDA_OK(cudaMemcpy(sT, A->d_sT, M * sizeof(float), cudaMemcpyDeviceToHost));
   } catch (const std::bad_alloc&) { return LQ_ERR_ALLOC; }
   return LQ_OK;
 }

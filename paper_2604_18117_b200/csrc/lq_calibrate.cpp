@@ -434,7 +434,8 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
                                   double* trace) {
   if (!cfg || !W16 || !out) return LQ_ERR_INVALID_ARG;
   if (cfg->K <= 0 || cfg->N <= 0 || cfg->rank < 0 || cfg->steps < 0) return LQ_ERR_INVALID_ARG;
-  if (cfg->branch < LQ_BRANCH_NONE || cfg->branch > LQ_BRANCH_W4A8) return LQ_ERR_INVALID_ARG;
+  if (cfg->branch < LQ_BRANCH_NONE || cfg->branch > LQ_BRANCH_MXFP4) return LQ_ERR_INVALID_ARG;
+  if (cfg->main_fmt == LQ_MAIN_MXFP4 || lq_branch_is_mxfp(cfg->branch)) return LQ_ERR_UNSUPPORTED;   // MXFP layers are imported
   if ((cfg->group != LQ_GROUP && cfg->group != LQ_MX_BLOCK) || cfg->rot_steps < 0) return LQ_ERR_UNSUPPORTED;
   if (cfg->K > LQ_MAX_K || (cfg->K % 8) || (cfg->N % 8) || cfg->rank > LQ_MAX_RANK) return LQ_ERR_UNSUPPORTED;
   if (cfg->branch == LQ_BRANCH_W16A16 && cfg->rank > 64) return LQ_ERR_UNSUPPORTED;

@@ -64,6 +64,9 @@ struct MxParams {
   int k_stages;           // Kpad / 128
   int branch_steps;       // 0: no branch; else MMAs of the branch stage (32 bytes of r each)
   int branch_f16;         // the branch operands are halves (W16A16 reference branch): no scales, summed by the tensor core
+  int branch_mx;          // the branch is MXFP as well: its up-projection is one more block-scaled stage onto the main accumulator
+  const uint8_t* sft;     // branch_mx: E8M0 bytes of T's block scales, [Mpad/128][512]
+  const uint8_t* sfl2;    // branch_mx: E8M0 bytes of L2's block scales, [Npad/128][512]
   int tiles_m, units_n;
   int by_units;           // how the CTAs share the work: 0 whole tiles, 1 128-column units
   const uint8_t* sfa;     // [Mpad/128][k_stages][512]
@@ -127,7 +130,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const bool has_branch = p.branch_steps > 0;
   // An fp16 branch has no scales: its product is accumulated onto the main accumulator by the tensor core and the drain
   // sees no branch at all.  An integer branch needs its fp32 scales applied per element: second accumulator.
-  const bool branch_acc = has_branch && !p.branch_f16;
+  const bool branch_acc = has_branch && !p.branch_f16 && !p.branch_mx;
   // Each CTA takes a contiguous, equal share of the work and walks it as 256-wide tiles (128-wide where a row block or
   // the share ends).  A 128-wide tile costs nearly as much as a 256-wide one (a stage's time is set by its hand-shakes
   // and instruction count, not its MMA width).  by_units = 0 shares whole tiles - row blocks cut into 256-wide tiles
@@ -212,10 +215,15 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const uint32_t a_dst = sm_stage + st * STAGE_BYTES, b_dst = a_dst + STAGE_A_BYTES;
         const uint32_t full = bar(B_FULL + st);
         if (elect_one()) {
-          mbar_expect_tx(full, STAGE_A_BYTES + width * (UNIT * LQ_KSTAGE));
+          mbar_expect_tx(full, STAGE_A_BYTES + width * (UNIT * LQ_KSTAGE) + (p.branch_mx ? (1 + width) * SF_BYTES : 0));
           tma_load_2d(a_dst, &tmT, 0, m0, full);
           tma_load_2d(b_dst, &tmL2, 0, n0, full);
           if (width == 2) tma_load_2d(b_dst + UNIT * LQ_KSTAGE, &tmL2, 0, n0 + UNIT, full);
+          if (p.branch_mx) {   // the block scales of T (rows) and of L2 (columns) along the rank
+            const uint32_t sf_dst = sm_sf + st * STAGE_SF_BYTES;
+            bulk_load(sf_dst, p.sft + (size_t)mb * SF_BYTES, SF_BYTES, full);
+            bulk_load(sf_dst + SF_BYTES, p.sfl2 + (size_t)nu * SF_BYTES, width * SF_BYTES, full);
+          }
         }
         __syncwarp();
         ++it;
@@ -270,9 +278,18 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const uint32_t a_addr = sm_stage + st * STAGE_BYTES, b_addr = a_addr + STAGE_A_BYTES;
         const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
         if (elect_one()) {
-          for (int j = 0; j < p.branch_steps; ++j) {
-            if (branch_acc) tc_mma<TC_I8>(tmem_base + TM_BR, adesc + 2 * j, bdesc + 2 * j, IDESC_I8 | idesc_shape(ncols), (uint32_t)j);
-            else tc_mma<TC_F16>(tmem_base, adesc + 2 * j, bdesc + 2 * j, IDESC_F16 | idesc_shape(ncols), 1u);   // 16 halves each
+          if (p.branch_mx) {
+            const uint32_t sf_addr = sm_sf + st * STAGE_SF_BYTES, tsfa = tmem_base + TM_SFA, tsfb = tmem_base + TM_SFB;
+            tc_cp_sf(tsfa, make_smem_desc_plain(sf_addr, 16, 128));
+            tc_cp_sf(tsfb, make_smem_desc_plain(sf_addr + SF_BYTES, 16, 128));
+            if (width == 2) tc_cp_sf(tsfb + 4, make_smem_desc_plain(sf_addr + 2 * SF_BYTES, 16, 128));
+            for (int j = 0; j < p.branch_steps; ++j)
+              tc_mma_mx(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc_mx(ncols, j), tsfa, tsfb, 1u);
+          } else {
+            for (int j = 0; j < p.branch_steps; ++j) {
+              if (branch_acc) tc_mma<TC_I8>(tmem_base + TM_BR, adesc + 2 * j, bdesc + 2 * j, IDESC_I8 | idesc_shape(ncols), (uint32_t)j);
+              else tc_mma<TC_F16>(tmem_base, adesc + 2 * j, bdesc + 2 * j, IDESC_F16 | idesc_shape(ncols), 1u);   // 16 halves each
+            }
           }
           tc_commit(bar(B_EMPTY + st));
         }
@@ -436,6 +453,8 @@ lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_
   p.M = A->M; p.N = L->N; p.Mpad = A->Mpad; p.Npad = L->Npad;
   p.k_stages = L->Kpad / LQ_KSTAGE;
   p.branch_f16 = L->f16_branch ? 1 : 0;
+  p.branch_mx = (L->mxfp && L->r > 0) ? 1 : 0;
+  p.sft = A->d_sft; p.sfl2 = L->d_sfl2;
   p.branch_steps = L->r == 0 ? 0 : lq_ceil_div(L->r, L->f16_branch ? 16 : 32);
   p.tiles_m = lq_ceil_div(A->M, LQ_BM);
   p.units_n = L->Npad / UNIT;

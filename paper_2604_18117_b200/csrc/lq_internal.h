@@ -37,6 +37,9 @@ static inline size_t lq_sfb_offset(int n, int kb, int Npad) {
   return ((size_t)(kb / 4) * (Npad / 128) + n / 128) * 512 + 16 * (n % 32) + 4 * ((n % 128) / 32) + kb % 4;
 }
 
+static inline bool lq_branch_is_mxfp(int branch) {
+  return branch == LQ_BRANCH_MXFP8 || branch == LQ_BRANCH_MXFP6 || branch == LQ_BRANCH_MXFP4;
+}
 static inline int lq_branch_wbits(int branch) {
   return branch == LQ_BRANCH_W8A8 ? 8 : branch == LQ_BRANCH_W6A6 ? 6 : branch == LQ_BRANCH_W4A8 ? 4 : 0;
 }
@@ -49,7 +52,11 @@ struct lq_layer {
   int K, N, r, G;          // logical sizes
   int Kpad, Npad, Gpad;    // Kpad: multiple of 128; Npad: multiple of LQ_BN; Gpad = Kpad / 64
   bool integer_branch, f16_branch, has_bias;
-  bool mx;                     // MXINT4 main branch (cfg.group == 32): G counts blocks of 32, sw holds powers of two
+  bool mx;                     // MX main branch (cfg.group == 32): G counts blocks of 32, sw holds powers of two
+  bool mxfp;                   // MXFP4 weights x MXFP8e4 activations (implies mx); the branch, if any, is MXFP too
+  std::vector<uint8_t> Wq8h;   // mxfp: [K][N] e4m3 bytes of the e2m1 weight elements
+  std::vector<uint8_t> L1e, L2e;   // mxfp: e4m3 bytes of the factor elements, [K][r] and [r][N]
+  std::vector<float> s1b, s2b; // mxfp: block scales 2^e of L1 [ceil(K/32)][r] and of L2 [ceil(r/32)][N]
   // host copy, canonical layouts
   std::vector<int8_t> Wq;      // [K][N]
   std::vector<uint16_t> sw;    // [G][N] half bits
@@ -71,6 +78,8 @@ struct lq_layer {
   uint8_t* d_L2c;              // [Npad][LQ_RCONT] bytes: int8 codes (or up to 64 halves) of column n, r contiguous
   float* d_sL2;                // [Npad]  (ones for W16A16)
   float* d_bias;               // [Npad]  (zeros without bias)
+  float* d_s1b;                // mxfp: 2^e1 [Kpad/32][rpad] (zero-padded columns)
+  uint8_t* d_sfl2;             // mxfp: E8M0 bytes of L2's block scales, [1][Npad/128][512] in the tensor-memory layout
   uint8_t* d_sfb;              // MXINT4: E8M0 bytes of the weight scales, [Kpad/128][Npad/128][512] in the 32 x 16-byte
                                // layout tensor memory wants (byte 16*(n%32) + 4*((n%128)/32) + block%4)
   CUtensorMap tmB;             // over d_Wq8, box [LQ_BN][128B], 128B swizzle
@@ -80,8 +89,9 @@ struct lq_layer {
 
 struct lq_act {
   int K, N, r, G, Kpad, Gpad, branch;
-  bool mx;
-  uint8_t* d_sfa;              // MXINT4: E8M0 bytes of the activation scales, [Mpad/128][Kpad/128][512], same layout
+  bool mx, mxfp;
+  uint8_t* d_sft;              // mxfp: E8M0 bytes of the rank-r intermediate's block scales, [Mpad/128][1][512]
+  uint8_t* d_sfa;              // MX: E8M0 bytes of the activation scales, [Mpad/128][Kpad/128][512], same layout
   int M_max, Mpad, device, main_kind;
   int M;                       // rows of the last lq_quantize_act
   uint8_t* d_qx8;              // [Mpad][Kpad] operand bytes of the 4-bit codes (A operand, K-major)

@@ -35,7 +35,7 @@ extern "C" lq_status lq_linear_forward_static(const lq_layer* L, const void* X, 
   if (!L || !X || !Y) return LQ_ERR_INVALID_ARG;
   if (L->device < 0 || L->device >= 64) return LQ_ERR_INVALID_ARG;      // layer not uploaded
   if (M <= 0) return LQ_ERR_INVALID_ARG;
-  if (L->mx) return LQ_ERR_UNSUPPORTED;                                 // SINT4 layers only
+  if (L->mx || L->mxfp) return LQ_ERR_UNSUPPORTED;                      // SINT4 layers only
   if (dt != LQ_OUT_F16 && dt != LQ_OUT_F32) return LQ_ERR_INVALID_ARG;
   if ((((uintptr_t)X) & 15) != 0 || (((uintptr_t)Y) & 15) != 0) return LQ_ERR_INVALID_ARG;
 

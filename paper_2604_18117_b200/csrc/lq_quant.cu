@@ -39,7 +39,8 @@ constexpr int BOX_K = 64;              // values of K per box: one 128-byte swiz
 constexpr int BOX_BYTES = TR * BOX_K * 2;
 constexpr float MAGIC = 12582912.0f;   // 1.5 * 2^23: adding it rounds to an integer (ties to even)
 constexpr int MAX_CONSUMER_WARPS = 9;
-enum { BR_NONE = 0, BR_INT = 1, BR_F16 = 2 };
+enum { BR_NONE = 0, BR_INT = 1, BR_F16 = 2, BR_MXFP = 3 };
+enum { MAIN_SINT4 = 0, MAIN_MXINT4 = 1, MAIN_MXFP = 2 };   // MXFP: MXFP8e4 activation codes for an MXFP4 weight
 
 struct QuantParams {
   int M, K, Kpad, Mpad;
@@ -55,6 +56,8 @@ struct QuantParams {
   float* sXb;           // [Mpad]
   const uint4* L1f;     // first factor in fragment order: [nbox][r tiles][32 lanes] x 16 bytes (int8) or 32 bytes (fp16)
   const float* sL1;     // [LQ_MAX_RANK]
+  const float* s1b;     // MXFP: block scales 2^e of the first factor, [Kpad/32][rpad]
+  uint8_t* sft;         // MXFP: E8M0 bytes of the rank-r intermediate's block scales, [Mpad/128][512]
   uint8_t* tq;          // [Mpad][LQ_RCONT]
   float* sT;            // [Mpad]
   int r, rpad;          // rank, rank rounded up to 8
@@ -82,6 +85,12 @@ __device__ __forceinline__ void mma_s8_16832(int (&c)[4], uint32_t a0, uint32_t 
       : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void mma_e4m3_16832(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                               uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ void mma_f16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                               uint32_t b1) {
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -97,6 +106,37 @@ __device__ __forceinline__ __half absmax16(const uint4& a, const uint4& b) {
   m = __hmax2(m, __hmax2(__hmax2(__habs2(q[0]), __habs2(q[1])), __hmax2(__habs2(q[2]), __habs2(q[3]))));
   return __hmax(__low2half(m), __high2half(m));
 }
+
+__device__ __forceinline__ __half absmax8(const uint4& a) {
+  const __half2* p = reinterpret_cast<const __half2*>(&a);
+  const __half2 m = __hmax2(__hmax2(__habs2(p[0]), __habs2(p[1])), __hmax2(__habs2(p[2]), __habs2(p[3])));
+  return __hmax(__low2half(m), __high2half(m));
+}
+
+// MXFP8e4 of eight values that share a block (Appendix A.3 "MX Formats"; conversion of the OCP specification the
+// paper cites): the block's exponent is e = floor(log2 a) - 8 for the block maximum a (e4m3's largest binade is 2^8),
+// -127 for an all-zero block; the elements are x / 2^e - exact - rounded to e4m3 by the hardware conversion
+// (nearest even, magnitudes above 448 clamped).  Returns the eight e4m3 bytes.
+__device__ __forceinline__ int mxfp8_exponent(float a) {
+  const int e = (int)(__float_as_uint(a) >> 23) - 127 - 8;
+  return (a > 0.f && e >= -126) ? e : -127;
+}
+__device__ __forceinline__ uint2 mxfp8_codes8(const uint4& v, int e) {
+  const __half2* h2 = reinterpret_cast<const __half2*>(&v);
+  const float inv = e == -127 ? 0.f : __uint_as_float((uint32_t)(127 - e) << 23);
+  float x[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __half22float2(h2[i]);
+    x[2 * i] = f.x * inv; x[2 * i + 1] = f.y * inv;
+  }
+  uint2 w;
+  w.x = f32x2_to_e4m3x2(x[1], x[0]) | (f32x2_to_e4m3x2(x[3], x[2]) << 16);
+  w.y = f32x2_to_e4m3x2(x[5], x[4]) | (f32x2_to_e4m3x2(x[7], x[6]) << 16);
+  return w;
+}
+// 2^e as a float (0 for the all-zero block's -127: its codes are zeros anyway)
+__device__ __forceinline__ float pow2f(int e) { return e <= -127 ? 0.f : __uint_as_float((uint32_t)(e + 127) << 23); }
 
 // Correctly rounded quotient a / b in binary32 from the correctly rounded reciprocal y = fl32(1/b), division free:
 // q0 = fl32(a y) is within one ulp of a / b, r = a - b q0 is exact in an FMA, and fl32(q0 + r y) is then the
@@ -190,9 +230,12 @@ __device__ __forceinline__ bool consumers_sync(uint32_t bar, uint32_t parity, in
 //   red       BR_INT: int I1[2][16][rpad]; BR_F16: float part[W][16][rpad]
 //   rowmax    int[2][16] (bit patterns of non-negative floats)
 //   abort     int
-template <bool MX, int BR, int NTR>   // NTR: 8-column tiles of the rank (rank <= 8 NTR)
+template <int MAIN, int BR, int NTR>   // NTR: 8-column tiles of the rank (rank <= 8 NTR)
 __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_kernel(const __grid_constant__ CUtensorMap tmX,
                                                                                  const QuantParams p) {
+  constexpr bool MX = MAIN == MAIN_MXINT4;
+  constexpr bool FP = MAIN == MAIN_MXFP;
+  constexpr bool FACC = BR == BR_F16 || BR == BR_MXFP;     // fp32 partial sums of the down-projection
   extern __shared__ uint8_t qsm_raw[];
   const uint32_t base = (smem_u32(qsm_raw) + 1023u) & ~1023u;
   uint8_t* smem = qsm_raw + (base - smem_u32(qsm_raw));
@@ -209,7 +252,7 @@ __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_ker
   uint8_t* red_ptr = smem + (size_t)nslot * BOX_BYTES + 16 * (size_t)nslot + 32;
   int* I1_s = reinterpret_cast<int*>(red_ptr);
   float* part_s = reinterpret_cast<float*>(red_ptr);
-  const size_t red_bytes = BR == BR_INT ? (size_t)2 * TR * p.rpad * 4 : BR == BR_F16 ? (size_t)W * TR * p.rpad * 4 : 0;
+  const size_t red_bytes = BR == BR_INT ? (size_t)2 * TR * p.rpad * 4 : FACC ? (size_t)W * TR * p.rpad * 4 : 0;
   int* rowmax_s = reinterpret_cast<int*>(red_ptr + red_bytes);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(rowmax_s + 2 * TR);
 
@@ -267,7 +310,8 @@ __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_ker
     };
     // this lane's two 16-byte chunks of a swizzled 128-byte row; rows gid and gid + 8 share the swizzle phase
     const uint32_t row_off = (uint32_t)gid * 128u;
-    const uint32_t c0 = (uint32_t)((2 * tig) ^ (gid & 7)) << 4, c1 = (uint32_t)((2 * tig + 1) ^ (gid & 7)) << 4;
+    // (MXFP: one 16-byte chunk from each of the box's two blocks of 32 instead: values 8 tig .. and 32 + 8 tig ..)
+    const uint32_t c0 = (uint32_t)((FP ? tig : 2 * tig) ^ (gid & 7)) << 4, c1 = (uint32_t)((FP ? 4 + tig : 2 * tig + 1) ^ (gid & 7)) << 4;
     uint32_t sync_par = 0;
     uint32_t tcount = 0;
     bool ok = true;
@@ -319,13 +363,13 @@ __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_ker
       }
       // ---- walk 2: codes, scales, down-projection
       int acci[BR == BR_INT ? NTR : 1][4];
-      float accf[BR == BR_F16 ? NTR : 1][4];
+      float accf[FACC ? NTR : 1][4];
 #pragma unroll
       for (int a = 0; a < NTR; ++a)
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
           if constexpr (BR == BR_INT) acci[a][b] = 0;
-          if constexpr (BR == BR_F16) accf[a][b] = 0.f;
+          if constexpr (FACC) accf[a][b] = 0.f;
         }
       {
         // First-factor fragments (read-only, shared by all CTAs, L2 resident) travel one box ahead of their use: the
@@ -350,6 +394,57 @@ __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_ker
           if (lane == 0) mbar_arrive(bar_empty(s0 + idx));   // the values are in registers: the slot may be refilled
           advance();
           const size_t koff = (size_t)(g * BOX_K);             // this box's first value of a row
+          if constexpr (FP) {
+            // l0 / h0: eight values of block 2g, l1 / h1: of block 2g + 1; a block's maximum lives in four lanes
+            float a00 = __half2float(absmax8(l0)), a01 = __half2float(absmax8(l1));
+            float a10 = __half2float(absmax8(h0)), a11 = __half2float(absmax8(h1));
+#pragma unroll
+            for (int o = 1; o <= 2; o <<= 1) {
+              a00 = fmaxf(a00, __shfl_xor_sync(0xffffffffu, a00, o)); a01 = fmaxf(a01, __shfl_xor_sync(0xffffffffu, a01, o));
+              a10 = fmaxf(a10, __shfl_xor_sync(0xffffffffu, a10, o)); a11 = fmaxf(a11, __shfl_xor_sync(0xffffffffu, a11, o));
+            }
+            const int e00 = mxfp8_exponent(a00), e01 = mxfp8_exponent(a01), e10 = mxfp8_exponent(a10), e11 = mxfp8_exponent(a11);
+            const uint2 w00 = mxfp8_codes8(l0, e00), w01 = mxfp8_codes8(l1, e01);
+            const uint2 w10 = mxfp8_codes8(h0, e10), w11 = mxfp8_codes8(h1, e11);
+            uint8_t* q_lo = p.qx8 + (size_t)m_lo * p.Kpad + koff + 8 * tig;
+            uint8_t* q_hi = q_lo + (size_t)8 * p.Kpad;
+            if (v_lo) { *reinterpret_cast<uint2*>(q_lo) = w00; *reinterpret_cast<uint2*>(q_lo + 32) = w01; }
+            if (v_hi) { *reinterpret_cast<uint2*>(q_hi) = w10; *reinterpret_cast<uint2*>(q_hi + 32) = w11; }
+            if (tig == 0) {
+              const int kb = 2 * g;                            // blocks kb, kb + 1 share a 4-block scale chunk
+              if (kb < p.G) {
+                if (v_lo) {
+                  uint8_t* sf = p.sfa + ((size_t)(m_lo >> 7) * (p.Kpad >> 7) + (kb >> 2)) * 512 + 16 * (m_lo & 31) + 4 * ((m_lo & 127) >> 5) + (kb & 3);
+                  sf[0] = (uint8_t)(e00 + 127);
+                  if (kb + 1 < p.G) sf[1] = (uint8_t)(e01 + 127);
+                }
+                if (v_hi) {
+                  uint8_t* sf = p.sfa + ((size_t)(m_hi >> 7) * (p.Kpad >> 7) + (kb >> 2)) * 512 + 16 * (m_hi & 31) + 4 * ((m_hi & 127) >> 5) + (kb & 3);
+                  sf[0] = (uint8_t)(e10 + 127);
+                  if (kb + 1 < p.G) sf[1] = (uint8_t)(e11 + 127);
+                }
+              }
+            }
+            if constexpr (BR == BR_MXFP) {
+              // a3: per block of 32 one MMA step on the codes just made (their bytes ARE the A fragments), the block's
+              // two power-of-two scales applied to its partial sums in fp32
+              const float sa00 = pow2f(e00), sa01 = pow2f(e01), sa10 = pow2f(e10), sa11 = pow2f(e11);
+#pragma unroll
+              for (int nt = 0; nt < NTR; ++nt) {
+                const float2 sb0 = __ldg(reinterpret_cast<const float2*>(p.s1b + (size_t)(2 * g) * p.rpad + nt * 8 + 2 * tig));
+                const float2 sb1 = __ldg(reinterpret_cast<const float2*>(p.s1b + (size_t)(2 * g + 1) * p.rpad + nt * 8 + 2 * tig));
+                float f0[4] = {0.f, 0.f, 0.f, 0.f}, f1[4] = {0.f, 0.f, 0.f, 0.f};
+                mma_e4m3_16832(f0, w00.x, w10.x, w00.y, w10.y, bfrag[nt].x, bfrag[nt].y);
+                mma_e4m3_16832(f1, w01.x, w11.x, w01.y, w11.y, bfrag[nt].z, bfrag[nt].w);
+                accf[nt][0] = fmaf(f0[0], sa00 * sb0.x, fmaf(f1[0], sa01 * sb1.x, accf[nt][0]));
+                accf[nt][1] = fmaf(f0[1], sa00 * sb0.y, fmaf(f1[1], sa01 * sb1.y, accf[nt][1]));
+                accf[nt][2] = fmaf(f0[2], sa10 * sb0.x, fmaf(f1[2], sa11 * sb1.x, accf[nt][2]));
+                accf[nt][3] = fmaf(f0[3], sa10 * sb0.y, fmaf(f1[3], sa11 * sb1.y, accf[nt][3]));
+              }
+            }
+            if (g + W < p.nbox) load_frags(g + W);
+            continue;
+          }
           uint4 w_lo, w_hi, b_lo = make_uint4(0, 0, 0, 0), b_hi = make_uint4(0, 0, 0, 0);
           // group maxima: 64 values = four lanes (SINT4), 32 values = two lanes (MXINT4)
           float a_lo = __half2float(absmax16(l0, l1)), a_hi = __half2float(absmax16(h0, h1));
@@ -486,6 +581,22 @@ __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_ker
               }
             }
           }
+        } else if constexpr (BR == BR_MXFP) {
+          // T = deq(Q(X)) deq(Q2(L1)) in fp32 (the warps' partial sums added in warp order), then MXFP8e4 along the rank:
+          // one block of 32 per warp pass, its maximum by a warp reduction
+          if (m < p.M) {
+            for (int c = 0; c * 32 < p.r; ++c) {
+              const int j = c * 32 + lane;
+              float v = 0.f;
+              if (j < p.rpad)
+                for (int w2 = 0; w2 < W; ++w2) v += part_s[((size_t)w2 * TR + rl) * p.rpad + j];
+              if (j >= p.r) v = 0.f;
+              const int e = mxfp8_exponent(warp_max(fabsf(v)));
+              const float inv = e == -127 ? 0.f : __uint_as_float((uint32_t)(127 - e) << 23);
+              p.tq[(size_t)m * LQ_RCONT + j] = (uint8_t)(f32x2_to_e4m3x2(0.f, v * inv) & 0xFF);
+              if (lane == 0) p.sft[(size_t)(m >> 7) * 512 + 16 * (m & 31) + 4 * ((m & 127) >> 5) + c] = (uint8_t)(e + 127);
+            }
+          }
         } else {
           // T = fp16(X L1): the warps' fp32 partial sums are added in warp order (the result does not depend on timing)
           if (m < p.M) {
@@ -498,7 +609,7 @@ __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_ker
           }
         }
       }
-      if constexpr (BR == BR_F16) {
+      if constexpr (FACC) {
         ok = consumers_sync(bar_sync + 16, sync_par, lane, abort_flag, p.status);   // partial sums may be overwritten
         if (!ok) break;
       }
@@ -526,7 +637,7 @@ LaunchPlan plan_launch(int nbox, int br, int rpad, int regs) {
       if (g_lq_quant_warps > 0 ? W != g_lq_quant_warps : W < 8) continue;
       const int threads = (W + 1) * 32;
       if (ctas * threads > 2048 || ctas * threads * ((regs + 7) / 8 * 8) > 65536) continue;
-      const size_t red = br == BR_INT ? (size_t)2 * TR * rpad * 4 : br == BR_F16 ? (size_t)W * TR * rpad * 4 : 0;
+      const size_t red = br == BR_INT ? (size_t)2 * TR * rpad * 4 : (br == BR_F16 || br == BR_MXFP) ? (size_t)W * TR * rpad * 4 : 0;
       const size_t fixed = 1024 + 64 + red + 2 * TR * 4 + 64;
       const size_t budget = std::min(SM_SMEM, SM_SMEM / ctas - 1024);
       if (budget < fixed + (size_t)W * (BOX_BYTES + 16)) continue;
@@ -547,17 +658,17 @@ LaunchPlan plan_launch(int nbox, int br, int rpad, int regs) {
   return best;
 }
 
-template <bool MX, int BR, int NTR>
+template <int MAIN, int BR, int NTR>
 cudaError_t launch_quant(const CUtensorMap& tm, QuantParams& p, int sms, cudaStream_t st) {
   static bool attr_set[64] = {false};
   static int regs[64] = {0};
   int dev = 0;
   cudaGetDevice(&dev);
   if (!attr_set[dev & 63]) {
-    cudaError_t e = cudaFuncSetAttribute(lq_quant_kernel<MX, BR, NTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(lq_quant_kernel<MAIN, BR, NTR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     cudaFuncAttributes fa;
-    if ((e = cudaFuncGetAttributes(&fa, lq_quant_kernel<MX, BR, NTR>)) != cudaSuccess) return e;
+    if ((e = cudaFuncGetAttributes(&fa, lq_quant_kernel<MAIN, BR, NTR>)) != cudaSuccess) return e;
     regs[dev & 63] = fa.numRegs;
     attr_set[dev & 63] = true;
   }
@@ -566,22 +677,29 @@ cudaError_t launch_quant(const CUtensorMap& tm, QuantParams& p, int sms, cudaStr
   p.depth = pl.depth; p.refetch = pl.refetch;
   int grid = sms * pl.ctas_per_sm;
   if (grid > p.ntiles) grid = p.ntiles;
-  lq_quant_kernel<MX, BR, NTR><<<grid, (pl.W + 1) * 32, pl.smem, st>>>(tm, p);
+  lq_quant_kernel<MAIN, BR, NTR><<<grid, (pl.W + 1) * 32, pl.smem, st>>>(tm, p);
   return cudaGetLastError();
 }
 
-template <bool MX>
+template <int MAIN>
 cudaError_t dispatch_quant(int br, int ntr, const CUtensorMap& tm, QuantParams& p, int sms, cudaStream_t st) {
-  if (br == BR_NONE) return launch_quant<MX, BR_NONE, 1>(tm, p, sms, st);
-  if (br == BR_INT) {
-    if (ntr <= 2) return launch_quant<MX, BR_INT, 2>(tm, p, sms, st);
-    if (ntr <= 4) return launch_quant<MX, BR_INT, 4>(tm, p, sms, st);
-    if (ntr <= 8) return launch_quant<MX, BR_INT, 8>(tm, p, sms, st);
-    return launch_quant<MX, BR_INT, 16>(tm, p, sms, st);
+  if (br == BR_NONE) return launch_quant<MAIN, BR_NONE, 1>(tm, p, sms, st);
+  if constexpr (MAIN == MAIN_MXFP) {
+    if (ntr <= 2) return launch_quant<MAIN, BR_MXFP, 2>(tm, p, sms, st);
+    if (ntr <= 4) return launch_quant<MAIN, BR_MXFP, 4>(tm, p, sms, st);
+    if (ntr <= 8) return launch_quant<MAIN, BR_MXFP, 8>(tm, p, sms, st);
+    return launch_quant<MAIN, BR_MXFP, 16>(tm, p, sms, st);
+  } else {
+    if (br == BR_INT) {
+      if (ntr <= 2) return launch_quant<MAIN, BR_INT, 2>(tm, p, sms, st);
+      if (ntr <= 4) return launch_quant<MAIN, BR_INT, 4>(tm, p, sms, st);
+      if (ntr <= 8) return launch_quant<MAIN, BR_INT, 8>(tm, p, sms, st);
+      return launch_quant<MAIN, BR_INT, 16>(tm, p, sms, st);
+    }
+    if (ntr <= 2) return launch_quant<MAIN, BR_F16, 2>(tm, p, sms, st);
+    if (ntr <= 4) return launch_quant<MAIN, BR_F16, 4>(tm, p, sms, st);
+    return launch_quant<MAIN, BR_F16, 8>(tm, p, sms, st);
   }
-  if (ntr <= 2) return launch_quant<MX, BR_F16, 2>(tm, p, sms, st);
-  if (ntr <= 4) return launch_quant<MX, BR_F16, 4>(tm, p, sms, st);
-  return launch_quant<MX, BR_F16, 8>(tm, p, sms, st);
 }
 
 }  // namespace
@@ -596,7 +714,7 @@ lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A,
   if (cudaSetDevice(A->device) != cudaSuccess) return LQ_ERR_CUDA;
   if (A->main_kind != LQ_KIND_E4M3) return LQ_ERR_UNSUPPORTED;
   const int abits = lq_branch_abits(L->cfg.branch);
-  const int br = L->f16_branch ? BR_F16 : (L->integer_branch && abits > 0) ? BR_INT : BR_NONE;
+  const int br = L->mxfp ? (L->r > 0 ? BR_MXFP : BR_NONE) : L->f16_branch ? BR_F16 : (L->integer_branch && abits > 0) ? BR_INT : BR_NONE;
   const int ntr = lq_quant_rank_tiles(L->r, L->f16_branch);
   QuantParams p;
   p.M = M; p.K = L->K; p.Kpad = L->Kpad; p.Mpad = A->Mpad; p.G = L->G;
@@ -607,6 +725,7 @@ lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A,
   p.sXb = A->d_sXb;
   p.L1f = reinterpret_cast<const uint4*>(L->f16_branch ? (const void*)L->d_L1h : (const void*)L->d_L1f);
   p.sL1 = L->d_sL1; p.tq = A->d_tq; p.sT = A->d_sT;
+  p.s1b = L->d_s1b; p.sft = A->d_sft;
   p.r = L->r; p.rpad = ntr * 8;
   p.qm = br == BR_INT ? (float)((1 << (abits - 1)) - 1) : 0.f;
   p.status = lq_device_status_ptr(A->device);
@@ -616,6 +735,7 @@ lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A,
   if (s != LQ_OK) return s;
   int sms = 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, A->device) != cudaSuccess) return LQ_ERR_CUDA;
-  const cudaError_t e = L->mx ? dispatch_quant<true>(br, ntr, tm, p, sms, st) : dispatch_quant<false>(br, ntr, tm, p, sms, st);
+  const cudaError_t e = L->mxfp ? dispatch_quant<MAIN_MXFP>(br, ntr, tm, p, sms, st)
+                        : L->mx ? dispatch_quant<MAIN_MXINT4>(br, ntr, tm, p, sms, st) : dispatch_quant<MAIN_SINT4>(br, ntr, tm, p, sms, st);
   return lq_note_cuda(e) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
 }

@@ -22,6 +22,24 @@ def import_oracle_layer(layer: dict):
     return h, cfg
 
 
+def import_oracle_mxfp_layer(layer: dict):
+    """An MXFP layer of oracle/lq_oracle_mxfp.py -> library handle: element values become their bit patterns
+    (e2m1 nibbles for the residual, e4m3 bytes for the factors), exponents become powers of two."""
+    K, N, r = layer["K"], layer["N"], layer["rank"]
+    branch = layer["branch"] if r > 0 else "none"
+    cfg = B.lq_config_default(K, N, r, branch)
+    cfg.group, cfg.main_fmt = 32, B.MAIN_MXFP4
+    sw = np.exp2(layer["ew"].astype(np.float64)).astype(np.float16)
+    if r > 0:
+        L1, L2 = B.e4m3_encode(layer["L1v"]), B.e4m3_encode(layer["L2v"])
+        s1 = np.exp2(layer["e1"].astype(np.float64)).astype(np.float32)
+        s2 = np.exp2(layer["e2"].astype(np.float64)).astype(np.float32)
+    else:
+        L1 = L2 = s1 = s2 = None
+    h = B.lq_layer_import(cfg, B.pack_e2m1(layer["Wv"]), sw, L1, s1, L2, s2, layer.get("bias"))
+    return h, cfg
+
+
 def gpu_forward(layer: dict, X16: np.ndarray, out_f32: bool = True, export: bool = True, device: int = 0,
                 store_qb: bool = True):
     """Runs lq_quantize_act + lq_linear_forward through the C ABI; returns (Y, exported act dict).
@@ -29,7 +47,7 @@ def gpu_forward(layer: dict, X16: np.ndarray, out_f32: bool = True, export: bool
     (the benchmark configuration leaves them on chip)."""
     import torch
     B.lq_set_option("store_qb", 1 if store_qb else 0)
-    h, cfg = import_oracle_layer(layer)
+    h, cfg = import_oracle_mxfp_layer(layer) if layer.get("main") == "mxfp4" else import_oracle_layer(layer)
     B.lq_layer_to_device(h, device)
     M = X16.shape[0]
     act = B.lq_act_create(h, M, device)
