@@ -51,6 +51,7 @@ def gemm_ops(M, K, N, r):
 NOMINAL_8BIT_TOPS = 4500.0      # dense 8-bit-operand class figure of the part (context, not the denominator of `frac`)
 SMS, FP32_LANES, SM_MAX_HZ = 148, 128, 1.965e9
 STACK_BLOCKS = 28
+MXFP_RANK, MXFP_BRANCH = 64, "mxfp8"   # Table 3's MXFP8e4 row: rank 64 at the memory of an fp16 rank-32 branch
 
 
 def layer_bounds(M, K, N, r, main, peaks):
@@ -58,12 +59,14 @@ def layer_bounds(M, K, N, r, main, peaks):
     K2 tensor: ops / (2 x bf16 burst); K2 drain (SINT4 only): 2 fp32 operations per output and group (G groups + the
     branch) on 128 lanes per SM at the maximum SM clock; K2 HBM: packed 4-bit codes, scales, branch codes in, fp16 Y
     out, weights once; K1 HBM: X in, codes and scales out."""
-    G = -(-K // (32 if main == "mxint4" else 64))
-    sc = G if main == "mxint4" else 2 * G
+    mx = main in ("mxint4", "mxfp4")
+    G = -(-K // (32 if mx else 64))
+    sc = G if mx else 2 * G
     t_tensor = gemm_ops(M, K, N, r) / (2.0 * peaks["bf16_tflops"] * 1e12)
-    t_drain = 0.0 if main == "mxint4" else 2.0 * M * N * (-(-K // 64) + (1 if r else 0)) / (SMS * FP32_LANES * SM_MAX_HZ)
+    t_drain = 0.0 if mx else 2.0 * M * N * (-(-K // 64) + (1 if r else 0)) / (SMS * FP32_LANES * SM_MAX_HZ)
     k2_bytes = M * (K // 2 + sc + r + 4) + 2 * M * N + (K * N // 2 + sc * N + r * N + 4 * N)
-    k1_bytes = M * (2 * K + K // 2 + K + sc + 4 + r + 4)
+    # quantizer output: packed 4-bit codes + 8-bit branch codes (MXFP: ONE 8-bit code stream for both branches)
+    k1_bytes = M * (2 * K + (K if main == "mxfp4" else K // 2 + K) + sc + 4 + r + 4)
     t_hbm2 = k2_bytes / (peaks["hbm_gbs"] * 1e9)
     t_hbm1 = k1_bytes / (peaks["hbm_gbs"] * 1e9)
     return {"t_tensor_us": t_tensor * 1e6, "t_drain_us": t_drain * 1e6, "t_hbm_gemm_us": t_hbm2 * 1e6,
@@ -157,26 +160,36 @@ def build_workload(args):
     return I, wl
 
 
+def oracle_layer(W, wl, args, steps):
+    """(calibrated oracle layer, its forward, the rank it used) for the format --main names."""
+    if args.main == "mxfp4":
+        from oracle import lq_oracle_mxfp as OF
+        layer, _ = OF.calibrate(W, MXFP_RANK, MXFP_BRANCH, steps=steps)
+        return layer, OF.forward, MXFP_RANK
+    from oracle import lq_oracle as O
+    layer, _ = O.calibrate(W, wl.rank, wl.branch, steps=steps, main=args.main)
+    return layer, O.forward, wl.rank
+
+
 def run_reference(args):
     """Reference arm: the CPU oracle as it stands, on a bounded row sample of the same layers."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    from oracle import lq_oracle as O
     I, wl = build_workload(args)
     layers = []
     for spec in wl.layers:
         X, W, _ = I.layer_inputs(wl, spec, M=SAMPLE_ROWS)
-        layer, _ = O.calibrate(W, wl.rank, wl.branch, steps=args.calib_steps, main=args.main)
+        layer, fwd, r = oracle_layer(W, wl, args, args.calib_steps)
         layers.append((spec, X, layer))
-    ops_sample = sum(layer_ops(SAMPLE_ROWS, s.K, s.N, wl.rank) for s, _, _ in layers)
+    ops_sample = sum(layer_ops(SAMPLE_ROWS, s.K, s.N, r) for s, _, _ in layers)
     for _ in range(args.warmup):
         for _, X, layer in layers:
-            O.forward(X, layer)
+            fwd(X, layer)
     t0 = time.perf_counter()
     for _ in range(args.steps):
         for _, X, layer in layers:
-            O.forward(X, layer)
+            fwd(X, layer)
     dt = time.perf_counter() - t0
     value = ops_sample * args.steps / dt / 1e12
     cores = blas_threads()
@@ -192,10 +205,14 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-MAIN_NAMES = {"sint4": "SINT4 group 64 (fp16 scales)", "mxint4": "MXINT4 block 32 (power-of-two scales)"}
+MAIN_NAMES = {"sint4": "SINT4 group 64 (fp16 scales)", "mxint4": "MXINT4 block 32 (power-of-two scales)",
+              "mxfp4": "MXFP4e2 weights x MXFP8e4 activations, block 32 (power-of-two scales)"}
 
 
 def workload_config(wl, args):
+    if args.main == "mxfp4":      # the MXFP study has its own branch: rank and format of Table 3's MXFP8e4 row
+        import dataclasses
+        wl = dataclasses.replace(wl, rank=MXFP_RANK, branch=MXFP_BRANCH)
     if wl.config in (1, 2):
         desc = (f"config{wl.config}: PixArt-class block linears (qkv 1152->3456, attn-out 1152->1152, fc1 1152->4608, "
                 f"fc2 4608->1152), M={wl.M} rows (4096 tokens x batch 2), rank {wl.rank}, main W4A4 {MAIN_NAMES[args.main]}, "
@@ -224,19 +241,18 @@ def workload_config(wl, args):
 def cpu_baseline(wl, I, args):
     """The oracle on this machine's host cores: 256 sampled rows per layer, all layers, repeated
     until about 10 s have passed."""
-    from oracle import lq_oracle as O
     layers = []
     for spec in wl.layers:
         X, W, _ = I.layer_inputs(wl, spec, M=SAMPLE_ROWS)
-        layer, _ = O.calibrate(W, wl.rank, wl.branch, steps=0, main=args.main)
+        layer, fwd, r = oracle_layer(W, wl, args, 0)
         layers.append((spec, X, layer))
-    ops = sum(layer_ops(SAMPLE_ROWS, s.K, s.N, wl.rank) for s, _, _ in layers)
+    ops = sum(layer_ops(SAMPLE_ROWS, s.K, s.N, r) for s, _, _ in layers)
     for _, X, layer in layers:
-        O.forward(X, layer)
+        fwd(X, layer)
     n, t0 = 0, time.perf_counter()
     while True:
         for _, X, layer in layers:
-            O.forward(X, layer)
+            fwd(X, layer)
         n += 1
         dt = time.perf_counter() - t0
         if dt > 10.0 or n >= 200:
@@ -282,7 +298,10 @@ def run_ours(args):
         layers = []
         for spec in wl.layers:
             Xh, W, bias = I.layer_inputs(wl, spec, seed=D.shard_seed(0, rank), with_bias=True)
-            cfg = B.lq_config_default(spec.K, spec.N, r, wl.branch)
+            if main == "mxfp4":
+                cfg = B.lq_config_default(spec.K, spec.N, MXFP_RANK, MXFP_BRANCH)
+            else:
+                cfg = B.lq_config_default(spec.K, spec.N, r, wl.branch)
             cfg.steps = args.calib_steps
             if main == "mxint4":
                 cfg.group = 32
@@ -301,6 +320,7 @@ def run_ours(args):
 
     def measure(main, layers, steps, sample_clocks):
         """Device-resident timing of `steps` steps; returns per-step and per-launch CUDA-event times."""
+        r = MXFP_RANK if main == "mxfp4" else wl.rank
         def step(timed=None):
             if args.l2 == "flush" and not stack:
                 flush.zero_()
@@ -373,6 +393,7 @@ def run_ours(args):
 
     def summarise(main, res):
         """value / roofline records of one measured format."""
+        r = MXFP_RANK if main == "mxfp4" else wl.rank
         ops_step = repeats * sum(layer_ops(M, L["K"], L["N"], r) for L in res["layers"])
         gops_block = sum(gemm_ops(M, L["K"], L["N"], r) for L in res["layers"])
         gemm_ms = sum(L["gemm_us"] for L in res["layers"]) * 1e-3
@@ -382,7 +403,7 @@ def run_ours(args):
         bound_gemm_ms = sum(L["bounds_us"]["gemm_bound_us"] for L in res["layers"]) * 1e-3
         bound_quant_ms = sum(L["bounds_us"]["t_hbm_quant_us"] for L in res["layers"]) * 1e-3
         k1_bytes = sum(L["k1_bytes"] for L in res["layers"])
-        kname = "lq_gemm_mx_kernel" if main == "mxint4" else "lq_gemm_kernel"
+        kname = "lq_gemm_mx_kernel" if main in ("mxint4", "mxfp4") else "lq_gemm_kernel"
         roof = {"kernel": kname + " (one launch per layer)", "bound": "tensor",
                 "achieved": achieved, "peak": burst, "unit": "TOP/s", "frac": achieved / burst,
                 "traffic": gemm_traffic_bytes(main),
@@ -436,7 +457,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     e2e_s = D.max_over_ranks(e2e_s, world, dev)
-    ops_step = repeats * sum(layer_ops(M, L["spec"].K, L["spec"].N, r) for L in layers)
+    ops_step = repeats * sum(layer_ops(M, L["spec"].K, L["spec"].N, MXFP_RANK if args.main == "mxfp4" else r) for L in layers)
     specs = [L["spec"] for L in layers]
     teardown(layers)
 
@@ -451,6 +472,18 @@ def run_ours(args):
               "roofline": mx_s["roofline"], "roofline_quantizer": mx_s["roofline_quantizer"], "layers": mx_res["layers"],
               "clocks": mx_res["clocks"]}
         teardown(mx_layers)
+    fp = None
+    if args.main == "sint4" and wl.config == 1 and not args.no_mxint4:
+        # and with the MXFP formats of the mixed-precision study (Tables 3-4): MXFP4e2 weights, MXFP8e4 activations for
+        # both branches, MXFP8e4 factors of rank 64; every scale is applied by the tensor core
+        fp_layers = setup("mxfp4")
+        fp_res = measure("mxfp4", fp_layers, args.steps, True)
+        fp_s = summarise("mxfp4", fp_res)
+        fp = {"what": f"the same layer shapes with MXFP4e2 residual weights, MXFP8e4 activations and a rank-{MXFP_RANK} {MXFP_BRANCH} branch",
+              "value": fp_s["value"], "unit": UNIT, "ms_per_step": fp_s["ms_per_step"], "tokens_per_s": fp_s["tokens_per_s"],
+              "roofline": fp_s["roofline"], "roofline_quantizer": fp_s["roofline_quantizer"], "layers": fp_res["layers"],
+              "clocks": fp_res["clocks"]}
+        teardown(fp_layers)
 
     if rank == 0:
         nl = len(specs)
@@ -465,7 +498,7 @@ def run_ours(args):
                     "h2d_bytes_per_step": int(repeats * sum(M * sp.K * 2 for sp in specs)),
                     "d2h_bytes_per_step": int(repeats * sum(M * sp.N * 2 for sp in specs)),
                     "ms_per_step": e2e_s / e2e_steps * 1e3},
-            "gpu_launches": args.steps * repeats * nl * 2 * (2 if mx is not None else 1),
+            "gpu_launches": args.steps * repeats * nl * 2 * (1 + (mx is not None) + (fp is not None)),
             "roofline": summ["roofline"],
             "roofline_quantizer": summ["roofline_quantizer"],
             "layers": res["layers"],
@@ -473,6 +506,8 @@ def run_ours(args):
         }
         if mx is not None:
             line["mxint4"] = mx
+        if fp is not None:
+            line["mxfp4"] = fp
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(wl, I, args)
         print(json.dumps(line))
@@ -489,7 +524,7 @@ def main():
     ap.add_argument("--config", type=int, default=1)
     ap.add_argument("--rank", type=int, default=32)
     ap.add_argument("--branch", default=None)
-    ap.add_argument("--main", default="sint4", choices=["sint4", "mxint4"],
+    ap.add_argument("--main", default="sint4", choices=["sint4", "mxint4", "mxfp4"],
                     help="main-branch 4-bit format: sint4 = blocks of 64 with fp16 scales (the headline configuration), "
                          "mxint4 = blocks of 32 with power-of-two scales applied by the tensor core")
     ap.add_argument("--calib-steps", type=int, default=2, dest="calib_steps")

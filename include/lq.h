@@ -98,7 +98,9 @@ lq_status lq_config_default(lq_config* cfg, int32_t K, int32_t N, int32_t rank, 
  * Om^T L2: the same product) is then optimised to lower Q2's error (Cayley retraction steps,
  * best iterate kept); the factors are quantized with Q2; P = W - Q2(L1) Q2(L2) is quantized
  * with Q1 (SINT4 or MXINT4 blocks along K per output column, as cfg->group says; MXINT4 weight
- * exponents are kept within [-24, 15] so that 2^e is a finite fp16 number).
+ * exponents are kept within [-24, 15] so that 2^e is a finite fp16 number).  With main_fmt = LQ_MAIN_MXFP4,
+ * Q1 is MXFP4e2 and Q2 the branch's MXFP format (blocks of 32 along each factor's contraction axis; exponent
+ * floor(log2 max) - emax as in the OCP Microscaling conversion the paper cites; no rotation step: rot_steps must be 0).
  *   W_f16_host     [K][N] row-major IEEE half bits (the paper's d x n orientation), host
  *   bias_f16_host  [N] half bits or NULL, host
  *   out            receives a new layer (host copy only; see lq_layer_to_device)
@@ -117,8 +119,7 @@ lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W_f16_host,
  *   sL1, sL2  fp32 per-column scales [rank] and [N]; NULL for W16A16
  *   bias      [N] half bits or NULL
  * With rank == 0 or LQ_BRANCH_NONE the branch pointers are ignored.
- * MXFP layers (main_fmt = LQ_MAIN_MXFP4; the library has no host calibration for them: calibrate elsewhere, import
- * here; lq_calibrate returns UNSUPPORTED):
+ * MXFP layers (main_fmt = LQ_MAIN_MXFP4):
  *   Wq_packed [K][N/2] bytes: e2m1 bit patterns (sign, two exponent bits, one mantissa bit) as nibbles, same order
  *   sw        [ceil(K/32)][N] half bits: the block's power-of-two scale 2^e, e in [-24, 15]
  *   L1, L2    [K][rank] and [rank][N] bytes: e4m3 bit patterns of the elements (every e2m3 and e2m1 value is an

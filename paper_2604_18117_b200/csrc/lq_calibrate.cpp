@@ -268,6 +268,63 @@ void quant_main(const std::vector<double>& A, int K, int N, int8_t* codes, uint1
   }
 }
 
+// ---- MX formats with small-float elements (Appendix A.3 "MX Formats"; conversion of the OCP specification the paper cites)
+struct ElemFmt { int mant, emin, emax; double vmax; };
+const ElemFmt FMT_E4M3{3, -6, 8, 448.0}, FMT_E2M3{3, 0, 2, 7.5}, FMT_E2M1{1, 0, 2, 6.0};
+
+// x rounded to the nearest element value, ties to the even mantissa, clamped to the largest normal
+double round_to_element(double x, const ElemFmt& f) {
+  const double a = fabs(x);
+  if (a == 0.0) return 0.0;
+  int e = 0;
+  frexp(a, &e);                                         // a = m 2^e, m in [0.5, 1): floor(log2 a) = e - 1
+  e = std::max(f.emin, std::min(f.emax, e - 1));
+  const double quantum = ldexp(1.0, e - f.mant);
+  const double q = std::min(nearbyint(a / quantum) * quantum, f.vmax);   // default rounding mode: ties to even
+  return x < 0 ? -q : q;
+}
+
+// e4m3 bit pattern of a value that is exactly representable in e4m3 (every e2m3 and e2m1 value is)
+uint8_t e4m3_bits(double v) {
+  const double a = fabs(v);
+  uint8_t b = 0;
+  if (a > 0.0) {
+    int e = 0;
+    frexp(a, &e);
+    e -= 1;
+    if (e < -6) b = (uint8_t)nearbyint(a * 512.0);                       // subnormal: m / 8 * 2^-6
+    else b = (uint8_t)(((e + 7) << 3) | (int)nearbyint((a / ldexp(1.0, e) - 1.0) * 8.0));
+  }
+  return (uint8_t)(b | (v < 0 ? 0x80 : 0));
+}
+
+// MX quantizer of F [rows][cols] with blocks of 32 down each column: exponent floor(log2 max) - emax (0 for an all-zero
+// block, whose elements are zeros), elements rounded to the format.  Any of bytes (e4m3 patterns), scales (2^e as float,
+// [ceil(rows/32)][cols]) and Dq (dequantized values) may be null.
+void quant_mx_columns(const std::vector<double>& F, int rows, int cols, const ElemFmt& f, uint8_t* bytes, float* scales, double* Dq) {
+  const int nb = lq_ceil_div(rows, 32);
+#pragma omp parallel for schedule(static)
+  for (int b = 0; b < nb; ++b) {
+    const int t0 = b * 32, t1 = std::min(rows, t0 + 32);
+    for (int c = 0; c < cols; ++c) {
+      double a = 0.0;
+      for (int t = t0; t < t1; ++t) a = std::max(a, fabs(F[(size_t)t * cols + c]));
+      int e = 0;
+      if (a > 0.0) {
+        frexp(a, &e);
+        e = std::max(-127, std::min(127, e - 1 - f.emax));
+      }
+      const double sc = ldexp(1.0, e);
+      if (scales) scales[(size_t)b * cols + c] = (float)sc;
+      for (int t = t0; t < t1; ++t) {
+        const double el = round_to_element(F[(size_t)t * cols + c] / sc, f);
+        if (bytes) bytes[(size_t)t * cols + c] = e4m3_bits(el);
+        if (Dq) Dq[(size_t)t * cols + c] = el * sc;
+      }
+    }
+  }
+}
+
 // One fp32 scale per column of F [rows][cols]; codes [rows][cols].
 void quant_columns(const std::vector<double>& F, int rows, int cols, int bits, int8_t* codes, float* scales) {
   const float qm = (float)((1 << (bits - 1)) - 1);
@@ -435,7 +492,9 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
   if (!cfg || !W16 || !out) return LQ_ERR_INVALID_ARG;
   if (cfg->K <= 0 || cfg->N <= 0 || cfg->rank < 0 || cfg->steps < 0) return LQ_ERR_INVALID_ARG;
   if (cfg->branch < LQ_BRANCH_NONE || cfg->branch > LQ_BRANCH_MXFP4) return LQ_ERR_INVALID_ARG;
-  if (cfg->main_fmt == LQ_MAIN_MXFP4 || lq_branch_is_mxfp(cfg->branch)) return LQ_ERR_UNSUPPORTED;   // MXFP layers are imported
+  const bool mxfp = cfg->main_fmt == LQ_MAIN_MXFP4;
+  if (mxfp ? !(cfg->branch == LQ_BRANCH_NONE || lq_branch_is_mxfp(cfg->branch)) : lq_branch_is_mxfp(cfg->branch)) return LQ_ERR_UNSUPPORTED;
+  if (mxfp && (cfg->group != LQ_MX_BLOCK || cfg->rot_steps > 0)) return LQ_ERR_UNSUPPORTED;   // no rotation step for MXFP factors yet
   if ((cfg->group != LQ_GROUP && cfg->group != LQ_MX_BLOCK) || cfg->rot_steps < 0) return LQ_ERR_UNSUPPORTED;
   if (cfg->K > LQ_MAX_K || (cfg->K % 8) || (cfg->N % 8) || cfg->rank > LQ_MAX_RANK) return LQ_ERR_UNSUPPORTED;
   if (cfg->branch == LQ_BRANCH_W16A16 && cfg->rank > 64) return LQ_ERR_UNSUPPORTED;
@@ -456,9 +515,21 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
     Lr->Wq.resize((size_t)K * N);
     Lr->sw.resize((size_t)G * N);
     const double inv_size = 1.0 / ((double)K * (double)N);
+    // Q1 of a matrix: dequantized values into Dq; with `store`, the layer's residual codes and scales too
+    auto q1 = [&](const std::vector<double>& A_, double* Dq_, bool store) {
+      if (!mxfp) {
+        quant_main(A_, K, N, store ? Lr->Wq.data() : nullptr, store ? Lr->sw.data() : nullptr, Dq_, cfg->group);
+        return;
+      }
+      if (!store) { quant_mx_columns(A_, K, N, FMT_E2M1, nullptr, nullptr, Dq_); return; }
+      std::vector<float> sc((size_t)G * N);
+      Lr->Wq8h.resize((size_t)K * N);
+      quant_mx_columns(A_, K, N, FMT_E2M1, Lr->Wq8h.data(), sc.data(), Dq_);
+      for (size_t i = 0; i < sc.size(); ++i) Lr->sw[i] = float_to_half_bits(sc[i]);   // 2^e; weights far below 2^-24 are outside this library's range
+    };
     if (r == 0) {
       std::vector<double> Dq((size_t)K * N);
-      quant_main(W, K, N, Lr->Wq.data(), Lr->sw.data(), Dq.data(), cfg->group);
+      q1(W, Dq.data(), true);
       if (trace) {
         double loss = 0;
         for (size_t i = 0; i < W.size(); ++i) loss += (Dq[i] - W[i]) * (Dq[i] - W[i]);
@@ -479,7 +550,7 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
       matmul_LR(L, R, K, N, r, D);
 #pragma omp parallel for schedule(static)
       for (long long i = 0; i < (long long)A.size(); ++i) A[i] = W[i] + D[i];
-      quant_main(A, K, N, nullptr, nullptr, E.data(), cfg->group);            // E <- deq(Q1(W + LR))
+      q1(A, E.data(), false);                                                  // E <- deq(Q1(W + LR))
       double loss = 0;
 #pragma omp parallel for reduction(+ : loss) schedule(static)
       for (long long i = 0; i < (long long)A.size(); ++i) {
@@ -528,7 +599,13 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
     for (double& v : L1) v = -v;
     if (cfg->rot_steps > 0) rotate_factors(L1, L2, K, N, r, Lr->f16_branch ? 0 : lq_branch_wbits(cfg->branch), cfg->rot_steps, (double)cfg->rot_lr);
     std::vector<double> L1d(L1.size()), L2d(L2.size());
-    if (Lr->f16_branch) {
+    if (mxfp) {
+      const ElemFmt& f = cfg->branch == LQ_BRANCH_MXFP8 ? FMT_E4M3 : cfg->branch == LQ_BRANCH_MXFP6 ? FMT_E2M3 : FMT_E2M1;
+      Lr->L1e.resize(L1.size()); Lr->L2e.resize(L2.size());
+      Lr->s1b.resize((size_t)lq_ceil_div(K, 32) * r); Lr->s2b.resize((size_t)lq_ceil_div(r, 32) * N);
+      quant_mx_columns(L1, K, r, f, Lr->L1e.data(), Lr->s1b.data(), L1d.data());   // blocks along K per column of L1
+      quant_mx_columns(L2, r, N, f, Lr->L2e.data(), Lr->s2b.data(), L2d.data());   // blocks along the rank per column of L2
+    } else if (Lr->f16_branch) {
       Lr->L1h.resize(L1.size()); Lr->L2h.resize(L2.size());
       for (size_t i = 0; i < L1.size(); ++i) { Lr->L1h[i] = float_to_half_bits((float)L1[i]); L1d[i] = half_bits_to_float(Lr->L1h[i]); }
       for (size_t i = 0; i < L2.size(); ++i) { Lr->L2h[i] = float_to_half_bits((float)L2[i]); L2d[i] = half_bits_to_float(Lr->L2h[i]); }
@@ -544,7 +621,7 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
     }
     matmul_LR(L1d, L2d, K, N, r, D);
     for (size_t i = 0; i < A.size(); ++i) A[i] = W[i] - D[i];     // P = W - Q2(L1) Q2(L2)
-    quant_main(A, K, N, Lr->Wq.data(), Lr->sw.data(), nullptr, cfg->group);
+    q1(A, nullptr, true);
     *out = owner.release();
     return LQ_OK;
   } catch (const std::bad_alloc&) {

@@ -29,11 +29,12 @@ def import_oracle_mxfp_layer(layer: dict):
     branch = layer["branch"] if r > 0 else "none"
     cfg = B.lq_config_default(K, N, r, branch)
     cfg.group, cfg.main_fmt = 32, B.MAIN_MXFP4
-    sw = np.exp2(layer["ew"].astype(np.float64)).astype(np.float16)
+    live = lambda e: np.where(e == -127, 0, e).astype(np.float64)       # an all-zero block: any scale does, its elements are zeros
+    sw = np.exp2(live(layer["ew"])).astype(np.float16)
     if r > 0:
         L1, L2 = B.e4m3_encode(layer["L1v"]), B.e4m3_encode(layer["L2v"])
-        s1 = np.exp2(layer["e1"].astype(np.float64)).astype(np.float32)
-        s2 = np.exp2(layer["e2"].astype(np.float64)).astype(np.float32)
+        s1 = np.exp2(live(layer["e1"])).astype(np.float32)
+        s2 = np.exp2(live(layer["e2"])).astype(np.float32)
     else:
         L1 = L2 = s1 = s2 = None
     h = B.lq_layer_import(cfg, B.pack_e2m1(layer["Wv"]), sw, L1, s1, L2, s2, layer.get("bias"))

@@ -173,3 +173,53 @@ def test_first_adam_steps_match_the_oracle_trajectory():
         assert np.allclose(trace, tr_o, rtol=1e-7, atol=0), (main, trace, tr_o)
         assert abs(tr_o[1] - tr_o[0]) > 1e-4 * tr_o[0]     # the step is visible in the objective
         B.lq_layer_free(h)
+
+
+def _export_mxfp_as_oracle_layer(h):
+    from oracle import lq_oracle_mxfp as F
+    cfg = B.lq_layer_info(h)
+    ex = B.lq_layer_export(h)
+    K, N, r = cfg.K, cfg.N, cfg.rank
+    lo, hi = ex["Wq_packed"] & 0xF, ex["Wq_packed"] >> 4
+    grid = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6, -0.0, -0.5, -1, -1.5, -2, -3, -4, -6], dtype=np.float32)
+    Wv = np.empty((K, N), np.float32); Wv[:, 0::2] = grid[lo]; Wv[:, 1::2] = grid[hi]
+    layer = {"main": "mxfp4", "branch": B.BRANCH_NAME[cfg.branch], "rank": r, "K": K, "N": N, "bias": None,
+             "Wv": Wv, "ew": np.log2(ex["sw"].astype(np.float64)).astype(np.int16)}
+    if r > 0:
+        layer.update(L1v=B.e4m3_decode(ex["L1"]), e1=np.log2(ex["sL1"].astype(np.float64)).astype(np.int16),
+                     L2v=B.e4m3_decode(ex["L2"]), e2=np.log2(ex["sL2"].astype(np.float64)).astype(np.int16))
+    return layer
+
+
+def test_mxfp_calibration_follows_the_oracle():
+    """lq_calibrate with the MXFP4 residual and an MXFP8 / MXFP6 / MXFP4 branch: the first Adam steps follow the MXFP
+    oracle's objective trace (same argument as for the integer formats: well separated singular values, two steps), the
+    stored factors are on their format's grid, and the stored residual is Q1 of W - Q2(L1) Q2(L2) (Figure 1)."""
+    from oracle import lq_oracle_mxfp as F
+    rng = np.random.default_rng(12)
+    K, N, r = 96, 32, 3
+    U, _ = np.linalg.qr(rng.standard_normal((K, N)))
+    V, _ = np.linalg.qr(rng.standard_normal((N, N)))
+    sig = np.concatenate([[0.9, 0.6, 0.35], np.linspace(0.05, 0.01, N - 3)])
+    W = ((U * sig[None, :]) @ V.T).astype(np.float16)
+    for branch in ("mxfp8", "mxfp6", "mxfp4"):
+        cfg = B.lq_config_default(K, N, r, branch)
+        assert cfg.main_fmt == B.MAIN_MXFP4 and cfg.group == 32 and abs(cfg.lr - 1e-3) < 1e-9   # FP formats: 1e-3 (Appendix A.2)
+        cfg.steps = 2
+        h, trace = B.lq_calibrate(cfg, W, want_trace=True)
+        _, tr_o = F.calibrate(W, r, branch, steps=2)
+        assert np.allclose(trace, tr_o, rtol=1e-7, atol=0), (branch, trace, tr_o)
+        layer = _export_mxfp_as_oracle_layer(h)
+        fmt = F.BRANCH_FORMAT[branch]
+        grid = F.element_values(fmt).astype(np.float32)
+        assert np.isin(np.abs(layer["L1v"]), grid).all() and np.isin(np.abs(layer["L2v"]), grid).all()
+        D = F.deq_columns(layer["L1v"], layer["e1"]) @ F.deq_columns(layer["L2v"], layer["e2"])
+        Wv, ew = F.q_columns(W.astype(np.float64) - D, "e2m1")
+        assert np.array_equal(F.deq_columns(Wv, ew), F.deq_columns(layer["Wv"], layer["ew"]))
+        B.lq_layer_free(h)
+    cfg = B.lq_config_default(K, N, 0, "none")
+    cfg.group, cfg.main_fmt = 32, B.MAIN_MXFP4
+    h, _ = B.lq_calibrate(cfg, W)
+    layer = _export_mxfp_as_oracle_layer(h)
+    assert np.array_equal(F.deq_columns(layer["Wv"], layer["ew"]), F.q1_dequant(W.astype(np.float64)))
+    B.lq_layer_free(h)
