@@ -35,6 +35,16 @@
 
 #include "lq_device.cuh"
 
+#ifdef LQ_TIMELINE
+// Timeline build only: copies this kernel's stamp lists of the last launch to the host and clears them.
+extern "C" int lq_debug_timeline_mx(unsigned long long* host_out) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return 1;
+  if (cudaMemcpyFromSymbol(host_out, g_lq_timeline, sizeof(unsigned long long) * lqdev::TL_LISTS * lqdev::TL_CAP) != cudaSuccess) return 1;
+  static unsigned long long zeros[lqdev::TL_LISTS][lqdev::TL_CAP];
+  return cudaMemcpyToSymbol(g_lq_timeline, zeros, sizeof(zeros)) == cudaSuccess ? 0 : 1;
+}
+#endif
+
 namespace {
 
 using namespace lqdev;
@@ -169,6 +179,11 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   tc_fence_after();
   const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
 
+  LQ_TL_DECL((blockIdx.x == 0 && lane == 0)
+                 ? (warp == 0 ? (int)TL_PRODUCER : warp == 1 ? (int)TL_MMA : warp == FIRST_DRAIN_WARP ? (int)TL_DRAIN_FIRST
+                    : warp == FIRST_DRAIN_WARP + NUM_DRAIN_WARPS - 1 ? (int)TL_DRAIN_LAST : -1)
+                 : -1);
+
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     uint32_t it = 0, tc = 0;
@@ -196,6 +211,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int st = it % NSTAGE;
         ok = mbar_wait_warp(bar(B_EMPTY + st), ((it / NSTAGE) & 1) ^ 1, abort_flag, p.status, LQ_STAGE_PRODUCER);
         if (!ok) break;
+        LQ_TL(EV_P_SLOT_FREE, s);
         const uint32_t a_dst = sm_stage + st * STAGE_BYTES, b_dst = a_dst + STAGE_A_BYTES, sf_dst = sm_sf + st * STAGE_SF_BYTES;
         const uint32_t full = bar(B_FULL + st);
         if (elect_one()) {
@@ -207,6 +223,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           bulk_load(sf_dst + SF_BYTES, sfb + (size_t)s * p.units_n * SF_BYTES, width * SF_BYTES, full);
         }
         __syncwarp();
+        LQ_TL(EV_P_ISSUED, s);
       }
       if (has_branch && ok) {   // the branch operands: the containers of tq (128 rows) and L2q (256 rows), r contiguous
         const int st = it % NSTAGE;
@@ -245,11 +262,13 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       ok = mbar_wait_warp(bar(B_TEMPTY), (tc & 1) ^ 1, abort_flag, p.status, LQ_STAGE_MMA);
       if (!ok) break;
       tc_fence_after();
+      LQ_TL(EV_M_ACC_FREE, 0);
       for (int s = 0; s < p.k_stages && ok; ++s, ++it) {
         const int st = it % NSTAGE;
         ok = mbar_wait_warp(bar(B_FULL + st), (it / NSTAGE) & 1, abort_flag, p.status, LQ_STAGE_MMA);
         if (!ok) break;
         tc_fence_after();
+        LQ_TL(EV_M_STAGE_FULL, s);
         const uint32_t a_addr = sm_stage + st * STAGE_BYTES, b_addr = a_addr + STAGE_A_BYTES, sf_addr = sm_sf + st * STAGE_SF_BYTES;
         const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(b_addr);
         const uint32_t tsfa = tmem_base + TM_SFA, tsfb = tmem_base + TM_SFB;
@@ -263,6 +282,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           tc_commit(bar(B_EMPTY + st));
         }
         __syncwarp();
+        LQ_TL(EV_M_ISSUED, s);
       }
       if (!ok) break;
       if (has_branch) {
@@ -298,6 +318,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       }
       if (elect_one()) tc_commit(bar(B_TFULL));
       __syncwarp();
+      LQ_TL(EV_TILE, 0);
     }
   } else {
     // ------------------------------------------------------------------ drain + epilogue
@@ -316,9 +337,11 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int rb = tc & 1;
       float acc[2][2][4][4];                            // [half][m16 tile][n8 tile][fragment register]
       uint32_t w0[2][8];                                // cgi == 0: the branch columns that the scale factors alias
+      LQ_TL(EV_D_OPEN, 0);
       ok = mbar_wait_idle(bar(B_TFULL), tc & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
       if (!ok) break;
       tc_fence_after();
+      LQ_TL(EV_D_ACC_FULL, 0);
       // hand-over: every load is issued before the one wait; the main accumulator lands in the registers it stays in
 #pragma unroll
       for (int h = 0; h < 2; ++h)
@@ -335,6 +358,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(B_TEMPTY));
+      LQ_TL(EV_D_LOADED, 0);
       // y = main + U sT sL2 + bias, under the next tile's main loop (the tensor core has already applied the block
       // scales to main)
       ok = mbar_wait(bar(B_RFULL + rb), (tc >> 1) & 1, abort_flag, p.status, LQ_STAGE_DRAIN);
@@ -379,6 +403,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       tc_fence_before();
       __syncwarp();
       if (lane == 0) { mbar_arrive(bar(B_BEMPTY)); mbar_arrive(bar(B_REMPTY + rb)); }
+      LQ_TL(EV_D_DONE, 0);
       // epilogue
       const int row_w = m0 + quad * 32;                 // first row of this group's part
 #pragma unroll
@@ -424,6 +449,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
         }
       }
+      LQ_TL(EV_D_EPI_END, 0);
     }
   }
 
