@@ -82,16 +82,19 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+TRAFFIC_RECORDS = {"sint4": ("gemm_dram_traffic.json", "lq_gemm_kernel"), "mxint4": ("gemm_mx_dram_traffic.json", "lq_gemm_mx_kernel"),
+                   "mxfp4": ("gemm_mxfp_dram_traffic.json", "lq_gemm_mx_kernel")}
+
+
 def gemm_traffic_bytes(main="sint4"):
-    """DRAM bytes of one step's GEMM launches as measured by ncu (profiles/gemm*_dram_traffic.json),
-    or None when the GEMM source differs from the one that was profiled (or none was taken)."""
-    import hashlib
-    stem = "lq_gemm_mx" if main == "mxint4" else "lq_gemm"
-    rec = os.path.join(ROOT, "profiles", "gemm_mx_dram_traffic.json" if main == "mxint4" else "gemm_dram_traffic.json")
-    src = os.path.join(ROOT, "paper_2604_18117_b200", "csrc", stem + ".cu")
+    """DRAM bytes of one step's GEMM launches as measured by ncu (profiles/gemm*_dram_traffic.json, written by
+    paper_2604_18117_b200.ncu_summary), or None when the kernel's sources differ from the ones that were profiled
+    (or no capture was taken)."""
+    from paper_2604_18117_b200.ncu_summary import sources_sha256
+    name, kernel = TRAFFIC_RECORDS[main]
     try:
-        d = json.load(open(rec))
-        if hashlib.sha256(open(src, "rb").read()).hexdigest() != d[stem + "_cu_sha256"]:
+        d = json.load(open(os.path.join(ROOT, "profiles", name)))
+        if d["kernel"] != kernel or d["sources_sha256"] != sources_sha256(kernel):
             return None
         return int(d["dram_bytes_per_step"])
     except (OSError, KeyError, ValueError):
