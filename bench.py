@@ -52,6 +52,8 @@ NOMINAL_8BIT_TOPS = 4500.0      # dense 8-bit-operand class figure of the part (
 SMS, FP32_LANES, SM_MAX_HZ = 148, 128, 1.965e9
 STACK_BLOCKS = 28
 MXFP_RANK, MXFP_BRANCH = 64, "mxfp8"   # Table 3's MXFP8e4 row: rank 64 at the memory of an fp16 rank-32 branch
+MXINT_RANK, MXINT_BRANCH = 64, "mxint8"   # Table 3's MXINT8 row
+STUDY = {"mxfp4": (MXFP_RANK, MXFP_BRANCH), "mxint4a8": (MXINT_RANK, MXINT_BRANCH)}   # formats with a branch of their own
 
 
 def layer_bounds(M, K, N, r, main, peaks):
@@ -59,14 +61,14 @@ def layer_bounds(M, K, N, r, main, peaks):
     K2 tensor: ops / (2 x bf16 burst); K2 drain (SINT4 only): 2 fp32 operations per output and group (G groups + the
     branch) on 128 lanes per SM at the maximum SM clock; K2 HBM: packed 4-bit codes, scales, branch codes in, fp16 Y
     out, weights once; K1 HBM: X in, codes and scales out."""
-    mx = main in ("mxint4", "mxfp4")
+    mx = main in ("mxint4", "mxfp4", "mxint4a8")
     G = -(-K // (32 if mx else 64))
     sc = G if mx else 2 * G
     t_tensor = gemm_ops(M, K, N, r) / (2.0 * peaks["bf16_tflops"] * 1e12)
     t_drain = 0.0 if mx else 2.0 * M * N * (-(-K // 64) + (1 if r else 0)) / (SMS * FP32_LANES * SM_MAX_HZ)
     k2_bytes = M * (K // 2 + sc + r + 4) + 2 * M * N + (K * N // 2 + sc * N + r * N + 4 * N)
     # quantizer output: packed 4-bit codes + 8-bit branch codes (MXFP: ONE 8-bit code stream for both branches)
-    k1_bytes = M * (2 * K + (K if main == "mxfp4" else K // 2 + K) + sc + 4 + r + 4)
+    k1_bytes = M * (2 * K + (K if main in ("mxfp4", "mxint4a8") else K // 2 + K) + sc + 4 + r + 4)
     t_hbm2 = k2_bytes / (peaks["hbm_gbs"] * 1e9)
     t_hbm1 = k1_bytes / (peaks["hbm_gbs"] * 1e9)
     return {"t_tensor_us": t_tensor * 1e6, "t_drain_us": t_drain * 1e6, "t_hbm_gemm_us": t_hbm2 * 1e6,
@@ -82,7 +84,7 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
-TRAFFIC_RECORDS = {"sint4": ("gemm_dram_traffic.json", "lq_gemm_kernel"), "mxint4": ("gemm_mx_dram_traffic.json", "lq_gemm_mx_kernel"),
+TRAFFIC_RECORDS = {"mxint4a8": ("gemm_mxint4a8_dram_traffic.json", "lq_gemm_mx_kernel"), "sint4": ("gemm_dram_traffic.json", "lq_gemm_kernel"), "mxint4": ("gemm_mx_dram_traffic.json", "lq_gemm_mx_kernel"),
                    "mxfp4": ("gemm_mxfp_dram_traffic.json", "lq_gemm_mx_kernel")}
 
 
@@ -169,6 +171,10 @@ def oracle_layer(W, wl, args, steps):
         from oracle import lq_oracle_mxfp as OF
         layer, _ = OF.calibrate(W, MXFP_RANK, MXFP_BRANCH, steps=steps)
         return layer, OF.forward, MXFP_RANK
+    if args.main == "mxint4a8":
+        from oracle import lq_oracle_mxint as OI
+        layer, _ = OI.calibrate(W, MXINT_RANK, MXINT_BRANCH, steps=steps)
+        return layer, OI.forward, MXINT_RANK
     from oracle import lq_oracle as O
     layer, _ = O.calibrate(W, wl.rank, wl.branch, steps=steps, main=args.main)
     return layer, O.forward, wl.rank
@@ -209,13 +215,14 @@ def run_reference(args):
 
 
 MAIN_NAMES = {"sint4": "SINT4 group 64 (fp16 scales)", "mxint4": "MXINT4 block 32 (power-of-two scales)",
-              "mxfp4": "MXFP4e2 weights x MXFP8e4 activations, block 32 (power-of-two scales)"}
+              "mxfp4": "MXFP4e2 weights x MXFP8e4 activations, block 32 (power-of-two scales)",
+              "mxint4a8": "MXINT4 weights x MXINT8 activations, block 32 (power-of-two scales; 8-bit codes as two 4-bit digit planes)"}
 
 
 def workload_config(wl, args):
-    if args.main == "mxfp4":      # the MXFP study has its own branch: rank and format of Table 3's MXFP8e4 row
+    if args.main in STUDY:        # the mixed-precision study's formats have their own branch: rank and format of Table 3's rows
         import dataclasses
-        wl = dataclasses.replace(wl, rank=MXFP_RANK, branch=MXFP_BRANCH)
+        wl = dataclasses.replace(wl, rank=STUDY[args.main][0], branch=STUDY[args.main][1])
     if wl.config in (1, 2):
         desc = (f"config{wl.config}: PixArt-class block linears (qkv 1152->3456, attn-out 1152->1152, fc1 1152->4608, "
                 f"fc2 4608->1152), M={wl.M} rows (4096 tokens x batch 2), rank {wl.rank}, main W4A4 {MAIN_NAMES[args.main]}, "
@@ -301,8 +308,8 @@ def run_ours(args):
         layers = []
         for spec in wl.layers:
             Xh, W, bias = I.layer_inputs(wl, spec, seed=D.shard_seed(0, rank), with_bias=True)
-            if main == "mxfp4":
-                cfg = B.lq_config_default(spec.K, spec.N, MXFP_RANK, MXFP_BRANCH)
+            if main in STUDY:
+                cfg = B.lq_config_default(spec.K, spec.N, *STUDY[main])
             else:
                 cfg = B.lq_config_default(spec.K, spec.N, r, wl.branch)
             cfg.steps = args.calib_steps
@@ -323,7 +330,7 @@ def run_ours(args):
 
     def measure(main, layers, steps, sample_clocks):
         """Device-resident timing of `steps` steps; returns per-step and per-launch CUDA-event times."""
-        r = MXFP_RANK if main == "mxfp4" else wl.rank
+        r = STUDY[main][0] if main in STUDY else wl.rank
         def step(timed=None):
             if args.l2 == "flush" and not stack:
                 flush.zero_()
@@ -396,7 +403,7 @@ def run_ours(args):
 
     def summarise(main, res):
         """value / roofline records of one measured format."""
-        r = MXFP_RANK if main == "mxfp4" else wl.rank
+        r = STUDY[main][0] if main in STUDY else wl.rank
         ops_step = repeats * sum(layer_ops(M, L["K"], L["N"], r) for L in res["layers"])
         gops_block = sum(gemm_ops(M, L["K"], L["N"], r) for L in res["layers"])
         gemm_ms = sum(L["gemm_us"] for L in res["layers"]) * 1e-3
@@ -406,7 +413,7 @@ def run_ours(args):
         bound_gemm_ms = sum(L["bounds_us"]["gemm_bound_us"] for L in res["layers"]) * 1e-3
         bound_quant_ms = sum(L["bounds_us"]["t_hbm_quant_us"] for L in res["layers"]) * 1e-3
         k1_bytes = sum(L["k1_bytes"] for L in res["layers"])
-        kname = "lq_gemm_mx_kernel" if main in ("mxint4", "mxfp4") else "lq_gemm_kernel"
+        kname = "lq_gemm_mx_kernel" if main in ("mxint4", "mxfp4", "mxint4a8") else "lq_gemm_kernel"
         roof = {"kernel": kname + " (one launch per layer)", "bound": "tensor",
                 "achieved": achieved, "peak": burst, "unit": "TOP/s", "frac": achieved / burst,
                 "traffic": gemm_traffic_bytes(main),
@@ -460,7 +467,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     e2e_s = D.max_over_ranks(e2e_s, world, dev)
-    ops_step = repeats * sum(layer_ops(M, L["spec"].K, L["spec"].N, MXFP_RANK if args.main == "mxfp4" else r) for L in layers)
+    ops_step = repeats * sum(layer_ops(M, L["spec"].K, L["spec"].N, STUDY[args.main][0] if args.main in STUDY else r) for L in layers)
     specs = [L["spec"] for L in layers]
     teardown(layers)
 
@@ -487,6 +494,18 @@ def run_ours(args):
               "roofline": fp_s["roofline"], "roofline_quantizer": fp_s["roofline_quantizer"], "layers": fp_res["layers"],
               "clocks": fp_res["clocks"]}
         teardown(fp_layers)
+    i8 = None
+    if args.main == "sint4" and wl.config == 1 and not args.no_mxint4:
+        # and the study's integer row: MXINT4 weights, MXINT8 activations for both branches (two digit planes per 8-bit
+        # code, so the kernel issues twice the MMAs the op count credits), MXINT8 factors of rank 64
+        i8_layers = setup("mxint4a8")
+        i8_res = measure("mxint4a8", i8_layers, args.steps, True)
+        i8_s = summarise("mxint4a8", i8_res)
+        i8 = {"what": f"the same layer shapes with MXINT4 residual weights, MXINT8 activations and a rank-{MXINT_RANK} {MXINT_BRANCH} branch",
+              "value": i8_s["value"], "unit": UNIT, "ms_per_step": i8_s["ms_per_step"], "tokens_per_s": i8_s["tokens_per_s"],
+              "roofline": i8_s["roofline"], "roofline_quantizer": i8_s["roofline_quantizer"], "layers": i8_res["layers"],
+              "clocks": i8_res["clocks"]}
+        teardown(i8_layers)
 
     if rank == 0:
         nl = len(specs)
@@ -501,7 +520,7 @@ def run_ours(args):
                     "h2d_bytes_per_step": int(repeats * sum(M * sp.K * 2 for sp in specs)),
                     "d2h_bytes_per_step": int(repeats * sum(M * sp.N * 2 for sp in specs)),
                     "ms_per_step": e2e_s / e2e_steps * 1e3},
-            "gpu_launches": args.steps * repeats * nl * 2 * (1 + (mx is not None) + (fp is not None)),
+            "gpu_launches": args.steps * repeats * nl * 2 * (1 + (mx is not None) + (fp is not None) + (i8 is not None)),
             "roofline": summ["roofline"],
             "roofline_quantizer": summ["roofline_quantizer"],
             "layers": res["layers"],
@@ -511,6 +530,8 @@ def run_ours(args):
             line["mxint4"] = mx
         if fp is not None:
             line["mxfp4"] = fp
+        if i8 is not None:
+            line["mxint4a8"] = i8
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(wl, I, args)
         print(json.dumps(line))
@@ -527,7 +548,7 @@ def main():
     ap.add_argument("--config", type=int, default=1)
     ap.add_argument("--rank", type=int, default=32)
     ap.add_argument("--branch", default=None)
-    ap.add_argument("--main", default="sint4", choices=["sint4", "mxint4", "mxfp4"],
+    ap.add_argument("--main", default="sint4", choices=["sint4", "mxint4", "mxfp4", "mxint4a8"],
                     help="main-branch 4-bit format: sint4 = blocks of 64 with fp16 scales (the headline configuration), "
                          "mxint4 = blocks of 32 with power-of-two scales applied by the tensor core")
     ap.add_argument("--calib-steps", type=int, default=2, dest="calib_steps")

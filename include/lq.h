@@ -56,14 +56,22 @@ typedef enum {
    * the rank-r intermediate are MXFP8e4.  Only with main_fmt = LQ_MAIN_MXFP4. */
   LQ_BRANCH_MXFP8 = 5,
   LQ_BRANCH_MXFP6 = 6,
-  LQ_BRANCH_MXFP4 = 7
+  LQ_BRANCH_MXFP4 = 7,
+  /* Integer MX branches of the same study (Table 3's integer rows): factors in blocks of 32 with a power-of-two
+   * scale and signed 8-bit / 4-bit integer codes; the activations of BOTH branches and the rank-r intermediate
+   * are MXINT8.  Only with main_fmt = LQ_MAIN_MXINT4_A8; rank <= 64. */
+  LQ_BRANCH_MXINT8 = 8,
+  LQ_BRANCH_MXINT4 = 9
 } lq_branch_fmt;
 
 /* 4-bit format of the residual (main) branch, Appendix A.3. */
 typedef enum {
   LQ_MAIN_AUTO = 0,    /* from `group`: 64 -> SINT4 (integer codes, fp16 scale per 64), 32 -> MXINT4           */
-  LQ_MAIN_MXFP4 = 2    /* MXFP4e2 weights (e2m1 elements, power-of-two scale per 32; group must be 32) times
+  LQ_MAIN_MXFP4 = 2,   /* MXFP4e2 weights (e2m1 elements, power-of-two scale per 32; group must be 32) times
                           MXFP8e4 activations, all scales applied by the tensor core (Tables 3-4)              */
+  LQ_MAIN_MXINT4_A8 = 3 /* MXINT4 weights (group must be 32) times MXINT8 activations (Table 3's integer rows): an
+                          8-bit code travels as two 4-bit digits, code = 16 hi + lo, each an exact E4M3 operand
+                          with block scales 2^(e+4) and 2^e, so the tensor core applies every scale here too    */
 } lq_main_fmt;
 
 typedef enum { LQ_OUT_F16 = 0, LQ_OUT_F32 = 1 } lq_out_dtype;
@@ -101,6 +109,8 @@ lq_status lq_config_default(lq_config* cfg, int32_t K, int32_t N, int32_t rank, 
  * exponents are kept within [-24, 15] so that 2^e is a finite fp16 number).  With main_fmt = LQ_MAIN_MXFP4,
  * Q1 is MXFP4e2 and Q2 the branch's MXFP format (blocks of 32 along each factor's contraction axis; exponent
  * floor(log2 max) - emax as in the OCP Microscaling conversion the paper cites; no rotation step: rot_steps must be 0).
+ * With main_fmt = LQ_MAIN_MXINT4_A8, Q1 is MXINT4 and Q2 the branch's MX integer format (blocks of 32 along each
+ * factor's contraction axis, the smallest power-of-two scale that does not clip; rot_steps must be 0).
  *   W_f16_host     [K][N] row-major IEEE half bits (the paper's d x n orientation), host
  *   bias_f16_host  [N] half bits or NULL, host
  *   out            receives a new layer (host copy only; see lq_layer_to_device)
@@ -124,7 +134,10 @@ lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W_f16_host,
  *   sw        [ceil(K/32)][N] half bits: the block's power-of-two scale 2^e, e in [-24, 15]
  *   L1, L2    [K][rank] and [rank][N] bytes: e4m3 bit patterns of the elements (every e2m3 and e2m1 value is an
  *             e4m3 value, so the three MXFP branch formats arrive in one encoding)
- *   sL1, sL2  fp32 powers of two: [ceil(K/32)][rank] (blocks of L1 along K) and [ceil(rank/32)][N] (of L2 along rank) */
+ *   sL1, sL2  fp32 powers of two: [ceil(K/32)][rank] (blocks of L1 along K) and [ceil(rank/32)][N] (of L2 along rank)
+ * Integer MX layers with 8-bit activations (main_fmt = LQ_MAIN_MXINT4_A8): Wq_packed and sw as for MXINT4;
+ *   L1, L2    int8 codes [K][rank] and [rank][N], within [-127, 127] (LQ_BRANCH_MXINT8) or [-7, 7] (LQ_BRANCH_MXINT4)
+ *   sL1, sL2  fp32 powers of two 2^e, e in [-120, 120]: [ceil(K/32)][rank] and [ceil(rank/32)][N] */
 lq_status lq_layer_import(const lq_config* cfg, const uint8_t* Wq_packed, const uint16_t* sw,
                           const void* L1, const float* sL1, const void* L2, const float* sL2,
                           const uint16_t* bias, lq_layer** out);
@@ -226,6 +239,9 @@ lq_status lq_linear_forward_static(const lq_layer* layer, const void* X_f16_dev,
  * parity checks); NULL skips a part.  qx int8 [M][K], sx half bits [M][G] (MXINT4: the block
  * exponents e as int16 [M][G], since 2^e may lie below the fp16 range), qb int8 [M][K],
  * sXb float [M], tq int8 [M][rank] (W16A16: half bits [M][rank]), sT float [M].
+ * MXFP: qx and tq are the e4m3 bytes, sT the block exponents of the intermediate as floats [M][ceil(rank/32)].
+ * Integer MX with 8-bit activations: qx and tq are the int8 codes (16 hi + lo of the two stored digits), sx the
+ * block exponents as for MXINT4, sT the block exponents of the intermediate as floats [M][ceil(rank/32)].
  * Synchronises `cuda_stream`. */
 lq_status lq_act_export(const lq_act* act, int8_t* qx, uint16_t* sx, int8_t* qb, float* sXb,
                         void* tq, float* sT, void* cuda_stream);

@@ -15,8 +15,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liblq.so")
 
 LQ_OK = 0
-BRANCH = {"none": 0, "w16a16": 1, "w8a8": 2, "w6a6": 3, "w4a8": 4, "mxfp8": 5, "mxfp6": 6, "mxfp4": 7}
-MAIN_AUTO, MAIN_MXFP4 = 0, 2
+BRANCH = {"none": 0, "w16a16": 1, "w8a8": 2, "w6a6": 3, "w4a8": 4, "mxfp8": 5, "mxfp6": 6, "mxfp4": 7,
+          "mxint8": 8, "mxint4": 9}
+MAIN_AUTO, MAIN_MXFP4, MAIN_MXINT4_A8 = 0, 2, 3
 BRANCH_NAME = {v: k for k, v in BRANCH.items()}
 OUT_F16, OUT_F32 = 0, 1
 GROUP = 64
@@ -190,6 +191,9 @@ def lq_layer_export(layer) -> dict:
     if cfg.main_fmt == MAIN_MXFP4 and r > 0:
         L1, L2 = np.zeros((K, r), np.uint8), np.zeros((r, N), np.uint8)               # e4m3 bit patterns
         sL1, sL2 = np.zeros((G, r), np.float32), np.zeros((-(-r // 32), N), np.float32)
+    elif cfg.main_fmt == MAIN_MXINT4_A8 and r > 0:
+        L1, L2 = np.zeros((K, r), np.int8), np.zeros((r, N), np.int8)                 # integer codes
+        sL1, sL2 = np.zeros((G, r), np.float32), np.zeros((-(-r // 32), N), np.float32)   # block scales 2^e
     elif r > 0 and cfg.branch == BRANCH["w16a16"]:
         L1, L2 = np.zeros((K, r), np.float16), np.zeros((r, N), np.float16)
     elif r > 0:
@@ -250,9 +254,9 @@ def lq_linear_forward_static(layer, X_dev_ptr: int, M: int, Y_dev_ptr: int, dtyp
 
 def lq_act_export(act, M: int, cfg: LqConfig, stream: int = 0) -> dict:
     K, r, G = cfg.K, cfg.rank, -(-cfg.K // cfg.group)
-    if cfg.main_fmt == MAIN_MXFP4:
-        # MXFP: qx / tq are e4m3 bit patterns (decode with e4m3_decode), sx the int16 block exponents of X,
-        # sT the block exponents of the rank-r intermediate as floats [M, ceil(r/32)]
+    if cfg.main_fmt in (MAIN_MXFP4, MAIN_MXINT4_A8):
+        # MXFP: qx / tq are e4m3 bit patterns (decode with e4m3_decode); integer MX with 8-bit activations: the int8 codes.
+        # sx: the int16 block exponents of X; sT: the block exponents of the rank-r intermediate as floats [M, ceil(r/32)]
         out = {"qx": np.zeros((M, K), np.int8), "sx": np.zeros((M, G), np.int16), "qb": None, "sXb": None, "tq": None, "sT": None}
         if r > 0 and cfg.branch != BRANCH["none"]:
             out["tq"] = np.zeros((M, r), np.int8)

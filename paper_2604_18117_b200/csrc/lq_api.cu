@@ -85,19 +85,26 @@ extern "C" lq_status lq_config_default(lq_config* cfg, int32_t K, int32_t N, int
   cfg->rot_steps = 0; cfg->rot_lr = 0.5f; cfg->seed = 0;
   cfg->main_fmt = LQ_MAIN_AUTO; cfg->reserved = 0;
   if (lq_branch_is_mxfp(branch)) { cfg->main_fmt = LQ_MAIN_MXFP4; cfg->group = LQ_MX_BLOCK; cfg->lr = 1e-3f; }
+  if (lq_branch_is_mxint(branch)) { cfg->main_fmt = LQ_MAIN_MXINT4_A8; cfg->group = LQ_MX_BLOCK; }
   return LQ_OK;
 }
 
 static lq_status check_config(const lq_config* c) {
   if (!c) return LQ_ERR_INVALID_ARG;
   if (c->K <= 0 || c->N <= 0 || c->rank < 0) return LQ_ERR_INVALID_ARG;
-  if (c->branch < LQ_BRANCH_NONE || c->branch > LQ_BRANCH_MXFP4) return LQ_ERR_INVALID_ARG;
+  if (c->branch < LQ_BRANCH_NONE || c->branch > LQ_BRANCH_MXINT4) return LQ_ERR_INVALID_ARG;
   if (c->group != LQ_GROUP && c->group != LQ_MX_BLOCK) return LQ_ERR_UNSUPPORTED;
-  if (c->main_fmt != LQ_MAIN_AUTO && c->main_fmt != LQ_MAIN_MXFP4) return LQ_ERR_INVALID_ARG;
+  if (c->main_fmt != LQ_MAIN_AUTO && c->main_fmt != LQ_MAIN_MXFP4 && c->main_fmt != LQ_MAIN_MXINT4_A8) return LQ_ERR_INVALID_ARG;
   // MXFP4 weights go with blocks of 32 and an MXFP (or no) branch; MXFP branches go with nothing else
   if (c->main_fmt == LQ_MAIN_MXFP4 && (c->group != LQ_MX_BLOCK || !(c->branch == LQ_BRANCH_NONE || lq_branch_is_mxfp(c->branch))))
     return LQ_ERR_UNSUPPORTED;
   if (c->main_fmt != LQ_MAIN_MXFP4 && lq_branch_is_mxfp(c->branch)) return LQ_ERR_UNSUPPORTED;
+  // MXINT8 activations go with MXINT4 weights in blocks of 32 and an integer MX (or no) branch of rank <= 64 (the two
+  // digit planes of the rank-r intermediate share the 128-byte container)
+  if (c->main_fmt == LQ_MAIN_MXINT4_A8 &&
+      (c->group != LQ_MX_BLOCK || !(c->branch == LQ_BRANCH_NONE || lq_branch_is_mxint(c->branch)) || (c->branch != LQ_BRANCH_NONE && c->rank > 64)))
+    return LQ_ERR_UNSUPPORTED;
+  if (c->main_fmt != LQ_MAIN_MXINT4_A8 && lq_branch_is_mxint(c->branch)) return LQ_ERR_UNSUPPORTED;
   if (c->K > LQ_MAX_K || (c->K % 8) != 0) return LQ_ERR_UNSUPPORTED;
   if ((c->N % 8) != 0) return LQ_ERR_UNSUPPORTED;
   if (c->rank > LQ_MAX_RANK) return LQ_ERR_UNSUPPORTED;
@@ -117,11 +124,12 @@ lq_layer* lq_layer_new(const lq_config* cfg) {
   L->cfg.rank = L->r;
   L->mx = cfg->group == LQ_MX_BLOCK;
   L->mxfp = cfg->main_fmt == LQ_MAIN_MXFP4;
+  L->a8 = cfg->main_fmt == LQ_MAIN_MXINT4_A8;
   L->G = lq_ceil_div(L->K, cfg->group);
   L->Kpad = lq_round_up(L->K, LQ_KSTAGE);
   L->Gpad = L->Kpad / LQ_GROUP;
   L->Npad = lq_round_up(L->N, LQ_BN);
-  L->integer_branch = L->r > 0 && L->cfg.branch != LQ_BRANCH_W16A16 && !lq_branch_is_mxfp(L->cfg.branch);
+  L->integer_branch = L->r > 0 && L->cfg.branch != LQ_BRANCH_W16A16 && !lq_branch_is_mxfp(L->cfg.branch) && !lq_branch_is_mxint(L->cfg.branch);
   L->f16_branch = L->r > 0 && L->cfg.branch == LQ_BRANCH_W16A16;
   L->has_bias = false;
   L->device = -1;
@@ -228,6 +236,20 @@ extern "C" lq_status lq_layer_import(const lq_config* cfg, const uint8_t* Wq_pac
       const uint16_t* a = (const uint16_t*)L1; const uint16_t* b = (const uint16_t*)L2;
       L->L1h.assign(a, a + (size_t)K * r);
       L->L2h.assign(b, b + (size_t)r * N);
+    } else if (L->a8 && r > 0) {
+      if (!sL1 || !sL2) { delete L; return LQ_ERR_INVALID_ARG; }
+      const int qm = L->cfg.branch == LQ_BRANCH_MXINT8 ? 127 : 7;
+      const int nbK = lq_ceil_div(K, LQ_MX_BLOCK), nbR = lq_ceil_div(r, LQ_MX_BLOCK);
+      const int8_t* a = (const int8_t*)L1; const int8_t* b = (const int8_t*)L2;
+      L->L1q.assign(a, a + (size_t)K * r);
+      L->L2q.assign(b, b + (size_t)r * N);
+      for (int8_t v : L->L1q) if (v > qm || v < -qm) { delete L; return LQ_ERR_INVALID_ARG; }
+      for (int8_t v : L->L2q) if (v > qm || v < -qm) { delete L; return LQ_ERR_INVALID_ARG; }
+      L->s1b.assign(sL1, sL1 + (size_t)nbK * r);
+      L->s2b.assign(sL2, sL2 + (size_t)nbR * N);
+      int e = 0;
+      for (float v : L->s1b) if (!pow2_exponent(v, &e) || e < -120 || e > 120) { delete L; return LQ_ERR_INVALID_ARG; }
+      for (float v : L->s2b) if (!pow2_exponent(v, &e) || e < -120 || e > 120) { delete L; return LQ_ERR_INVALID_ARG; }
     }
     if (bias) { L->bias.assign(bias, bias + N); L->has_bias = true; }
   } catch (const std::bad_alloc&) { delete L; return LQ_ERR_ALLOC; }
@@ -270,6 +292,11 @@ extern "C" lq_status lq_layer_export(const lq_layer* L, uint8_t* Wq_packed, uint
   } else if (L->f16_branch) {
     if (L1) memcpy(L1, L->L1h.data(), (size_t)K * r * 2);
     if (L2) memcpy(L2, L->L2h.data(), (size_t)r * N * 2);
+  } else if (L->a8 && r > 0) {
+    if (L1) memcpy(L1, L->L1q.data(), (size_t)K * r);
+    if (L2) memcpy(L2, L->L2q.data(), (size_t)r * N);
+    if (sL1) memcpy(sL1, L->s1b.data(), L->s1b.size() * sizeof(float));
+    if (sL2) memcpy(sL2, L->s2b.data(), L->s2b.size() * sizeof(float));
   }
   if (bias && L->has_bias) memcpy(bias, L->bias.data(), N * sizeof(uint16_t));
   return LQ_OK;
@@ -436,7 +463,7 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
       for (int n = 0; n < N; ++n) s2[n] = L->sL2[n];
       for (int j = 0; j < r; ++j)
         for (int n = 0; n < N; ++n) l2c[(size_t)n * LQ_RCONT + j] = (uint8_t)L->L2q[(size_t)j * N + n];
-    } else if (L->mxfp && r > 0) {
+    } else if ((L->mxfp || L->a8) && r > 0) {
       // B fragments of mma.sync.m16n8k32 (e4m3) for the MXFP quantizer, whose lanes hold two runs of eight values per
       // box (one per block of 32): lane 4 c + t carries k = 64 box + 32 j + 8 t + 0..7 of column 8 tile + c, j = 0, 1
       const int ntiles = lq_quant_rank_tiles(r, false), nbox = Kpad / 64, rpad = ntiles * 8;
@@ -449,7 +476,7 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
             for (int blk = 0; blk < 2; ++blk)
               for (int i = 0; i < 8; ++i) {
                 const int k = b * 64 + 32 * blk + 8 * (lane & 3) + i;
-                dst[8 * blk + i] = (j < r && k < K) ? L->L1e[(size_t)k * r + j] : 0;
+                dst[8 * blk + i] = (j < r && k < K) ? (L->a8 ? (uint8_t)L->L1q[(size_t)k * r + j] : L->L1e[(size_t)k * r + j]) : 0;
               }
           }
       if ((st = upload(&L->d_L1f, l1f)) != LQ_OK) return st;
@@ -457,16 +484,36 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
       for (int b = 0; b < lq_ceil_div(K, 32); ++b)
         for (int j = 0; j < r; ++j) s1b[(size_t)b * rpad + j] = L->s1b[(size_t)b * r + j];
       if ((st = upload(&L->d_s1b, s1b)) != LQ_OK) return st;
-      for (int j = 0; j < r; ++j)
-        for (int n = 0; n < N; ++n) l2c[(size_t)n * LQ_RCONT + j] = L->L2e[(size_t)j * N + n];
       // E8M0 bytes of L2's block scales along the rank, one 128-byte-of-rank stage: [1][Npad/128][512]
       std::vector<uint8_t> sfl2((size_t)(Npad / 128) * 512, 127);
-      for (int c = 0; c < lq_ceil_div(r, 32); ++c)
-        for (int n = 0; n < N; ++n) {
-          int e = 0;
-          pow2_exponent(L->s2b[(size_t)c * N + n], &e);
-          sfl2[lq_sfb_offset(n, c, Npad)] = (uint8_t)(e + 127);
-        }
+      if (L->a8) {
+        // two digit planes, code = 16 hi + lo: hi digits of rank index j at byte j, lo digits at byte 64 + j (rank <= 64);
+        // the four 32-byte K blocks of the stage are (hi, block 0), (hi, block 1), (lo, block 0), (lo, block 1) with
+        // scales 2^(e+4), 2^(e+4), 2^e, 2^e
+        for (int j = 0; j < r; ++j)
+          for (int n = 0; n < N; ++n) {
+            int hi, lo;
+            lq_split_digits(L->L2q[(size_t)j * N + n], &hi, &lo);
+            l2c[(size_t)n * LQ_RCONT + j] = lq_digit_e4m3(hi);
+            l2c[(size_t)n * LQ_RCONT + 64 + j] = lq_digit_e4m3(lo);
+          }
+        for (int c = 0; c < lq_ceil_div(r, 32); ++c)
+          for (int n = 0; n < N; ++n) {
+            int e = 0;
+            pow2_exponent(L->s2b[(size_t)c * N + n], &e);
+            sfl2[lq_sfb_offset(n, c, Npad)] = (uint8_t)(e + 4 + 127);
+            sfl2[lq_sfb_offset(n, 2 + c, Npad)] = (uint8_t)(e + 127);
+          }
+      } else {
+        for (int j = 0; j < r; ++j)
+          for (int n = 0; n < N; ++n) l2c[(size_t)n * LQ_RCONT + j] = L->L2e[(size_t)j * N + n];
+        for (int c = 0; c < lq_ceil_div(r, 32); ++c)
+          for (int n = 0; n < N; ++n) {
+            int e = 0;
+            pow2_exponent(L->s2b[(size_t)c * N + n], &e);
+            sfl2[lq_sfb_offset(n, c, Npad)] = (uint8_t)(e + 127);
+          }
+      }
       if ((st = upload(&L->d_sfl2, sfl2)) != LQ_OK) return st;
     } else if (L->f16_branch) {
       // the same fragment order with 16 halves per lane (mma.sync.m16n8k16, four k steps per box)
@@ -512,31 +559,31 @@ extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device,
   if (!A) return LQ_ERR_ALLOC;
   memset(A, 0, sizeof(*A));
   A->K = L->K; A->N = L->N; A->r = L->r; A->G = L->G; A->Kpad = L->Kpad; A->Gpad = L->Gpad;
-  A->mx = L->mx; A->mxfp = L->mxfp;
+  A->mx = L->mx; A->mxfp = L->mxfp; A->a8 = L->a8; A->planes = L->a8 ? 2 : 1;
   A->branch = L->cfg.branch; A->M_max = M_max; A->Mpad = lq_round_up(M_max, LQ_BM);
   A->device = device; A->main_kind = L->main_kind; A->M = 0;
   if (cudaSetDevice(device) != cudaSuccess) { delete A; return LQ_ERR_CUDA; }
-  const size_t Mp = A->Mpad, Kp = A->Kpad;
-  bool ok = cudaMalloc((void**)&A->d_qx8, Mp * Kp) == cudaSuccess &&
+  const size_t Mp = A->Mpad, Kp = A->Kpad, Kx = (size_t)A->planes * Kp;   // Kx: bytes per row of the main codes
+  bool ok = cudaMalloc((void**)&A->d_qx8, Mp * Kx) == cudaSuccess &&
             cudaMalloc((void**)&A->d_sx, (size_t)A->Gpad * Mp * sizeof(float)) == cudaSuccess &&
             cudaMalloc((void**)&A->d_qb, Mp * Kp) == cudaSuccess &&
             cudaMalloc((void**)&A->d_sXb, Mp * sizeof(float)) == cudaSuccess &&
             cudaMalloc((void**)&A->d_tq, Mp * LQ_RCONT) == cudaSuccess &&
             cudaMalloc((void**)&A->d_sT, Mp * sizeof(float)) == cudaSuccess &&
-            (!A->mx || cudaMalloc((void**)&A->d_sfa, (Mp / 128) * (Kp / 128) * 512) == cudaSuccess) &&
-            (!A->mxfp || cudaMalloc((void**)&A->d_sft, (Mp / 128) * 512) == cudaSuccess);
+            (!A->mx || cudaMalloc((void**)&A->d_sfa, (Mp / 128) * (Kx / 128) * 512) == cudaSuccess) &&
+            (!(A->mxfp || A->a8) || cudaMalloc((void**)&A->d_sft, (Mp / 128) * 512) == cudaSuccess);
   if (!ok) { lq_act_free(A); return LQ_ERR_ALLOC; }
   // padding rows/columns are read by the GEMM's tiles: start from defined contents
-  cudaMemset(A->d_qx8, 0, Mp * Kp);
+  cudaMemset(A->d_qx8, 0, Mp * Kx);
   cudaMemset(A->d_sx, 0, (size_t)A->Gpad * Mp * sizeof(float));
   cudaMemset(A->d_qb, 0, Mp * Kp);
   cudaMemset(A->d_sXb, 0, Mp * sizeof(float));
   cudaMemset(A->d_tq, 0, Mp * LQ_RCONT);
   cudaMemset(A->d_sT, 0, Mp * sizeof(float));
-  if (A->mx) cudaMemset(A->d_sfa, 127, (Mp / 128) * (Kp / 128) * 512);
-  if (A->mxfp) cudaMemset(A->d_sft, 127, (Mp / 128) * 512);
+  if (A->mx) cudaMemset(A->d_sfa, 127, (Mp / 128) * (Kx / 128) * 512);
+  if (A->mxfp || A->a8) cudaMemset(A->d_sft, 127, (Mp / 128) * 512);
   lq_status st;
-  if ((st = lq_make_tmap_bytes(&A->tmA, A->d_qx8, Mp, Kp, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
+  if ((st = lq_make_tmap_bytes(&A->tmA, A->d_qx8, Mp, Kx, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
   if ((st = lq_make_tmap_bytes(&A->tmT, A->d_tq, Mp, LQ_RCONT, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
   if (cudaDeviceSynchronize() != cudaSuccess) { lq_act_free(A); return LQ_ERR_CUDA; }
   *out = A;
@@ -559,7 +606,7 @@ extern "C" lq_status lq_act_free(lq_act* A) {
 
 static bool act_matches(const lq_layer* L, const lq_act* A) {
   return L && A && L->device == A->device && L->device >= 0 && L->K == A->K && L->N == A->N && L->r == A->r &&
-         L->cfg.branch == A->branch && L->main_kind == A->main_kind && L->mx == A->mx && L->mxfp == A->mxfp;
+         L->cfg.branch == A->branch && L->main_kind == A->main_kind && L->mx == A->mx && L->mxfp == A->mxfp && L->a8 == A->a8;
 }
 
 extern "C" lq_status lq_quantize_act(const lq_layer* L, const void* X, int32_t M, lq_act* A, void* stream) {
@@ -628,16 +675,16 @@ static lq_status forward_host(const lq_layer* L, lq_act* A, const void* Xh, int3
     // a view of the activation record that starts at row m0 (m0 is a multiple of the row tile)
     lq_act V = *A;
     V.M = Mc; V.M_max = Mc;
-    V.d_qx8 = A->d_qx8 + (size_t)m0 * A->Kpad;
+    V.d_qx8 = A->d_qx8 + (size_t)m0 * A->Kpad * A->planes;
     V.d_qb = A->d_qb + (size_t)m0 * A->Kpad;
     V.d_sx = A->d_sx + m0;                                     // [Gpad][Mpad]: the row stride stays Mpad
     V.d_sXb = A->d_sXb + m0;
     V.d_tq = A->d_tq + (size_t)m0 * LQ_RCONT;
     V.d_sT = A->d_sT + m0;
-    if (A->mx) V.d_sfa = A->d_sfa + (size_t)(m0 / 128) * (A->Kpad / 128) * 512;
-    if (A->mxfp) V.d_sft = A->d_sft + (size_t)(m0 / 128) * 512;
+    if (A->mx) V.d_sfa = A->d_sfa + (size_t)(m0 / 128) * (A->Kpad / 128) * A->planes * 512;
+    if (A->mxfp || A->a8) V.d_sft = A->d_sft + (size_t)(m0 / 128) * 512;
     lq_status s;
-    if ((s = lq_make_tmap_bytes(&V.tmA, V.d_qx8, (uint64_t)(A->Mpad - m0), A->Kpad, LQ_BM)) != LQ_OK) return s;
+    if ((s = lq_make_tmap_bytes(&V.tmA, V.d_qx8, (uint64_t)(A->Mpad - m0), (uint64_t)A->Kpad * A->planes, LQ_BM)) != LQ_OK) return s;
     if ((s = lq_make_tmap_bytes(&V.tmT, V.d_tq, (uint64_t)(A->Mpad - m0), LQ_RCONT, LQ_BM)) != LQ_OK) return s;
     if ((s = lq_launch_quantize(L, xd, Mc, &V, st)) != LQ_OK) return s;
     if ((s = (L->mx ? lq_launch_gemm_mx(L, &V, yd, dt, st) : lq_launch_gemm(L, &V, yd, dt, st))) != LQ_OK) return s;
@@ -673,6 +720,13 @@ static int decode_code(uint8_t b, int kind) {
   return (b & 0x80) ? -mag : mag;
 }
 
+// value of a digit byte written by the MXINT8 quantizer (an E4M3 image of an integer in [-8, 8])
+static int decode_digit(uint8_t b) {
+  for (int d = -8; d <= 8; ++d)
+    if (lq_digit_e4m3(d) == b) return d;
+  return (b & 0x7F) == 0 ? 0 : 99;   // -0 reads as 0; anything else surfaces as a parity failure
+}
+
 extern "C" lq_status lq_act_export(const lq_act* A, int8_t* qx, uint16_t* sx, int8_t* qb, float* sXb, void* tq,
                                    float* sT, void* stream) {
   if (!A || A->M <= 0) return LQ_ERR_INVALID_ARG;
@@ -682,7 +736,13 @@ extern "C" lq_status lq_act_export(const lq_act* A, int8_t* qx, uint16_t* sx, in
   const int M = A->M, K = A->K, G = A->G, r = A->r;
   const size_t Kp = A->Kpad, Mp = A->Mpad;
   try {
-    if (qx) {
+    if (qx && A->a8) {
+      std::vector<uint8_t> h((size_t)M * 2 * Kp);
+      CUDA_OK(cudaMemcpy(h.data(), A->d_qx8, h.size(), cudaMemcpyDeviceToHost));
+      for (int m = 0; m < M; ++m)
+        for (int k = 0; k < K; ++k)
+          qx[(size_t)m * K + k] = (int8_t)(16 * decode_digit(h[(size_t)m * 2 * Kp + k]) + decode_digit(h[(size_t)m * 2 * Kp + Kp + k]));
+    } else if (qx) {
       std::vector<uint8_t> h((size_t)M * Kp);
       CUDA_OK(cudaMemcpy(h.data(), A->d_qx8, h.size(), cudaMemcpyDeviceToHost));
       for (int m = 0; m < M; ++m)
@@ -690,11 +750,12 @@ extern "C" lq_status lq_act_export(const lq_act* A, int8_t* qx, uint16_t* sx, in
           qx[(size_t)m * K + k] = A->mxfp ? (int8_t)h[m * Kp + k] : (int8_t)decode_code(h[m * Kp + k], A->main_kind);
     }
     if (sx && A->mx) {
-      std::vector<uint8_t> h((Mp / 128) * (Kp / 128) * 512);
+      const size_t Kx = (size_t)A->planes * Kp;                   // a8: the lo plane's scale bytes carry e itself
+      std::vector<uint8_t> h((Mp / 128) * (Kx / 128) * 512);
       CUDA_OK(cudaMemcpy(h.data(), A->d_sfa, h.size(), cudaMemcpyDeviceToHost));
       for (int m = 0; m < M; ++m)
         for (int g = 0; g < G; ++g) {
-          const int e = (int)h[lq_sf_offset(m, g, (int)Kp)] - 127;
+          const int e = (int)h[lq_sf_offset(m, g + (A->a8 ? (int)(Kp / 32) : 0), (int)Kx)] - 127;
           sx[(size_t)m * G + g] = (uint16_t)(int16_t)e;            // MXINT4: the block exponent itself (scale 2^e)
         }
     } else if (sx) {
@@ -706,19 +767,33 @@ extern "C" lq_status lq_act_export(const lq_act* A, int8_t* qx, uint16_t* sx, in
           sx[(size_t)m * G + g] = __half_raw(v).x;
         }
     }
-    if (qb && A->branch != LQ_BRANCH_NONE && A->branch != LQ_BRANCH_W16A16 && !A->mxfp) {
+    if (qb && A->branch != LQ_BRANCH_NONE && A->branch != LQ_BRANCH_W16A16 && !A->mxfp && !A->a8) {
       std::vector<int8_t> h((size_t)M * Kp);
       CUDA_OK(cudaMemcpy(h.data(), A->d_qb, h.size(), cudaMemcpyDeviceToHost));
       for (int m = 0; m < M; ++m) memcpy(qb + (size_t)m * K, h.data() + m * Kp, K);
     }
-    if (sXb && r > 0 && !A->mxfp) CUDA_OK(cudaMemcpy(sXb, A->d_sXb, M * sizeof(float), cudaMemcpyDeviceToHost));
+    if (sXb && r > 0 && !A->mxfp && !A->a8) CUDA_OK(cudaMemcpy(sXb, A->d_sXb, M * sizeof(float), cudaMemcpyDeviceToHost));
     if (tq && r > 0) {
       std::vector<uint8_t> h((size_t)M * LQ_RCONT);
       CUDA_OK(cudaMemcpy(h.data(), A->d_tq, h.size(), cudaMemcpyDeviceToHost));
       const int eb = A->branch == LQ_BRANCH_W16A16 ? 2 : 1;
-      for (int m = 0; m < M; ++m) memcpy((uint8_t*)tq + (size_t)m * r * eb, h.data() + (size_t)m * LQ_RCONT, (size_t)r * eb);
+      if (A->a8) {
+        for (int m = 0; m < M; ++m)
+          for (int j = 0; j < r; ++j)
+            ((int8_t*)tq)[(size_t)m * r + j] =
+                (int8_t)(16 * decode_digit(h[(size_t)m * LQ_RCONT + j]) + decode_digit(h[(size_t)m * LQ_RCONT + 64 + j]));
+      } else {
+        for (int m = 0; m < M; ++m) memcpy((uint8_t*)tq + (size_t)m * r * eb, h.data() + (size_t)m * LQ_RCONT, (size_t)r * eb);
+      }
     }
-    if (sT && r > 0 && A->mxfp) {
+    if (sT && r > 0 && A->a8) {
+      // the block exponents of the rank-r intermediate (the lo plane's scale bytes), as floats [M][ceil(r/32)]
+      std::vector<uint8_t> h((Mp / 128) * 512);
+      CUDA_OK(cudaMemcpy(h.data(), A->d_sft, h.size(), cudaMemcpyDeviceToHost));
+      const int nbR = lq_ceil_div(r, LQ_MX_BLOCK);
+      for (int m = 0; m < M; ++m)
+        for (int c = 0; c < nbR; ++c) sT[(size_t)m * nbR + c] = (float)((int)h[lq_sf_offset(m, 2 + c, 128)] - 127);
+    } else if (sT && r > 0 && A->mxfp) {
       // MXFP: the block exponents of the rank-r intermediate as floats, [M][ceil(r/32)]
       std::vector<uint8_t> h((Mp / 128) * 512);
       CUDA_OK(cudaMemcpy(h.data(), A->d_sft, h.size(), cudaMemcpyDeviceToHost));

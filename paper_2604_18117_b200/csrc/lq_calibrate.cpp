@@ -325,6 +325,37 @@ void quant_mx_columns(const std::vector<double>& F, int rows, int cols, const El
   }
 }
 
+// MX integer quantizer of F [rows][cols] with blocks of 32 down each column (Appendix A.3 "MX Formats": MXINT8 / MXINT4):
+// the block's exponent is the smallest e with qmax 2^e >= max|v| (0 for an all-zero block, whose codes are zeros), codes
+// rint_even(v / 2^e) within [-qmax, qmax].  scales: 2^e as float, [ceil(rows/32)][cols]; Dq: dequantized values.
+void quant_mxint_columns(const std::vector<double>& F, int rows, int cols, int bits, int8_t* codes, float* scales, double* Dq) {
+  const int nb = lq_ceil_div(rows, 32);
+  const double qmax = (double)((1 << (bits - 1)) - 1);
+#pragma omp parallel for schedule(static)
+  for (int b = 0; b < nb; ++b) {
+    const int t0 = b * 32, t1 = std::min(rows, t0 + 32);
+    for (int c = 0; c < cols; ++c) {
+      double a = 0.0;
+      for (int t = t0; t < t1; ++t) a = std::max(a, fabs(F[(size_t)t * cols + c]));
+      int e = 0;
+      if (a > 0.0) {
+        int x = 0;
+        const double m = frexp(a, &x);                            // a = m 2^x, m in [0.5, 1)
+        e = (m <= qmax / ldexp(1.0, bits - 1)) ? x - (bits - 1) : x - (bits - 2);
+        e = std::max(-127, std::min(127, e));
+      }
+      const double sc = ldexp(1.0, e);
+      scales[(size_t)b * cols + c] = (float)sc;
+      for (int t = t0; t < t1; ++t) {
+        double q = nearbyint(F[(size_t)t * cols + c] / sc);
+        q = std::max(-qmax, std::min(qmax, q));
+        codes[(size_t)t * cols + c] = (int8_t)q;
+        Dq[(size_t)t * cols + c] = q * sc;
+      }
+    }
+  }
+}
+
 // One fp32 scale per column of F [rows][cols]; codes [rows][cols].
 void quant_columns(const std::vector<double>& F, int rows, int cols, int bits, int8_t* codes, float* scales) {
   const float qm = (float)((1 << (bits - 1)) - 1);
@@ -491,8 +522,11 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
                                   double* trace) {
   if (!cfg || !W16 || !out) return LQ_ERR_INVALID_ARG;
   if (cfg->K <= 0 || cfg->N <= 0 || cfg->rank < 0 || cfg->steps < 0) return LQ_ERR_INVALID_ARG;
-  if (cfg->branch < LQ_BRANCH_NONE || cfg->branch > LQ_BRANCH_MXFP4) return LQ_ERR_INVALID_ARG;
+  if (cfg->branch < LQ_BRANCH_NONE || cfg->branch > LQ_BRANCH_MXINT4) return LQ_ERR_INVALID_ARG;
   const bool mxfp = cfg->main_fmt == LQ_MAIN_MXFP4;
+  const bool a8 = cfg->main_fmt == LQ_MAIN_MXINT4_A8;
+  if (a8 ? !(cfg->branch == LQ_BRANCH_NONE || lq_branch_is_mxint(cfg->branch)) : lq_branch_is_mxint(cfg->branch)) return LQ_ERR_UNSUPPORTED;
+  if (a8 && (cfg->group != LQ_MX_BLOCK || cfg->rot_steps > 0 || (cfg->branch != LQ_BRANCH_NONE && cfg->rank > 64))) return LQ_ERR_UNSUPPORTED;
   if (mxfp ? !(cfg->branch == LQ_BRANCH_NONE || lq_branch_is_mxfp(cfg->branch)) : lq_branch_is_mxfp(cfg->branch)) return LQ_ERR_UNSUPPORTED;
   if (mxfp && (cfg->group != LQ_MX_BLOCK || cfg->rot_steps > 0)) return LQ_ERR_UNSUPPORTED;   // no rotation step for MXFP factors yet
   if ((cfg->group != LQ_GROUP && cfg->group != LQ_MX_BLOCK) || cfg->rot_steps < 0) return LQ_ERR_UNSUPPORTED;
@@ -605,6 +639,12 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
       Lr->s1b.resize((size_t)lq_ceil_div(K, 32) * r); Lr->s2b.resize((size_t)lq_ceil_div(r, 32) * N);
       quant_mx_columns(L1, K, r, f, Lr->L1e.data(), Lr->s1b.data(), L1d.data());   // blocks along K per column of L1
       quant_mx_columns(L2, r, N, f, Lr->L2e.data(), Lr->s2b.data(), L2d.data());   // blocks along the rank per column of L2
+    } else if (a8) {
+      const int bw = cfg->branch == LQ_BRANCH_MXINT8 ? 8 : 4;
+      Lr->L1q.resize(L1.size()); Lr->L2q.resize(L2.size());
+      Lr->s1b.resize((size_t)lq_ceil_div(K, 32) * r); Lr->s2b.resize((size_t)lq_ceil_div(r, 32) * N);
+      quant_mxint_columns(L1, K, r, bw, Lr->L1q.data(), Lr->s1b.data(), L1d.data());   // blocks along K per column of L1
+      quant_mxint_columns(L2, r, N, bw, Lr->L2q.data(), Lr->s2b.data(), L2d.data());   // blocks along the rank per column of L2
     } else if (Lr->f16_branch) {
       Lr->L1h.resize(L1.size()); Lr->L2h.resize(L2.size());
       for (size_t i = 0; i < L1.size(); ++i) { Lr->L1h[i] = float_to_half_bits((float)L1[i]); L1d[i] = half_bits_to_float(Lr->L1h[i]); }

@@ -216,9 +216,10 @@ constexpr uint32_t IDESC_I8 = (2u << 4) | (1u << 7) | (1u << 10);    // S8 x S8 
 constexpr uint32_t IDESC_F8 = (1u << 4) | (0u << 7) | (0u << 10);    // E4M3 x E4M3 -> F32
 constexpr uint32_t IDESC_F16 = (1u << 4) | (0u << 7) | (0u << 10);   // F16 x F16 -> F32
 // instruction descriptor of the block-scaled kind: E4M3 x E4M3, E8M0 scales, K-major operands, scale-byte ids
-__device__ __forceinline__ constexpr uint32_t idesc_mx(int n, int sf_id) {
-  return ((uint32_t)sf_id << 4) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(LQ_BM >> 4) << 24) | ((uint32_t)sf_id << 29);
+__device__ __forceinline__ constexpr uint32_t idesc_mx2(int n, int a_sf_id, int b_sf_id) {
+  return ((uint32_t)b_sf_id << 4) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(LQ_BM >> 4) << 24) | ((uint32_t)a_sf_id << 29);
 }
+__device__ __forceinline__ constexpr uint32_t idesc_mx(int n, int sf_id) { return idesc_mx2(n, sf_id, sf_id); }
 
 // ---- timeline build (-DLQ_TIMELINE): per-role clock stamps of CTA 0 ----------------------
 // A stamp is one 8-byte store by lane 0 of the stamping warp: (event id << 48) | (tag << 40) | (clock64 & 2^40-1),

@@ -71,10 +71,14 @@ constexpr int TM_BR = 256, TM_SFA = 256, TM_SFB = TM_SFA + 4, TM_SF_ALIASED = 16
 
 struct MxParams {
   int M, N, Mpad, Npad;
-  int k_stages;           // Kpad / 128
+  int k_stages;           // stages of A per tile: Kpad / 128, times two when 8-bit activation codes come as two digit planes
+  int b_wrap;             // Kpad / 128: stage s reads B (and its scales) at stage s mod b_wrap - the planes share the weights
   int branch_steps;       // 0: no branch; else MMAs of the branch stage (32 bytes of r each)
   int branch_f16;         // the branch operands are halves (W16A16 reference branch): no scales, summed by the tensor core
-  int branch_mx;          // the branch is MXFP as well: its up-projection is one more block-scaled stage onto the main accumulator
+  int branch_mx;          // the branch is MX as well: its up-projection is one more block-scaled stage onto the main
+                          // accumulator.  1: MXFP elements, K blocks in order.  2: 8-bit integer codes as digit planes on
+                          // both sides - the stage's four K blocks are (hi, 0), (hi, 1), (lo, 0), (lo, 1) and every
+                          // (plane of T, plane of L2) pair of the same rank block is one MMA
   const uint8_t* sft;     // branch_mx: E8M0 bytes of T's block scales, [Mpad/128][512]
   const uint8_t* sfl2;    // branch_mx: E8M0 bytes of L2's block scales, [Npad/128][512]
   int tiles_m, units_n;
@@ -216,11 +220,12 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const uint32_t full = bar(B_FULL + st);
         if (elect_one()) {
           mbar_expect_tx(full, STAGE_A_BYTES + width * (UNIT * LQ_KSTAGE) + (1 + width) * SF_BYTES);
+          const int sb = s >= p.b_wrap ? s - p.b_wrap : s;       // the lo digits' plane runs over the same weights
           tma_load_2d(a_dst, &tmA, s * LQ_KSTAGE, m0, full);
-          if (width == 2) tma_load_2d(b_dst, &tmB2, s * LQ_KSTAGE, n0, full);
-          else tma_load_2d(b_dst, &tmB, s * LQ_KSTAGE, n0, full);
+          if (width == 2) tma_load_2d(b_dst, &tmB2, sb * LQ_KSTAGE, n0, full);
+          else tma_load_2d(b_dst, &tmB, sb * LQ_KSTAGE, n0, full);
           bulk_load(sf_dst, sfa + (size_t)s * SF_BYTES, SF_BYTES, full);
-          bulk_load(sf_dst + SF_BYTES, sfb + (size_t)s * p.units_n * SF_BYTES, width * SF_BYTES, full);
+          bulk_load(sf_dst + SF_BYTES, sfb + (size_t)sb * p.units_n * SF_BYTES, width * SF_BYTES, full);
         }
         __syncwarp();
         LQ_TL(EV_P_ISSUED, s);
@@ -303,8 +308,16 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             tc_cp_sf(tsfa, make_smem_desc_plain(sf_addr, 16, 128));
             tc_cp_sf(tsfb, make_smem_desc_plain(sf_addr + SF_BYTES, 16, 128));
             if (width == 2) tc_cp_sf(tsfb + 4, make_smem_desc_plain(sf_addr + 2 * SF_BYTES, 16, 128));
-            for (int j = 0; j < p.branch_steps; ++j)
-              tc_mma_mx(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc_mx(ncols, j), tsfa, tsfb, 1u);
+            if (p.branch_mx == 2) {
+              for (int c = 0; c < p.branch_steps; ++c)
+                for (int q = 0; q < 4; ++q) {
+                  const int ja = c + 2 * (q >> 1), jb = c + 2 * (q & 1);   // K block of T's plane, of L2's plane
+                  tc_mma_mx(tmem_base, adesc + 2 * ja, bdesc + 2 * jb, idesc_mx2(ncols, ja, jb), tsfa, tsfb, 1u);
+                }
+            } else {
+              for (int j = 0; j < p.branch_steps; ++j)
+                tc_mma_mx(tmem_base, adesc + 2 * j, bdesc + 2 * j, idesc_mx(ncols, j), tsfa, tsfb, 1u);
+            }
           } else {
             for (int j = 0; j < p.branch_steps; ++j) {
               if (branch_acc) tc_mma<TC_I8>(tmem_base + TM_BR, adesc + 2 * j, bdesc + 2 * j, IDESC_I8 | idesc_shape(ncols), (uint32_t)j);
@@ -477,11 +490,12 @@ lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_
   if (!L->mx || !A->mx) return LQ_ERR_UNSUPPORTED;
   MxParams p;
   p.M = A->M; p.N = L->N; p.Mpad = A->Mpad; p.Npad = L->Npad;
-  p.k_stages = L->Kpad / LQ_KSTAGE;
+  p.b_wrap = L->Kpad / LQ_KSTAGE;
+  p.k_stages = p.b_wrap * A->planes;
   p.branch_f16 = L->f16_branch ? 1 : 0;
-  p.branch_mx = (L->mxfp && L->r > 0) ? 1 : 0;
+  p.branch_mx = L->r == 0 ? 0 : L->mxfp ? 1 : L->a8 ? 2 : 0;
   p.sft = A->d_sft; p.sfl2 = L->d_sfl2;
-  p.branch_steps = L->r == 0 ? 0 : lq_ceil_div(L->r, L->f16_branch ? 16 : 32);
+  p.branch_steps = L->r == 0 ? 0 : lq_ceil_div(L->r, L->f16_branch ? 16 : 32);   // a8: rank blocks of 32 (at most two)
   p.tiles_m = lq_ceil_div(A->M, LQ_BM);
   p.units_n = L->Npad / UNIT;
   p.sfa = A->d_sfa; p.sfb = L->d_sfb; p.sT = A->d_sT; p.sL2 = L->d_sL2; p.bias = L->d_bias;

@@ -40,6 +40,18 @@ static inline size_t lq_sfb_offset(int n, int kb, int Npad) {
 static inline bool lq_branch_is_mxfp(int branch) {
   return branch == LQ_BRANCH_MXFP8 || branch == LQ_BRANCH_MXFP6 || branch == LQ_BRANCH_MXFP4;
 }
+// An 8-bit code c in [-127, 127] as two digits, c = 16 hi + lo with lo in [-8, 7] and hi in [-8, 8]: both are exact
+// E4M3 values, so a block-scaled MMA can carry an 8-bit integer operand as two planes with scales 2^(e+4) and 2^e.
+static inline void lq_split_digits(int c, int* hi, int* lo) {
+  const int l = ((c + 8) & 15) - 8;
+  *lo = l; *hi = (c - l) / 16;
+}
+// E4M3 byte of an integer in [-8, 8] (bias 7, three mantissa bits; 8 = 1.0 * 2^3)
+static inline uint8_t lq_digit_e4m3(int d) {
+  static const uint8_t mag[9] = {0x00, 0x38, 0x40, 0x44, 0x48, 0x4A, 0x4C, 0x4E, 0x50};
+  return (uint8_t)((d < 0 ? 0x80 : 0x00) | mag[d < 0 ? -d : d]);
+}
+static inline bool lq_branch_is_mxint(int branch) { return branch == LQ_BRANCH_MXINT8 || branch == LQ_BRANCH_MXINT4; }
 static inline int lq_branch_wbits(int branch) {
   return branch == LQ_BRANCH_W8A8 ? 8 : branch == LQ_BRANCH_W6A6 ? 6 : branch == LQ_BRANCH_W4A8 ? 4 : 0;
 }
@@ -54,6 +66,8 @@ struct lq_layer {
   bool integer_branch, f16_branch, has_bias;
   bool mx;                     // MX main branch (cfg.group == 32): G counts blocks of 32, sw holds powers of two
   bool mxfp;                   // MXFP4 weights x MXFP8e4 activations (implies mx); the branch, if any, is MXFP too
+  bool a8;                     // MXINT4 weights x MXINT8 activations (implies mx): 8-bit codes travel as two E4M3 digit
+                               // planes (hi, lo); factors: int8 codes in L1q / L2q with block scales in s1b / s2b
   std::vector<uint8_t> Wq8h;   // mxfp: [K][N] e4m3 bytes of the e2m1 weight elements
   std::vector<uint8_t> L1e, L2e;   // mxfp: e4m3 bytes of the factor elements, [K][r] and [r][N]
   std::vector<float> s1b, s2b; // mxfp: block scales 2^e of L1 [ceil(K/32)][r] and of L2 [ceil(r/32)][N]
@@ -89,7 +103,8 @@ struct lq_layer {
 
 struct lq_act {
   int K, N, r, G, Kpad, Gpad, branch;
-  bool mx, mxfp;
+  bool mx, mxfp, a8;
+  int planes;                  // 1, or 2 (a8): digit planes of the main codes; qx8 rows are planes * Kpad bytes
   uint8_t* d_sft;              // mxfp: E8M0 bytes of the rank-r intermediate's block scales, [Mpad/128][1][512]
   uint8_t* d_sfa;              // MX: E8M0 bytes of the activation scales, [Mpad/128][Kpad/128][512], same layout
   int M_max, Mpad, device, main_kind;

@@ -39,8 +39,10 @@ constexpr int BOX_K = 64;              // values of K per box: one 128-byte swiz
 constexpr int BOX_BYTES = TR * BOX_K * 2;
 constexpr float MAGIC = 12582912.0f;   // 1.5 * 2^23: adding it rounds to an integer (ties to even)
 constexpr int MAX_CONSUMER_WARPS = 9;
-enum { BR_NONE = 0, BR_INT = 1, BR_F16 = 2, BR_MXFP = 3 };
-enum { MAIN_SINT4 = 0, MAIN_MXINT4 = 1, MAIN_MXFP = 2 };   // MXFP: MXFP8e4 activation codes for an MXFP4 weight
+enum { BR_NONE = 0, BR_INT = 1, BR_F16 = 2, BR_MXFP = 3, BR_MXINT = 4 };
+// MXFP: MXFP8e4 activation codes for an MXFP4 weight; MXINT8: MXINT8 activation codes for an MXINT4 weight, stored as
+// two E4M3 digit planes (code = 16 hi + lo)
+enum { MAIN_SINT4 = 0, MAIN_MXINT4 = 1, MAIN_MXFP = 2, MAIN_MXINT8 = 3 };
 
 struct QuantParams {
   int M, K, Kpad, Mpad;
@@ -49,9 +51,9 @@ struct QuantParams {
   int ntiles;           // ceil(M / 16)
   int depth;            // D: ring slots per consumer warp
   int refetch;          // 1: a warp's ring is smaller than its share of a tile, the producer streams every tile twice
-  uint8_t* qx8;         // [Mpad][Kpad]
+  uint8_t* qx8;         // [Mpad][Kpad] (MXINT8: [Mpad][2 Kpad], the hi digits' plane then the lo digits')
   float* sx;            // [Gpad][Mpad]
-  uint8_t* sfa;         // MXINT4: E8M0 scale bytes [Mpad/128][Kpad/128][512]
+  uint8_t* sfa;         // MXINT4: E8M0 scale bytes [Mpad/128][Kpad/128][512] (MXINT8: [Mpad/128][2 Kpad/128][512], by plane)
   int8_t* qb;           // [Mpad][Kpad] or null (not stored)
   float* sXb;           // [Mpad]
   const uint4* L1f;     // first factor in fragment order: [nbox][r tiles][32 lanes] x 16 bytes (int8) or 32 bytes (fp16)
@@ -137,6 +139,44 @@ __device__ __forceinline__ uint2 mxfp8_codes8(const uint4& v, int e) {
 }
 // 2^e as a float (0 for the all-zero block's -127: its codes are zeros anyway)
 __device__ __forceinline__ float pow2f(int e) { return e <= -127 ? 0.f : __uint_as_float((uint32_t)(e + 127) << 23); }
+
+// MXINT8 (Appendix A.3 "MX Formats": signed 8-bit codes, blocks of 32, power-of-two scale): the block's exponent is the
+// smallest e with 127 * 2^e >= a for the block maximum a = 1.f * 2^E: e = E - 6 if 1.f <= 127/64, else E - 5; at
+// least -127, and -127 for an all-zero block.
+__device__ __forceinline__ int mxint8_exponent(float a) {
+  const uint32_t ab = __float_as_uint(a);
+  const int e = (int)(ab >> 23) - 127 - (((ab & 0x7FFFFFu) <= 0x7E0000u) ? 6 : 5);
+  return a > 0.f ? max(e, -127) : -127;
+}
+// One value under the block's exponent: the code c = rint_even(x / 2^e) (the division is exact), as the int8 byte the
+// down-projection multiplies and as two digits c = 16 hi + lo, lo in [-8, 7], hi in [-8, 8], both exact E4M3 values.
+struct Code8 { float hi, lo; uint32_t byte; };
+__device__ __forceinline__ Code8 mxint8_code(float x, float inv) {
+  const float t = __fmaf_rn(x, inv, MAGIC);
+  const float c = __fadd_rn(t, -MAGIC);
+  Code8 r;
+  r.byte = __float_as_uint(t) & 0xFFu;                 // the low byte of (c + MAGIC)'s bit pattern is c
+  r.hi = floorf(__fmul_rn(__fadd_rn(c, 8.f), 0.0625f));
+  r.lo = __fmaf_rn(r.hi, -16.f, c);
+  return r;
+}
+// eight values of one block (one 16-byte vector of halves): the E4M3 bytes of the hi and lo digits and the int8 codes
+__device__ __forceinline__ void mxint8_codes8(const uint4& v, int e, uint2& hi, uint2& lo, uint2& s8) {
+  const __half2* h2 = reinterpret_cast<const __half2*>(&v);
+  const float inv = e == -127 ? 0.f : __uint_as_float((uint32_t)(127 - e) << 23);
+  Code8 c[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __half22float2(h2[i]);
+    c[2 * i] = mxint8_code(f.x, inv); c[2 * i + 1] = mxint8_code(f.y, inv);
+  }
+  hi.x = f32x2_to_e4m3x2(c[1].hi, c[0].hi) | (f32x2_to_e4m3x2(c[3].hi, c[2].hi) << 16);
+  hi.y = f32x2_to_e4m3x2(c[5].hi, c[4].hi) | (f32x2_to_e4m3x2(c[7].hi, c[6].hi) << 16);
+  lo.x = f32x2_to_e4m3x2(c[1].lo, c[0].lo) | (f32x2_to_e4m3x2(c[3].lo, c[2].lo) << 16);
+  lo.y = f32x2_to_e4m3x2(c[5].lo, c[4].lo) | (f32x2_to_e4m3x2(c[7].lo, c[6].lo) << 16);
+  s8.x = c[0].byte | (c[1].byte << 8) | (c[2].byte << 16) | (c[3].byte << 24);
+  s8.y = c[4].byte | (c[5].byte << 8) | (c[6].byte << 16) | (c[7].byte << 24);
+}
 
 // Correctly rounded quotient a / b in binary32 from the correctly rounded reciprocal y = fl32(1/b), division free:
 // q0 = fl32(a y) is within one ulp of a / b, r = a - b q0 is exact in an FMA, and fl32(q0 + r y) is then the
@@ -234,8 +274,9 @@ template <int MAIN, int BR, int NTR>   // NTR: 8-column tiles of the rank (rank 
 __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_kernel(const __grid_constant__ CUtensorMap tmX,
                                                                                  const QuantParams p) {
   constexpr bool MX = MAIN == MAIN_MXINT4;
-  constexpr bool FP = MAIN == MAIN_MXFP;
-  constexpr bool FACC = BR == BR_F16 || BR == BR_MXFP;     // fp32 partial sums of the down-projection
+  constexpr bool I8 = MAIN == MAIN_MXINT8;
+  constexpr bool FP = MAIN == MAIN_MXFP || I8;             // lanes hold eight values from each of a box's two blocks
+  constexpr bool FACC = BR == BR_F16 || BR == BR_MXFP || BR == BR_MXINT;     // fp32 partial sums of the down-projection
   extern __shared__ uint8_t qsm_raw[];
   const uint32_t base = (smem_u32(qsm_raw) + 1023u) & ~1023u;
   uint8_t* smem = qsm_raw + (base - smem_u32(qsm_raw));
@@ -402,6 +443,58 @@ __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_ker
             for (int o = 1; o <= 2; o <<= 1) {
               a00 = fmaxf(a00, __shfl_xor_sync(0xffffffffu, a00, o)); a01 = fmaxf(a01, __shfl_xor_sync(0xffffffffu, a01, o));
               a10 = fmaxf(a10, __shfl_xor_sync(0xffffffffu, a10, o)); a11 = fmaxf(a11, __shfl_xor_sync(0xffffffffu, a11, o));
+            }
+            if constexpr (I8) {
+              const int e00 = mxint8_exponent(a00), e01 = mxint8_exponent(a01), e10 = mxint8_exponent(a10), e11 = mxint8_exponent(a11);
+              uint2 h00, h01, h10, h11, d00, d01, d10, d11, s00, s01, s10, s11;   // hi digits, lo digits, int8 codes
+              mxint8_codes8(l0, e00, h00, d00, s00); mxint8_codes8(l1, e01, h01, d01, s01);
+              mxint8_codes8(h0, e10, h10, d10, s10); mxint8_codes8(h1, e11, h11, d11, s11);
+              const size_t xs = (size_t)2 * p.Kpad;                // bytes per row: the hi plane, then the lo plane
+              uint8_t* q_lo = p.qx8 + (size_t)m_lo * xs + koff + 8 * tig;
+              uint8_t* q_hi = q_lo + (size_t)8 * xs;
+              if (v_lo) {
+                *reinterpret_cast<uint2*>(q_lo) = h00; *reinterpret_cast<uint2*>(q_lo + 32) = h01;
+                *reinterpret_cast<uint2*>(q_lo + p.Kpad) = d00; *reinterpret_cast<uint2*>(q_lo + p.Kpad + 32) = d01;
+              }
+              if (v_hi) {
+                *reinterpret_cast<uint2*>(q_hi) = h10; *reinterpret_cast<uint2*>(q_hi + 32) = h11;
+                *reinterpret_cast<uint2*>(q_hi + p.Kpad) = d10; *reinterpret_cast<uint2*>(q_hi + p.Kpad + 32) = d11;
+              }
+              if (tig == 0) {
+                const int kb = 2 * g;                            // blocks kb, kb + 1 share a 4-block scale chunk
+                const size_t ks = (size_t)(p.Kpad >> 7);         // K stages per plane
+                if (kb < p.G) {
+                  if (v_lo) {
+                    uint8_t* sf = p.sfa + ((size_t)(m_lo >> 7) * 2 * ks + (kb >> 2)) * 512 + 16 * (m_lo & 31) + 4 * ((m_lo & 127) >> 5) + (kb & 3);
+                    sf[0] = (uint8_t)(e00 + 4 + 127); sf[ks * 512] = (uint8_t)(e00 + 127);
+                    if (kb + 1 < p.G) { sf[1] = (uint8_t)(e01 + 4 + 127); sf[ks * 512 + 1] = (uint8_t)(e01 + 127); }
+                  }
+                  if (v_hi) {
+                    uint8_t* sf = p.sfa + ((size_t)(m_hi >> 7) * 2 * ks + (kb >> 2)) * 512 + 16 * (m_hi & 31) + 4 * ((m_hi & 127) >> 5) + (kb & 3);
+                    sf[0] = (uint8_t)(e10 + 4 + 127); sf[ks * 512] = (uint8_t)(e10 + 127);
+                    if (kb + 1 < p.G) { sf[1] = (uint8_t)(e11 + 4 + 127); sf[ks * 512 + 1] = (uint8_t)(e11 + 127); }
+                  }
+                }
+              }
+              if constexpr (BR == BR_MXINT) {
+                // a3: per block of 32 one exact integer MMA step on the codes just made, then the block's two power-of-two
+                // scales in fp32 (|partial| <= 32 * 127 * 127 < 2^24: the conversion is exact)
+                const float sa00 = pow2f(e00), sa01 = pow2f(e01), sa10 = pow2f(e10), sa11 = pow2f(e11);
+#pragma unroll
+                for (int nt = 0; nt < NTR; ++nt) {
+                  const float2 sb0 = __ldg(reinterpret_cast<const float2*>(p.s1b + (size_t)(2 * g) * p.rpad + nt * 8 + 2 * tig));
+                  const float2 sb1 = __ldg(reinterpret_cast<const float2*>(p.s1b + (size_t)(2 * g + 1) * p.rpad + nt * 8 + 2 * tig));
+                  int i0[4] = {0, 0, 0, 0}, i1[4] = {0, 0, 0, 0};
+                  mma_s8_16832(i0, s00.x, s10.x, s00.y, s10.y, bfrag[nt].x, bfrag[nt].y);
+                  mma_s8_16832(i1, s01.x, s11.x, s01.y, s11.y, bfrag[nt].z, bfrag[nt].w);
+                  accf[nt][0] = fmaf(__int2float_rn(i0[0]), sa00 * sb0.x, fmaf(__int2float_rn(i1[0]), sa01 * sb1.x, accf[nt][0]));
+                  accf[nt][1] = fmaf(__int2float_rn(i0[1]), sa00 * sb0.y, fmaf(__int2float_rn(i1[1]), sa01 * sb1.y, accf[nt][1]));
+                  accf[nt][2] = fmaf(__int2float_rn(i0[2]), sa10 * sb0.x, fmaf(__int2float_rn(i1[2]), sa11 * sb1.x, accf[nt][2]));
+                  accf[nt][3] = fmaf(__int2float_rn(i0[3]), sa10 * sb0.y, fmaf(__int2float_rn(i1[3]), sa11 * sb1.y, accf[nt][3]));
+                }
+              }
+              if (g + W < p.nbox) load_frags(g + W);
+              continue;
             }
             const int e00 = mxfp8_exponent(a00), e01 = mxfp8_exponent(a01), e10 = mxfp8_exponent(a10), e11 = mxfp8_exponent(a11);
             const uint2 w00 = mxfp8_codes8(l0, e00), w01 = mxfp8_codes8(l1, e01);
@@ -581,6 +674,28 @@ __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_ker
               }
             }
           }
+        } else if constexpr (BR == BR_MXINT) {
+          // T in fp32 (the warps' partial sums added in warp order), then MXINT8 along the rank: one block of 32 per warp
+          // pass; the two digit planes of the codes share the row's container (hi at byte j, lo at byte 64 + j) and the
+          // scale chunk's four slots are (hi, block 0), (hi, block 1), (lo, block 0), (lo, block 1)
+          if (m < p.M) {
+            for (int c = 0; c * 32 < p.r; ++c) {
+              const int j = c * 32 + lane;
+              float v = 0.f;
+              if (j < p.rpad)
+                for (int w2 = 0; w2 < W; ++w2) v += part_s[((size_t)w2 * TR + rl) * p.rpad + j];
+              if (j >= p.r) v = 0.f;
+              const int e = mxint8_exponent(warp_max(fabsf(v)));
+              const float inv = e == -127 ? 0.f : __uint_as_float((uint32_t)(127 - e) << 23);
+              const Code8 cd = mxint8_code(v, inv);
+              p.tq[(size_t)m * LQ_RCONT + j] = (uint8_t)(f32x2_to_e4m3x2(0.f, cd.hi) & 0xFF);
+              p.tq[(size_t)m * LQ_RCONT + 64 + j] = (uint8_t)(f32x2_to_e4m3x2(0.f, cd.lo) & 0xFF);
+              if (lane == 0) {
+                uint8_t* sf = p.sft + (size_t)(m >> 7) * 512 + 16 * (m & 31) + 4 * ((m & 127) >> 5);
+                sf[c] = (uint8_t)(e + 4 + 127); sf[2 + c] = (uint8_t)(e + 127);
+              }
+            }
+          }
         } else if constexpr (BR == BR_MXFP) {
           // T = deq(Q(X)) deq(Q2(L1)) in fp32 (the warps' partial sums added in warp order), then MXFP8e4 along the rank:
           // one block of 32 per warp pass, its maximum by a warp reduction
@@ -637,7 +752,7 @@ LaunchPlan plan_launch(int nbox, int br, int rpad, int regs) {
       if (g_lq_quant_warps > 0 ? W != g_lq_quant_warps : W < 8) continue;
       const int threads = (W + 1) * 32;
       if (ctas * threads > 2048 || ctas * threads * ((regs + 7) / 8 * 8) > 65536) continue;
-      const size_t red = br == BR_INT ? (size_t)2 * TR * rpad * 4 : (br == BR_F16 || br == BR_MXFP) ? (size_t)W * TR * rpad * 4 : 0;
+      const size_t red = br == BR_INT ? (size_t)2 * TR * rpad * 4 : (br == BR_F16 || br == BR_MXFP || br == BR_MXINT) ? (size_t)W * TR * rpad * 4 : 0;
       const size_t fixed = 1024 + 64 + red + 2 * TR * 4 + 64;
       const size_t budget = std::min(SM_SMEM, SM_SMEM / ctas - 1024);
       if (budget < fixed + (size_t)W * (BOX_BYTES + 16)) continue;
@@ -684,7 +799,11 @@ cudaError_t launch_quant(const CUtensorMap& tm, QuantParams& p, int sms, cudaStr
 template <int MAIN>
 cudaError_t dispatch_quant(int br, int ntr, const CUtensorMap& tm, QuantParams& p, int sms, cudaStream_t st) {
   if (br == BR_NONE) return launch_quant<MAIN, BR_NONE, 1>(tm, p, sms, st);
-  if constexpr (MAIN == MAIN_MXFP) {
+  if constexpr (MAIN == MAIN_MXINT8) {
+    if (ntr <= 2) return launch_quant<MAIN, BR_MXINT, 2>(tm, p, sms, st);
+    if (ntr <= 4) return launch_quant<MAIN, BR_MXINT, 4>(tm, p, sms, st);
+    return launch_quant<MAIN, BR_MXINT, 8>(tm, p, sms, st);
+  } else if constexpr (MAIN == MAIN_MXFP) {
     if (ntr <= 2) return launch_quant<MAIN, BR_MXFP, 2>(tm, p, sms, st);
     if (ntr <= 4) return launch_quant<MAIN, BR_MXFP, 4>(tm, p, sms, st);
     if (ntr <= 8) return launch_quant<MAIN, BR_MXFP, 8>(tm, p, sms, st);
@@ -714,7 +833,7 @@ lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A,
   if (cudaSetDevice(A->device) != cudaSuccess) return LQ_ERR_CUDA;
   if (A->main_kind != LQ_KIND_E4M3) return LQ_ERR_UNSUPPORTED;
   const int abits = lq_branch_abits(L->cfg.branch);
-  const int br = L->mxfp ? (L->r > 0 ? BR_MXFP : BR_NONE) : L->f16_branch ? BR_F16 : (L->integer_branch && abits > 0) ? BR_INT : BR_NONE;
+  const int br = L->mxfp ? (L->r > 0 ? BR_MXFP : BR_NONE) : L->a8 ? (L->r > 0 ? BR_MXINT : BR_NONE) : L->f16_branch ? BR_F16 : (L->integer_branch && abits > 0) ? BR_INT : BR_NONE;
   const int ntr = lq_quant_rank_tiles(L->r, L->f16_branch);
   QuantParams p;
   p.M = M; p.K = L->K; p.Kpad = L->Kpad; p.Mpad = A->Mpad; p.G = L->G;
@@ -736,6 +855,7 @@ lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A,
   int sms = 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, A->device) != cudaSuccess) return LQ_ERR_CUDA;
   const cudaError_t e = L->mxfp ? dispatch_quant<MAIN_MXFP>(br, ntr, tm, p, sms, st)
+                        : L->a8 ? dispatch_quant<MAIN_MXINT8>(br, ntr, tm, p, sms, st)
                         : L->mx ? dispatch_quant<MAIN_MXINT4>(br, ntr, tm, p, sms, st) : dispatch_quant<MAIN_SINT4>(br, ntr, tm, p, sms, st);
   return lq_note_cuda(e) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
 }

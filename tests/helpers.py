@@ -41,6 +41,24 @@ def import_oracle_mxfp_layer(layer: dict):
     return h, cfg
 
 
+def import_oracle_mxint_layer(layer: dict):
+    """A layer of oracle/lq_oracle_mxint.py (MXINT4 weights, MXINT8 activations, MX integer factors) -> library handle."""
+    K, N, r = layer["K"], layer["N"], layer["rank"]
+    branch = layer["branch"] if r > 0 else "none"
+    cfg = B.lq_config_default(K, N, r, branch)
+    cfg.group, cfg.main_fmt = 32, B.MAIN_MXINT4_A8
+    live = lambda e: np.where(e == -127, 0, e).astype(np.float64)       # an all-zero block: any scale does, its codes are zeros
+    sw = np.exp2(live(layer["ew"])).astype(np.float16)
+    if r > 0:
+        L1, L2 = layer["L1q"].astype(np.int8), layer["L2q"].astype(np.int8)
+        s1 = np.exp2(live(layer["e1"])).astype(np.float32)
+        s2 = np.exp2(live(layer["e2"])).astype(np.float32)
+    else:
+        L1 = L2 = s1 = s2 = None
+    h = B.lq_layer_import(cfg, B.pack_nibbles(layer["Wq"].astype(np.int8)), sw, L1, s1, L2, s2, layer.get("bias"))
+    return h, cfg
+
+
 def gpu_forward(layer: dict, X16: np.ndarray, out_f32: bool = True, export: bool = True, device: int = 0,
                 store_qb: bool = True):
     """Runs lq_quantize_act + lq_linear_forward through the C ABI; returns (Y, exported act dict).
@@ -48,7 +66,8 @@ def gpu_forward(layer: dict, X16: np.ndarray, out_f32: bool = True, export: bool
     (the benchmark configuration leaves them on chip)."""
     import torch
     B.lq_set_option("store_qb", 1 if store_qb else 0)
-    h, cfg = import_oracle_mxfp_layer(layer) if layer.get("main") == "mxfp4" else import_oracle_layer(layer)
+    h, cfg = (import_oracle_mxfp_layer(layer) if layer.get("main") == "mxfp4" else
+              import_oracle_mxint_layer(layer) if layer.get("main") == "mxint4a8" else import_oracle_layer(layer))
     B.lq_layer_to_device(h, device)
     M = X16.shape[0]
     act = B.lq_act_create(h, M, device)

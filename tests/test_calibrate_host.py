@@ -1,6 +1,7 @@
 """lq_calibrate (host-side C++ in the library) checked on the CPU against closed forms and
 against the oracle's statement of the same procedure."""
 import numpy as np
+import pytest
 
 from oracle import lq_oracle as O
 from paper_2604_18117_b200 import binding as B
@@ -223,3 +224,42 @@ def test_mxfp_calibration_follows_the_oracle():
     layer = _export_mxfp_as_oracle_layer(h)
     assert np.array_equal(F.deq_columns(layer["Wv"], layer["ew"]), F.q1_dequant(W.astype(np.float64)))
     B.lq_layer_free(h)
+
+
+def test_mxint8_activation_layers_calibration_follows_the_oracle():
+    """lq_calibrate for MXINT4 weights with MXINT8 activations and an MXINT8 / MXINT4 branch (Table 3's integer rows):
+    the first Adam steps follow the oracle's objective trace, the stored factors are within their format's range and
+    on its grid, and the stored residual is Q1 of W - Q2(L1) Q2(L2)."""
+    from oracle import lq_oracle_mxint as OI
+    rng = np.random.default_rng(13)
+    K, N, r = 96, 32, 3
+    U, _ = np.linalg.qr(rng.standard_normal((K, N)))
+    V, _ = np.linalg.qr(rng.standard_normal((N, N)))
+    sig = np.concatenate([[0.9, 0.6, 0.35], np.linspace(0.05, 0.01, N - 3)])
+    W = ((U * sig[None, :]) @ V.T).astype(np.float16)
+    for branch in ("mxint8", "mxint4"):
+        cfg = B.lq_config_default(K, N, r, branch)
+        assert cfg.main_fmt == B.MAIN_MXINT4_A8 and cfg.group == 32 and abs(cfg.lr - 1e-4) < 1e-9   # integer formats: 1e-4
+        cfg.steps = 2
+        h, trace = B.lq_calibrate(cfg, W, want_trace=True)
+        _, tr_o = OI.calibrate(W, r, branch, steps=2)
+        assert np.allclose(trace, tr_o, rtol=1e-7, atol=0), (branch, trace, tr_o)
+        ex = B.lq_layer_export(h)
+        qm = 127 if branch == "mxint8" else 7
+        assert np.abs(ex["L1"]).max() <= qm and np.abs(ex["L2"]).max() <= qm
+        assert np.abs(ex["L1"]).max() > qm // 2                                  # the range is used: minimal exponents
+        e1 = np.log2(ex["sL1"].astype(np.float64)).astype(np.int16)
+        e2 = np.log2(ex["sL2"].astype(np.float64)).astype(np.int16)
+        L1d, L2d = OI.deq_columns(ex["L1"], e1), OI.deq_columns(ex["L2"], e2)
+        # idempotence pins the stored pair (codes, exponent): re-quantizing the dequantized factors changes nothing
+        assert np.array_equal(OI.deq_columns(*OI.q_columns(L1d, OI.FACTOR_BITS[branch])), L1d)
+        Wq = B.unpack_nibbles(ex["Wq_packed"])
+        ew = np.log2(ex["sw"].astype(np.float64)).astype(np.int16)
+        q, e = OI.q_columns(W.astype(np.float64) - L1d @ L2d, 4)
+        assert np.array_equal(OI.deq_columns(q, e), OI.deq_columns(Wq, ew))
+        B.lq_layer_free(h)
+    # unsupported combinations are refused before any work
+    cfg = B.lq_config_default(K, N, 96, "mxint8")
+    cfg.steps = 0
+    with pytest.raises(B.LqError):
+        B.lq_calibrate(cfg, W)
