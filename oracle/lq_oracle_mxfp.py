@@ -11,6 +11,9 @@ What it follows
 * Mixed-precision study (Section 4.3, Tables 3 and 4; Appendix A.2 "Quantization"): residual weights fixed to a
   4-bit MX format (MXFP4e2 here), activations forwarded to BOTH branches in one 8-bit MX format (MXFP8e4), low-rank
   factors in MXFP8e4 / MXFP6e2 / MXFP4e2 with rank 64 / 86 / 128 at equal memory.
+* Rank study (Section 4.3, Table 4): activations and low-rank factors share ONE sub-16-bit format, MXFP8e4 or MXFP6e2;
+  a layer's "act" entry names the activations' element format ("e4m3" when absent, "e2m3" for the MXFP6e2 rows) and
+  applies to X and to the re-quantized intermediate alike.
 * Decomposed forward and calibration: as in lq_oracle.py (Figure 1, Sections 3.2-3.3, Appendix B.2), with
   Q1 = MXFP4e2 along K per output column and Q2 = the branch format along each factor's contraction axis
   (L1 along K per column, L2 along r per column); learning rate 1e-3 for FP formats (Appendix A.2 "Optimization").
@@ -104,6 +107,7 @@ def forward(X16, layer):
     """Reference forward of one MXFP layer.
     layer: Wv float32 [K, N] (e2m1 element values), ew int16 [ceil(K/32), N]; branch "mxfp8" | "mxfp6" | "mxfp4" |
     "none"; rank; L1v [K, r], e1 [ceil(K/32), r]; L2v [r, N], e2 [ceil(r/32), N]; optional bias fp16 [N].
+    layer["act"] (optional): element format of the activations, "e4m3" (default) or "e2m3"; written MXFP8e4 below.
     Steps: (1) xa, ex = MXFP8e4 of X rows, shared by both branches; (2) main: sum over K blocks of
     2^(ex + ew) (xa_b Wv_b), exact element products; (3) T = sum over K blocks of 2^(ex + e1) (xa_b L1v_b);
     (4) tq, et = MXFP8e4 of T rows along r; (5) Y += sum over r blocks of 2^(et + e2) (tq_c L2v_c) (+ bias), float64."""
@@ -111,7 +115,8 @@ def forward(X16, layer):
     M, K = X.shape
     Wv, ew = layer["Wv"].astype(np.float64), layer["ew"]
     N = Wv.shape[1]
-    xa, ex = qmxfp(X, "e4m3")
+    act = layer.get("act", "e4m3")
+    xa, ex = qmxfp(X, act)
     out = {"xa": xa, "ex": ex}
     xa64 = xa.astype(np.float64)
     Y = np.zeros((M, N))
@@ -126,7 +131,7 @@ def forward(X16, layer):
         if has_branch:
             T += sa * np.exp2(layer["e1"][b, :].astype(np.float64))[None, :] * (xa64[:, k0:k1] @ layer["L1v"][k0:k1, :].astype(np.float64))
     if has_branch:
-        tq, et = qmxfp(T, "e4m3")
+        tq, et = qmxfp(T, act)
         out.update(T=T, tq=tq, et=et)
         tq64 = tq.astype(np.float64)
         for c in range(-(-r // MX_BLOCK)):

@@ -124,15 +124,24 @@ def _tiny_layer(rng, K, N, r, branch):
     return layer
 
 
-@pytest.mark.parametrize("branch,r", [("mxfp8", 5), ("mxfp6", 40), ("mxfp4", 33), ("none", 0)])
-def test_forward_against_python_scalars(branch, r):
+@pytest.mark.parametrize("branch,r,act", [("mxfp8", 5, "e4m3"), ("mxfp6", 40, "e4m3"), ("mxfp4", 33, "e4m3"), ("none", 0, "e4m3"),
+                                          ("mxfp6", 40, "e2m3"), ("none", 0, "e2m3")])
+def test_forward_against_python_scalars(branch, r, act):
     """Tiny ragged shapes (K = 72: two full blocks and a short one), every sum in exact rational arithmetic from the
     oracle's own element values and exponents of X and T (their quantizer is pinned above)."""
     rng = np.random.default_rng(3)
     M, K, N = 3, 72, 4
     layer = _tiny_layer(rng, K, N, r, branch)
+    if act != "e4m3":
+        layer["act"] = act                      # Table 4: activations in the branch's 6-bit format
     X = (rng.standard_normal((M, K)) * 2).astype(np.float16)
     out = F.forward(X, layer)
+    # the activations' images are the pinned quantizer's, in the format asked for (the 6-bit grid is coarser: it must show)
+    xa_ref, ex_ref = F.qmxfp(X.astype(np.float64), act)
+    assert np.array_equal(out["xa"], xa_ref) and np.array_equal(out["ex"], ex_ref)
+    assert np.isin(np.abs(out["xa"]), F.element_values(act).astype(np.float32)).all()
+    if act == "e2m3":
+        assert not np.array_equal(F.deq_mxfp(out["xa"], out["ex"]), F.deq_mxfp(*F.qmxfp(X.astype(np.float64), "e4m3")))
     fr = lambda x: Fraction(float(x))
     p2 = lambda e: Fraction(2) ** int(e)
     for m in range(M):
@@ -148,7 +157,7 @@ def test_forward_against_python_scalars(branch, r):
             y += fr(layer["bias"][n])
             assert abs(Fraction(float(out["Y"][m, n])) - y) <= abs(y) * Fraction(1, 10 ** 12) + Fraction(1, 10 ** 14)
     if r:
-        tq2, et2 = F.qmxfp(out["T"], "e4m3")
+        tq2, et2 = F.qmxfp(out["T"], act)
         assert np.array_equal(tq2, out["tq"]) and np.array_equal(et2, out["et"])
 
 
