@@ -74,6 +74,14 @@ typedef enum {
                           with block scales 2^(e+4) and 2^e, so the tensor core applies every scale here too    */
 } lq_main_fmt;
 
+/* Element format of the activations (X for both branches, and the rank-r intermediate) of an MXFP layer.  The rank
+ * study of Section 4.3 (Table 4) gives activations and factors ONE sub-16-bit format: MXFP8e4, or MXFP6e2. */
+typedef enum {
+  LQ_ACT_DEFAULT = 0,  /* SINT4 / MXINT4 main formats: their own 4-bit activations; MXFP4: MXFP8e4; MXINT4_A8: MXINT8 */
+  LQ_ACT_MXFP6 = 6     /* MXFP6e2 activations; only with main_fmt = LQ_MAIN_MXFP4 (the weights' kernels do not change:
+                          every e2m3 value is an e4m3 value)                                                     */
+} lq_act_fmt;
+
 typedef enum { LQ_OUT_F16 = 0, LQ_OUT_F32 = 1 } lq_out_dtype;
 
 /* One layer's shape and calibration settings. */
@@ -89,7 +97,7 @@ typedef struct {
   float rot_lr;       /* 500 steps at 0.5 (0.1 for the mixed-precision study) in Appendix A           */
   uint64_t seed;      /* start vectors of the host SVD iteration                                  */
   int32_t main_fmt;   /* an lq_main_fmt; 0 (default) = SINT4 / MXINT4 as `group` says                */
-  int32_t reserved;   /* 0                                                                          */
+  int32_t act_fmt;    /* an lq_act_fmt; 0 (default) = the main format's own activations                 */
 } lq_config;
 
 typedef struct lq_layer lq_layer; /* opaque: Q1(P) codes+scales, Q2(L1), Q2(L2), bias (Figure 1)  */

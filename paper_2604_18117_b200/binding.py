@@ -18,6 +18,7 @@ LQ_OK = 0
 BRANCH = {"none": 0, "w16a16": 1, "w8a8": 2, "w6a6": 3, "w4a8": 4, "mxfp8": 5, "mxfp6": 6, "mxfp4": 7,
           "mxint8": 8, "mxint4": 9}
 MAIN_AUTO, MAIN_MXFP4, MAIN_MXINT4_A8 = 0, 2, 3
+ACT_DEFAULT, ACT_MXFP6 = 0, 6
 BRANCH_NAME = {v: k for k, v in BRANCH.items()}
 OUT_F16, OUT_F32 = 0, 1
 GROUP = 64
@@ -27,7 +28,7 @@ class LqConfig(C.Structure):
     _fields_ = [("K", C.c_int32), ("N", C.c_int32), ("rank", C.c_int32), ("group", C.c_int32),
                 ("branch", C.c_int32), ("steps", C.c_int32), ("lr", C.c_float), ("beta1", C.c_float),
                 ("beta2", C.c_float), ("eps", C.c_float), ("rot_steps", C.c_int32), ("rot_lr", C.c_float),
-                ("seed", C.c_uint64), ("main_fmt", C.c_int32), ("reserved", C.c_int32)]
+                ("seed", C.c_uint64), ("main_fmt", C.c_int32), ("act_fmt", C.c_int32)]
 
 
 class LqError(RuntimeError):

@@ -83,7 +83,7 @@ extern "C" lq_status lq_config_default(lq_config* cfg, int32_t K, int32_t N, int
   cfg->K = K; cfg->N = N; cfg->rank = rank; cfg->group = LQ_GROUP; cfg->branch = branch;
   cfg->steps = 1000; cfg->lr = 1e-4f; cfg->beta1 = 0.9f; cfg->beta2 = 0.999f; cfg->eps = 1e-8f;
   cfg->rot_steps = 0; cfg->rot_lr = 0.5f; cfg->seed = 0;
-  cfg->main_fmt = LQ_MAIN_AUTO; cfg->reserved = 0;
+  cfg->main_fmt = LQ_MAIN_AUTO; cfg->act_fmt = LQ_ACT_DEFAULT;
   if (lq_branch_is_mxfp(branch)) { cfg->main_fmt = LQ_MAIN_MXFP4; cfg->group = LQ_MX_BLOCK; cfg->lr = 1e-3f; }
   if (lq_branch_is_mxint(branch)) { cfg->main_fmt = LQ_MAIN_MXINT4_A8; cfg->group = LQ_MX_BLOCK; }
   return LQ_OK;
@@ -99,6 +99,7 @@ static lq_status check_config(const lq_config* c) {
   if (c->main_fmt == LQ_MAIN_MXFP4 && (c->group != LQ_MX_BLOCK || !(c->branch == LQ_BRANCH_NONE || lq_branch_is_mxfp(c->branch))))
     return LQ_ERR_UNSUPPORTED;
   if (c->main_fmt != LQ_MAIN_MXFP4 && lq_branch_is_mxfp(c->branch)) return LQ_ERR_UNSUPPORTED;
+  if (c->act_fmt != LQ_ACT_DEFAULT && !(c->act_fmt == LQ_ACT_MXFP6 && c->main_fmt == LQ_MAIN_MXFP4)) return LQ_ERR_UNSUPPORTED;
   // MXINT8 activations go with MXINT4 weights in blocks of 32 and an integer MX (or no) branch of rank <= 64 (the two
   // digit planes of the rank-r intermediate share the 128-byte container)
   if (c->main_fmt == LQ_MAIN_MXINT4_A8 &&

@@ -525,6 +525,7 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
   if (cfg->branch < LQ_BRANCH_NONE || cfg->branch > LQ_BRANCH_MXINT4) return LQ_ERR_INVALID_ARG;
   const bool mxfp = cfg->main_fmt == LQ_MAIN_MXFP4;
   const bool a8 = cfg->main_fmt == LQ_MAIN_MXINT4_A8;
+  if (cfg->act_fmt != LQ_ACT_DEFAULT && !(cfg->act_fmt == LQ_ACT_MXFP6 && mxfp)) return LQ_ERR_UNSUPPORTED;
   if (a8 ? !(cfg->branch == LQ_BRANCH_NONE || lq_branch_is_mxint(cfg->branch)) : lq_branch_is_mxint(cfg->branch)) return LQ_ERR_UNSUPPORTED;
   if (a8 && (cfg->group != LQ_MX_BLOCK || cfg->rot_steps > 0 || (cfg->branch != LQ_BRANCH_NONE && cfg->rank > 64))) return LQ_ERR_UNSUPPORTED;
   if (mxfp ? !(cfg->branch == LQ_BRANCH_NONE || lq_branch_is_mxfp(cfg->branch)) : lq_branch_is_mxfp(cfg->branch)) return LQ_ERR_UNSUPPORTED;

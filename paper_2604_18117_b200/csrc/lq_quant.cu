@@ -63,6 +63,7 @@ struct QuantParams {
   uint8_t* tq;          // [Mpad][LQ_RCONT]
   float* sT;            // [Mpad]
   int r, rpad;          // rank, rank rounded up to 8
+  int act6;             // MXFP: the activations (X and the rank-r intermediate) are MXFP6e2 instead of MXFP8e4
   float qm;             // largest branch activation code
   int32_t* status;
 };
@@ -115,15 +116,28 @@ __device__ __forceinline__ __half absmax8(const uint4& a) {
   return __hmax(__low2half(m), __high2half(m));
 }
 
-// MXFP8e4 of eight values that share a block (Appendix A.3 "MX Formats"; conversion of the OCP specification the
-// paper cites): the block's exponent is e = floor(log2 a) - 8 for the block maximum a (e4m3's largest binade is 2^8),
-// -127 for an all-zero block; the elements are x / 2^e - exact - rounded to e4m3 by the hardware conversion
-// (nearest even, magnitudes above 448 clamped).  Returns the eight e4m3 bytes.
-__device__ __forceinline__ int mxfp8_exponent(float a) {
-  const int e = (int)(__float_as_uint(a) >> 23) - 127 - 8;
+// MXFP8e4 / MXFP6e2 of eight values that share a block (Appendix A.3 "MX Formats"; conversion of the OCP specification
+// the paper cites): the block's exponent is e = floor(log2 a) - emax for the block maximum a (emax = 8: e4m3's largest
+// binade, 2: e2m3's), -127 for an all-zero block; the elements are x / 2^e - exact - rounded to the element format by
+// the hardware conversion (nearest even, magnitudes above the largest normal clamped).  Every e2m3 value is an e4m3
+// value, so both formats are stored, and multiplied, as e4m3 bytes: the 6-bit path rounds to e2m3 first and widens
+// the result (e2m3 -> f16 -> e4m3, both exact).
+__device__ __forceinline__ int mxfp8_exponent(float a, bool six = false) {
+  const int e = (int)(__float_as_uint(a) >> 23) - 127 - (six ? 2 : 8);
   return (a > 0.f && e >= -126) ? e : -127;
 }
-__device__ __forceinline__ uint2 mxfp8_codes8(const uint4& v, int e) {
+__device__ __forceinline__ uint32_t f32x2_to_e4m3x2_via_e2m3(float hi, float lo) {
+  uint16_t r6, r8;
+  uint32_t h2;
+  asm("cvt.rn.satfinite.e2m3x2.f32 %0, %1, %2;" : "=h"(r6) : "f"(hi), "f"(lo));
+  asm("cvt.rn.f16x2.e2m3x2 %0, %1;" : "=r"(h2) : "h"(r6));
+  asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(r8) : "r"(h2));
+  return (uint32_t)r8;
+}
+__device__ __forceinline__ uint32_t mxfp_pair(float hi, float lo, bool six) {
+  return six ? f32x2_to_e4m3x2_via_e2m3(hi, lo) : f32x2_to_e4m3x2(hi, lo);
+}
+__device__ __forceinline__ uint2 mxfp8_codes8(const uint4& v, int e, bool six = false) {
   const __half2* h2 = reinterpret_cast<const __half2*>(&v);
   const float inv = e == -127 ? 0.f : __uint_as_float((uint32_t)(127 - e) << 23);
   float x[8];
@@ -133,8 +147,8 @@ __device__ __forceinline__ uint2 mxfp8_codes8(const uint4& v, int e) {
     x[2 * i] = f.x * inv; x[2 * i + 1] = f.y * inv;
   }
   uint2 w;
-  w.x = f32x2_to_e4m3x2(x[1], x[0]) | (f32x2_to_e4m3x2(x[3], x[2]) << 16);
-  w.y = f32x2_to_e4m3x2(x[5], x[4]) | (f32x2_to_e4m3x2(x[7], x[6]) << 16);
+  w.x = mxfp_pair(x[1], x[0], six) | (mxfp_pair(x[3], x[2], six) << 16);
+  w.y = mxfp_pair(x[5], x[4], six) | (mxfp_pair(x[7], x[6], six) << 16);
   return w;
 }
 // 2^e as a float (0 for the all-zero block's -127: its codes are zeros anyway)
@@ -496,9 +510,10 @@ __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_ker
               if (g + W < p.nbox) load_frags(g + W);
               continue;
             }
-            const int e00 = mxfp8_exponent(a00), e01 = mxfp8_exponent(a01), e10 = mxfp8_exponent(a10), e11 = mxfp8_exponent(a11);
-            const uint2 w00 = mxfp8_codes8(l0, e00), w01 = mxfp8_codes8(l1, e01);
-            const uint2 w10 = mxfp8_codes8(h0, e10), w11 = mxfp8_codes8(h1, e11);
+            const bool six = p.act6 != 0;
+            const int e00 = mxfp8_exponent(a00, six), e01 = mxfp8_exponent(a01, six), e10 = mxfp8_exponent(a10, six), e11 = mxfp8_exponent(a11, six);
+            const uint2 w00 = mxfp8_codes8(l0, e00, six), w01 = mxfp8_codes8(l1, e01, six);
+            const uint2 w10 = mxfp8_codes8(h0, e10, six), w11 = mxfp8_codes8(h1, e11, six);
             uint8_t* q_lo = p.qx8 + (size_t)m_lo * p.Kpad + koff + 8 * tig;
             uint8_t* q_hi = q_lo + (size_t)8 * p.Kpad;
             if (v_lo) { *reinterpret_cast<uint2*>(q_lo) = w00; *reinterpret_cast<uint2*>(q_lo + 32) = w01; }
@@ -706,9 +721,9 @@ __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_ker
               if (j < p.rpad)
                 for (int w2 = 0; w2 < W; ++w2) v += part_s[((size_t)w2 * TR + rl) * p.rpad + j];
               if (j >= p.r) v = 0.f;
-              const int e = mxfp8_exponent(warp_max(fabsf(v)));
+              const int e = mxfp8_exponent(warp_max(fabsf(v)), p.act6 != 0);
               const float inv = e == -127 ? 0.f : __uint_as_float((uint32_t)(127 - e) << 23);
-              p.tq[(size_t)m * LQ_RCONT + j] = (uint8_t)(f32x2_to_e4m3x2(0.f, v * inv) & 0xFF);
+              p.tq[(size_t)m * LQ_RCONT + j] = (uint8_t)(mxfp_pair(0.f, v * inv, p.act6 != 0) & 0xFF);
               if (lane == 0) p.sft[(size_t)(m >> 7) * 512 + 16 * (m & 31) + 4 * ((m & 127) >> 5) + c] = (uint8_t)(e + 127);
             }
           }
@@ -846,6 +861,7 @@ lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A,
   p.sL1 = L->d_sL1; p.tq = A->d_tq; p.sT = A->d_sT;
   p.s1b = L->d_s1b; p.sft = A->d_sft;
   p.r = L->r; p.rpad = ntr * 8;
+  p.act6 = (L->mxfp && L->cfg.act_fmt == LQ_ACT_MXFP6) ? 1 : 0;
   p.qm = br == BR_INT ? (float)((1 << (abits - 1)) - 1) : 0.f;
   p.status = lq_device_status_ptr(A->device);
   if (!p.status) return LQ_ERR_CUDA;

@@ -29,6 +29,8 @@ def import_oracle_mxfp_layer(layer: dict):
     branch = layer["branch"] if r > 0 else "none"
     cfg = B.lq_config_default(K, N, r, branch)
     cfg.group, cfg.main_fmt = 32, B.MAIN_MXFP4
+    if layer.get("act", "e4m3") == "e2m3":
+        cfg.act_fmt = B.ACT_MXFP6                                         # Table 4: activations in the 6-bit format too
     live = lambda e: np.where(e == -127, 0, e).astype(np.float64)       # an all-zero block: any scale does, its elements are zeros
     sw = np.exp2(live(layer["ew"])).astype(np.float16)
     if r > 0:

@@ -100,3 +100,19 @@ def test_mxfp_degenerate_inputs():
     X[4, ::2] = np.float16(-65504)
     X[5] = (rng.integers(-8, 9, K) * 2.0 ** -20).astype(np.float16)
     _check(_layer(rng, K, N, r, "mxfp8"), X)
+
+
+@pytest.mark.parametrize("branch,r", [("mxfp6", 64), ("mxfp6", 128), ("none", 0)])
+def test_mxfp6_activations_table_4_rows(branch, r):
+    """The rank study's unified 6-bit rows (Table 4): MXFP6e2 activations - X for both branches and the rank-r
+    intermediate - with MXFP6e2 factors; the activation elements must lie on the e2m3 grid and match the oracle bit for
+    bit, the rest as for 8-bit activations."""
+    rng = np.random.default_rng(40 + r)
+    M, K, N = 300, 1152, 384
+    X = (rng.standard_normal((M, K))).astype(np.float16)
+    X[:, rng.choice(K, 8, replace=False)] *= 20
+    X[5, :64] = 0
+    X[6, :32] = [7.5, 7.75, 8.0, 0.0625, 0.1875, -0.3125] + [0.0] * 26       # the clamp, a binade change, subnormal ties
+    layer = _layer(rng, K, N, r, branch)
+    layer["act"] = "e2m3"
+    _check(layer, X)
