@@ -263,3 +263,19 @@ def test_mxint8_activation_layers_calibration_follows_the_oracle():
     cfg.steps = 0
     with pytest.raises(B.LqError):
         B.lq_calibrate(cfg, W)
+
+
+def test_activation_format_option_is_checked():
+    """MXFP6e2 activations (Table 4's 6-bit rows) exist for MXFP layers only; anything else is refused up front."""
+    rng = np.random.default_rng(1)
+    W = (rng.standard_normal((64, 32)) * 0.02).astype(np.float16)
+    cfg = B.lq_config_default(64, 32, 4, "mxfp6")
+    cfg.steps, cfg.act_fmt = 1, B.ACT_MXFP6
+    h, _ = B.lq_calibrate(cfg, W)
+    assert B.lq_layer_info(h).act_fmt == B.ACT_MXFP6
+    B.lq_layer_free(h)
+    for branch in ("w8a8", "mxint8"):
+        cfg = B.lq_config_default(64, 32, 4, branch)
+        cfg.steps, cfg.act_fmt = 1, B.ACT_MXFP6
+        with pytest.raises(B.LqError):
+            B.lq_calibrate(cfg, W)
