@@ -284,8 +284,11 @@ __device__ __forceinline__ bool consumers_sync(uint32_t bar, uint32_t parity, in
 //   red       BR_INT: int I1[2][16][rpad]; BR_F16: float part[W][16][rpad]
 //   rowmax    int[2][16] (bit patterns of non-negative floats)
 //   abort     int
+// Instances for rank > 32 (NTR >= 8) hold 32 or more accumulator and as many fragment registers per thread: compiled
+// for two CTAs per SM (96 registers) they spill, so they are compiled for one (measured: rank 64 10-33 % faster,
+// rank 128 10-20 %); the launch planner picks the residency from the register count it reads back.
 template <int MAIN, int BR, int NTR>   // NTR: 8-column tiles of the rank (rank <= 8 NTR)
-__global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, 2) lq_quant_kernel(const __grid_constant__ CUtensorMap tmX,
+__global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, NTR >= 8 ? 1 : 2) lq_quant_kernel(const __grid_constant__ CUtensorMap tmX,
                                                                                  const QuantParams p) {
   constexpr bool MX = MAIN == MAIN_MXINT4;
   constexpr bool I8 = MAIN == MAIN_MXINT8;
