@@ -103,7 +103,7 @@ __device__ __forceinline__ bool elect_one() {
   return pred != 0;
 }
 
-// ---- bulk copies (TMA), never with cluster multicast --------------------------------------
+// ---- bulk copies (TMA): every copy goes to the issuing CTA only -----------------------------
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),

@@ -72,7 +72,6 @@ constexpr int TM_BR = 256, TM_SFA = 256, TM_SFB = TM_SFA + 4, TM_SF_ALIASED = 16
 struct MxParams {
   int M, N, Mpad, Npad;
   int k_stages;           // stages of A per tile: Kpad / 128, times two when 8-bit activation codes come as two digit planes
-  int b_wrap;             // Kpad / 128: stage s reads B (and its scales) at stage s mod b_wrap - the planes share the weights
   int branch_steps;       // 0: no branch; else MMAs of the branch stage (32 bytes of r each)
   int branch_f16;         // the branch operands are halves (W16A16 reference branch): no scales, summed by the tensor core
   int branch_mx;          // the branch is MX as well: its up-projection is one more block-scaled stage onto the main
@@ -83,6 +82,10 @@ struct MxParams {
   const uint8_t* sfl2;    // branch_mx: E8M0 bytes of L2's block scales, [Npad/128][512]
   int tiles_m, units_n;
   int by_units;           // how the CTAs share the work: 0 whole tiles, 1 128-column units
+  int b_wrap;             // Kpad / 128: stage s reads B (and its scales) at stage s mod b_wrap - the planes share the weights
+                          // (kept in what was the padding before the next pointer: this kernel sits at its register
+                          // cap, and moving its other parameters changed the allocation ptxas found - 50 % more spill
+                          // traffic and 15 % longer launches)
   const uint8_t* sfa;     // [Mpad/128][k_stages][512]
   const uint8_t* sfb;     // [k_stages][Npad/128][512]: the scale bytes of two neighbouring 128-column units are contiguous
   const float* sT;        // [Mpad]
@@ -190,7 +193,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    uint32_t it = 0, tc = 0;
+    uint32_t it = 0, tc = 0, rarmed = 0;
     bool ok = true;
     for (int w = w_begin, w_next; w < w_end && ok; w = w_next, ++tc) {
       int mb, nu, width;
@@ -210,6 +213,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           bulk_load(dst + (LQ_BM + 2 * UNIT) * 4, p.bias + n0, width * UNIT * 4, rfull);
         }
         __syncwarp();
+        ++rarmed;
       }
       for (int s = 0; s < p.k_stages && ok; ++s, ++it) {
         const int st = it % NSTAGE;
@@ -251,9 +255,18 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         ++it;
       }
     }
-    if (!ok) {   // let copies in flight land before the CTA's shared memory goes away
-      const long long t0 = clock64();
-      while (clock64() - t0 < 2000000ll) { }
+    if (!ok && lane == 0) {
+      // aborting: give the copies already issued a bounded time to land before the CTA's shared memory goes away
+      // (`it` stages have been armed; the last NSTAGE of them may still be in flight)
+      const uint32_t n = it < (uint32_t)NSTAGE ? it : (uint32_t)NSTAGE;
+      for (uint32_t i = 1; i <= n; ++i) {
+        const uint32_t j = it - i;
+        mbar_settle(bar(B_FULL + (int)(j % NSTAGE)), (j / NSTAGE) & 1);
+      }
+      for (uint32_t i = 1; i <= (rarmed < 2u ? rarmed : 2u); ++i) {     // and the tiles' scale vectors
+        const uint32_t j = rarmed - i;
+        mbar_settle(bar(B_RFULL + (int)(j & 1)), (j >> 1) & 1);
+      }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
