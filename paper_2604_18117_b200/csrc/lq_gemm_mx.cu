@@ -121,6 +121,9 @@ __device__ __forceinline__ void combine_fragment(float (&a)[4], const uint32_t* 
   }
 }
 
+// BRANCH_ACC: the layer has an integer branch with fp32 scales, whose product needs an accumulator of its own.  The
+// other instance (no branch, fp16 branch, MX branches) carries none of that code or its registers.
+template <bool BRANCH_ACC>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmT,
@@ -147,7 +150,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const bool has_branch = p.branch_steps > 0;
   // An fp16 branch has no scales: its product is accumulated onto the main accumulator by the tensor core and the drain
   // sees no branch at all.  An integer branch needs its fp32 scales applied per element: second accumulator.
-  const bool branch_acc = has_branch && !p.branch_f16 && !p.branch_mx;
+  constexpr bool branch_acc = BRANCH_ACC;                 // = has_branch && !p.branch_f16 && !p.branch_mx, decided by the host
   // Each CTA takes a contiguous, equal share of the work and walks it as 256-wide tiles (128-wide where a row block or
   // the share ends).  A 128-wide tile costs nearly as much as a 256-wide one (a stage's time is set by its hand-shakes
   // and instruction count, not its MMA width).  by_units = 0 shares whole tiles - row blocks cut into 256-wide tiles
@@ -492,7 +495,9 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
 lq_status lq_gemm_mx_prepare(int device) {
   if (cudaSetDevice(device) != cudaSuccess) return LQ_ERR_CUDA;
-  if (lq_note_cuda(cudaFuncSetAttribute(lq_gemm_mx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) !=
+  if (lq_note_cuda(cudaFuncSetAttribute(lq_gemm_mx_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) !=
+          cudaSuccess ||
+      lq_note_cuda(cudaFuncSetAttribute(lq_gemm_mx_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES)) !=
       cudaSuccess)
     return LQ_ERR_CUDA;
   return LQ_OK;
@@ -521,6 +526,9 @@ lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_
   const long long tiles = (long long)p.tiles_m * ((p.units_n + 1) / 2);
   if (ctas > tiles) ctas = (int)tiles;
   p.by_units = (p.units_n & 1) && tiles < 4ll * ctas;
-  lq_gemm_mx_kernel<<<ctas, GEMM_THREADS, SMEM_BYTES, st>>>(A->tmA, L->tmB, L->tmB2, A->tmT, L->tmL2, p);
+  if (p.branch_steps > 0 && !p.branch_f16 && !p.branch_mx)
+    lq_gemm_mx_kernel<true><<<ctas, GEMM_THREADS, SMEM_BYTES, st>>>(A->tmA, L->tmB, L->tmB2, A->tmT, L->tmL2, p);
+  else
+    lq_gemm_mx_kernel<false><<<ctas, GEMM_THREADS, SMEM_BYTES, st>>>(A->tmA, L->tmB, L->tmB2, A->tmT, L->tmL2, p);
   return lq_note_cuda(cudaGetLastError()) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
 }
