@@ -59,7 +59,7 @@ typedef enum {
   LQ_BRANCH_MXFP4 = 7,
   /* Integer MX branches of the same study (Table 3's integer rows): factors in blocks of 32 with a power-of-two
    * scale and signed 8-bit / 4-bit integer codes; the activations of BOTH branches and the rank-r intermediate
-   * are MXINT8.  Only with main_fmt = LQ_MAIN_MXINT4_A8; rank <= 64. */
+   * are MXINT8.  Only with main_fmt = LQ_MAIN_MXINT4_A8; rank <= 64 with MXINT8 factors, <= 128 with MXINT4 factors. */
   LQ_BRANCH_MXINT8 = 8,
   LQ_BRANCH_MXINT4 = 9
 } lq_branch_fmt;

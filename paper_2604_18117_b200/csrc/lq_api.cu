@@ -100,10 +100,11 @@ static lq_status check_config(const lq_config* c) {
     return LQ_ERR_UNSUPPORTED;
   if (c->main_fmt != LQ_MAIN_MXFP4 && lq_branch_is_mxfp(c->branch)) return LQ_ERR_UNSUPPORTED;
   if (c->act_fmt != LQ_ACT_DEFAULT && !(c->act_fmt == LQ_ACT_MXFP6 && c->main_fmt == LQ_MAIN_MXFP4)) return LQ_ERR_UNSUPPORTED;
-  // MXINT8 activations go with MXINT4 weights in blocks of 32 and an integer MX (or no) branch of rank <= 64 (the two
-  // digit planes of the rank-r intermediate share the 128-byte container)
+  // MXINT8 activations go with MXINT4 weights in blocks of 32 and an integer MX (or no) branch; MXINT8 factors: rank <= 64
+  // (both operands of the up-projection carry two digit planes, which share a 128-byte container each); MXINT4 factors:
+  // rank <= 128 (one plane for L2, a container per plane for the intermediate)
   if (c->main_fmt == LQ_MAIN_MXINT4_A8 &&
-      (c->group != LQ_MX_BLOCK || !(c->branch == LQ_BRANCH_NONE || lq_branch_is_mxint(c->branch)) || (c->branch != LQ_BRANCH_NONE && c->rank > 64)))
+      (c->group != LQ_MX_BLOCK || !(c->branch == LQ_BRANCH_NONE || lq_branch_is_mxint(c->branch)) || (c->branch == LQ_BRANCH_MXINT8 && c->rank > 64)))
     return LQ_ERR_UNSUPPORTED;
   if (c->main_fmt != LQ_MAIN_MXINT4_A8 && lq_branch_is_mxint(c->branch)) return LQ_ERR_UNSUPPORTED;
   if (c->K > LQ_MAX_K || (c->K % 8) != 0) return LQ_ERR_UNSUPPORTED;
@@ -487,7 +488,18 @@ extern "C" lq_status lq_layer_to_device(lq_layer* L, int device) {
       if ((st = upload(&L->d_s1b, s1b)) != LQ_OK) return st;
       // E8M0 bytes of L2's block scales along the rank, one 128-byte-of-rank stage: [1][Npad/128][512]
       std::vector<uint8_t> sfl2((size_t)(Npad / 128) * 512, 127);
-      if (L->a8) {
+      if (L->a8 && L->cfg.branch == LQ_BRANCH_MXINT4) {
+        // 4-bit codes are their own lo digit: one plane, K blocks in order (the intermediate brings its two planes as two
+        // stages against this one)
+        for (int j = 0; j < r; ++j)
+          for (int n = 0; n < N; ++n) l2c[(size_t)n * LQ_RCONT + j] = lq_digit_e4m3(L->L2q[(size_t)j * N + n]);
+        for (int c = 0; c < lq_ceil_div(r, 32); ++c)
+          for (int n = 0; n < N; ++n) {
+            int e = 0;
+            pow2_exponent(L->s2b[(size_t)c * N + n], &e);
+            sfl2[lq_sfb_offset(n, c, Npad)] = (uint8_t)(e + 127);
+          }
+      } else if (L->a8) {
         // two digit planes, code = 16 hi + lo: hi digits of rank index j at byte j, lo digits at byte 64 + j (rank <= 64);
         // the four 32-byte K blocks of the stage are (hi, block 0), (hi, block 1), (lo, block 0), (lo, block 1) with
         // scales 2^(e+4), 2^(e+4), 2^e, 2^e
@@ -561,6 +573,7 @@ extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device,
   memset(A, 0, sizeof(*A));
   A->K = L->K; A->N = L->N; A->r = L->r; A->G = L->G; A->Kpad = L->Kpad; A->Gpad = L->Gpad;
   A->mx = L->mx; A->mxfp = L->mxfp; A->a8 = L->a8; A->planes = L->a8 ? 2 : 1;
+  A->tq_stride = (L->a8 && L->cfg.branch == LQ_BRANCH_MXINT4) ? 2 * LQ_RCONT : LQ_RCONT;
   A->branch = L->cfg.branch; A->M_max = M_max; A->Mpad = lq_round_up(M_max, LQ_BM);
   A->device = device; A->main_kind = L->main_kind; A->M = 0;
   if (cudaSetDevice(device) != cudaSuccess) { delete A; return LQ_ERR_CUDA; }
@@ -569,23 +582,23 @@ extern "C" lq_status lq_act_create(const lq_layer* L, int32_t M_max, int device,
             cudaMalloc((void**)&A->d_sx, (size_t)A->Gpad * Mp * sizeof(float)) == cudaSuccess &&
             cudaMalloc((void**)&A->d_qb, Mp * Kp) == cudaSuccess &&
             cudaMalloc((void**)&A->d_sXb, Mp * sizeof(float)) == cudaSuccess &&
-            cudaMalloc((void**)&A->d_tq, Mp * LQ_RCONT) == cudaSuccess &&
+            cudaMalloc((void**)&A->d_tq, Mp * A->tq_stride) == cudaSuccess &&
             cudaMalloc((void**)&A->d_sT, Mp * sizeof(float)) == cudaSuccess &&
             (!A->mx || cudaMalloc((void**)&A->d_sfa, (Mp / 128) * (Kx / 128) * 512) == cudaSuccess) &&
-            (!(A->mxfp || A->a8) || cudaMalloc((void**)&A->d_sft, (Mp / 128) * 512) == cudaSuccess);
+            (!(A->mxfp || A->a8) || cudaMalloc((void**)&A->d_sft, (Mp / 128) * 512 * (A->tq_stride / LQ_RCONT)) == cudaSuccess);
   if (!ok) { lq_act_free(A); return LQ_ERR_ALLOC; }
   // padding rows/columns are read by the GEMM's tiles: start from defined contents
   cudaMemset(A->d_qx8, 0, Mp * Kx);
   cudaMemset(A->d_sx, 0, (size_t)A->Gpad * Mp * sizeof(float));
   cudaMemset(A->d_qb, 0, Mp * Kp);
   cudaMemset(A->d_sXb, 0, Mp * sizeof(float));
-  cudaMemset(A->d_tq, 0, Mp * LQ_RCONT);
+  cudaMemset(A->d_tq, 0, Mp * A->tq_stride);
   cudaMemset(A->d_sT, 0, Mp * sizeof(float));
   if (A->mx) cudaMemset(A->d_sfa, 127, (Mp / 128) * (Kx / 128) * 512);
-  if (A->mxfp || A->a8) cudaMemset(A->d_sft, 127, (Mp / 128) * 512);
+  if (A->mxfp || A->a8) cudaMemset(A->d_sft, 127, (Mp / 128) * 512 * (A->tq_stride / LQ_RCONT));
   lq_status st;
   if ((st = lq_make_tmap_bytes(&A->tmA, A->d_qx8, Mp, Kx, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
-  if ((st = lq_make_tmap_bytes(&A->tmT, A->d_tq, Mp, LQ_RCONT, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
+  if ((st = lq_make_tmap_bytes(&A->tmT, A->d_tq, Mp, (uint64_t)A->tq_stride, LQ_BM)) != LQ_OK) { lq_act_free(A); return st; }
   if (cudaDeviceSynchronize() != cudaSuccess) { lq_act_free(A); return LQ_ERR_CUDA; }
   *out = A;
   return LQ_OK;
@@ -680,13 +693,13 @@ static lq_status forward_host(const lq_layer* L, lq_act* A, const void* Xh, int3
     V.d_qb = A->d_qb + (size_t)m0 * A->Kpad;
     V.d_sx = A->d_sx + m0;                                     // [Gpad][Mpad]: the row stride stays Mpad
     V.d_sXb = A->d_sXb + m0;
-    V.d_tq = A->d_tq + (size_t)m0 * LQ_RCONT;
+    V.d_tq = A->d_tq + (size_t)m0 * A->tq_stride;
     V.d_sT = A->d_sT + m0;
     if (A->mx) V.d_sfa = A->d_sfa + (size_t)(m0 / 128) * (A->Kpad / 128) * A->planes * 512;
-    if (A->mxfp || A->a8) V.d_sft = A->d_sft + (size_t)(m0 / 128) * 512;
+    if (A->mxfp || A->a8) V.d_sft = A->d_sft + (size_t)(m0 / 128) * 512 * (A->tq_stride / LQ_RCONT);
     lq_status s;
     if ((s = lq_make_tmap_bytes(&V.tmA, V.d_qx8, (uint64_t)(A->Mpad - m0), (uint64_t)A->Kpad * A->planes, LQ_BM)) != LQ_OK) return s;
-    if ((s = lq_make_tmap_bytes(&V.tmT, V.d_tq, (uint64_t)(A->Mpad - m0), LQ_RCONT, LQ_BM)) != LQ_OK) return s;
+    if ((s = lq_make_tmap_bytes(&V.tmT, V.d_tq, (uint64_t)(A->Mpad - m0), (uint64_t)A->tq_stride, LQ_BM)) != LQ_OK) return s;
     if ((s = lq_launch_quantize(L, xd, Mc, &V, st)) != LQ_OK) return s;
     if ((s = (L->mx ? lq_launch_gemm_mx(L, &V, yd, dt, st) : lq_launch_gemm(L, &V, yd, dt, st))) != LQ_OK) return s;
     CUDA_OK(cudaEventRecord(A->ev_y[c], st));
@@ -775,25 +788,28 @@ extern "C" lq_status lq_act_export(const lq_act* A, int8_t* qx, uint16_t* sx, in
     }
     if (sXb && r > 0 && !A->mxfp && !A->a8) CUDA_OK(cudaMemcpy(sXb, A->d_sXb, M * sizeof(float), cudaMemcpyDeviceToHost));
     if (tq && r > 0) {
-      std::vector<uint8_t> h((size_t)M * LQ_RCONT);
+      const size_t ts = (size_t)A->tq_stride, lo_at = ts / 2;     // a8: the lo digits sit half a container row after the hi digits
+      std::vector<uint8_t> h((size_t)M * ts);
       CUDA_OK(cudaMemcpy(h.data(), A->d_tq, h.size(), cudaMemcpyDeviceToHost));
       const int eb = A->branch == LQ_BRANCH_W16A16 ? 2 : 1;
       if (A->a8) {
         for (int m = 0; m < M; ++m)
           for (int j = 0; j < r; ++j)
             ((int8_t*)tq)[(size_t)m * r + j] =
-                (int8_t)(16 * decode_digit(h[(size_t)m * LQ_RCONT + j]) + decode_digit(h[(size_t)m * LQ_RCONT + 64 + j]));
+                (int8_t)(16 * decode_digit(h[(size_t)m * ts + j]) + decode_digit(h[(size_t)m * ts + lo_at + j]));
       } else {
-        for (int m = 0; m < M; ++m) memcpy((uint8_t*)tq + (size_t)m * r * eb, h.data() + (size_t)m * LQ_RCONT, (size_t)r * eb);
+        for (int m = 0; m < M; ++m) memcpy((uint8_t*)tq + (size_t)m * r * eb, h.data() + (size_t)m * ts, (size_t)r * eb);
       }
     }
     if (sT && r > 0 && A->a8) {
       // the block exponents of the rank-r intermediate (the lo plane's scale bytes), as floats [M][ceil(r/32)]
-      std::vector<uint8_t> h((Mp / 128) * 512);
+      const bool split = A->tq_stride != LQ_RCONT;                // two chunks per row block: hi plane, lo plane
+      std::vector<uint8_t> h((Mp / 128) * 512 * (split ? 2 : 1));
       CUDA_OK(cudaMemcpy(h.data(), A->d_sft, h.size(), cudaMemcpyDeviceToHost));
       const int nbR = lq_ceil_div(r, LQ_MX_BLOCK);
       for (int m = 0; m < M; ++m)
-        for (int c = 0; c < nbR; ++c) sT[(size_t)m * nbR + c] = (float)((int)h[lq_sf_offset(m, 2 + c, 128)] - 127);
+        for (int c = 0; c < nbR; ++c)
+          sT[(size_t)m * nbR + c] = (float)((int)h[split ? lq_sf_offset(m, 4 + c, 256) : lq_sf_offset(m, 2 + c, 128)] - 127);
     } else if (sT && r > 0 && A->mxfp) {
       // MXFP: the block exponents of the rank-r intermediate as floats, [M][ceil(r/32)]
       std::vector<uint8_t> h((Mp / 128) * 512);

@@ -527,7 +527,7 @@ extern "C" lq_status lq_calibrate(const lq_config* cfg, const uint16_t* W16, con
   const bool a8 = cfg->main_fmt == LQ_MAIN_MXINT4_A8;
   if (cfg->act_fmt != LQ_ACT_DEFAULT && !(cfg->act_fmt == LQ_ACT_MXFP6 && mxfp)) return LQ_ERR_UNSUPPORTED;
   if (a8 ? !(cfg->branch == LQ_BRANCH_NONE || lq_branch_is_mxint(cfg->branch)) : lq_branch_is_mxint(cfg->branch)) return LQ_ERR_UNSUPPORTED;
-  if (a8 && (cfg->group != LQ_MX_BLOCK || cfg->rot_steps > 0 || (cfg->branch != LQ_BRANCH_NONE && cfg->rank > 64))) return LQ_ERR_UNSUPPORTED;
+  if (a8 && (cfg->group != LQ_MX_BLOCK || cfg->rot_steps > 0 || (cfg->branch == LQ_BRANCH_MXINT8 && cfg->rank > 64))) return LQ_ERR_UNSUPPORTED;
   if (mxfp ? !(cfg->branch == LQ_BRANCH_NONE || lq_branch_is_mxfp(cfg->branch)) : lq_branch_is_mxfp(cfg->branch)) return LQ_ERR_UNSUPPORTED;
   if (mxfp && (cfg->group != LQ_MX_BLOCK || cfg->rot_steps > 0)) return LQ_ERR_UNSUPPORTED;   // no rotation step for MXFP factors yet
   if ((cfg->group != LQ_GROUP && cfg->group != LQ_MX_BLOCK) || cfg->rot_steps < 0) return LQ_ERR_UNSUPPORTED;

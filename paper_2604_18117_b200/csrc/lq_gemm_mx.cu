@@ -77,7 +77,8 @@ struct MxParams {
   int branch_mx;          // the branch is MX as well: its up-projection is one more block-scaled stage onto the main
                           // accumulator.  1: MXFP elements, K blocks in order.  2: 8-bit integer codes as digit planes on
                           // both sides - the stage's four K blocks are (hi, 0), (hi, 1), (lo, 0), (lo, 1) and every
-                          // (plane of T, plane of L2) pair of the same rank block is one MMA
+                          // (plane of T, plane of L2) pair of the same rank block is one MMA.  3: the same codes with 4-bit
+                          // factors (one plane) and rank up to 128: two stages like mode 1, one per plane of T
   const uint8_t* sft;     // branch_mx: E8M0 bytes of T's block scales, [Mpad/128][512]
   const uint8_t* sfl2;    // branch_mx: E8M0 bytes of L2's block scales, [Npad/128][512]
   int tiles_m, units_n;
@@ -148,6 +149,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // provably warp-uniform
   const int lane = threadIdx.x & 31;
   const bool has_branch = p.branch_steps > 0;
+  const int nbst = p.branch_mx == 3 ? 2 : 1;              // stages of the branch per tile
   // An fp16 branch has no scales: its product is accumulated onto the main accumulator by the tensor core and the drain
   // sees no branch at all.  An integer branch needs its fp32 scales applied per element: second accumulator.
   constexpr bool branch_acc = BRANCH_ACC;                 // = has_branch && !p.branch_f16 && !p.branch_mx, decided by the host
@@ -237,7 +239,9 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         __syncwarp();
         LQ_TL(EV_P_ISSUED, s);
       }
-      if (has_branch && ok) {   // the branch operands: the containers of tq (128 rows) and L2q (256 rows), r contiguous
+      // the branch operands: the containers of tq (128 rows) and L2q (256 rows), r contiguous; mode 3 brings the two
+      // digit planes of tq as two stages against the same L2q
+      for (int bs = 0; bs < nbst && has_branch && ok; ++bs) {
         const int st = it % NSTAGE;
         ok = mbar_wait_warp(bar(B_EMPTY + st), ((it / NSTAGE) & 1) ^ 1, abort_flag, p.status, LQ_STAGE_PRODUCER);
         if (!ok) break;
@@ -245,12 +249,12 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const uint32_t full = bar(B_FULL + st);
         if (elect_one()) {
           mbar_expect_tx(full, STAGE_A_BYTES + width * (UNIT * LQ_KSTAGE) + (p.branch_mx ? (1 + width) * SF_BYTES : 0));
-          tma_load_2d(a_dst, &tmT, 0, m0, full);
+          tma_load_2d(a_dst, &tmT, bs * LQ_KSTAGE, m0, full);
           tma_load_2d(b_dst, &tmL2, 0, n0, full);
           if (width == 2) tma_load_2d(b_dst + UNIT * LQ_KSTAGE, &tmL2, 0, n0 + UNIT, full);
           if (p.branch_mx) {   // the block scales of T (rows) and of L2 (columns) along the rank
             const uint32_t sf_dst = sm_sf + st * STAGE_SF_BYTES;
-            bulk_load(sf_dst, p.sft + (size_t)mb * SF_BYTES, SF_BYTES, full);
+            bulk_load(sf_dst, p.sft + ((size_t)mb * nbst + bs) * SF_BYTES, SF_BYTES, full);
             bulk_load(sf_dst + SF_BYTES, p.sfl2 + (size_t)nu * SF_BYTES, width * SF_BYTES, full);
           }
         }
@@ -306,7 +310,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         LQ_TL(EV_M_ISSUED, s);
       }
       if (!ok) break;
-      if (has_branch) {
+      for (int bs = 0; bs < nbst && has_branch; ++bs) {
         const int st = it % NSTAGE;
         ok = mbar_wait_warp(bar(B_FULL + st), (it / NSTAGE) & 1, abort_flag, p.status, LQ_STAGE_MMA);
         if (!ok) break;
@@ -345,6 +349,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         __syncwarp();
         ++it;
       }
+      if (!ok) break;
       if (elect_one()) tc_commit(bar(B_TFULL));
       __syncwarp();
       LQ_TL(EV_TILE, 0);
@@ -511,7 +516,7 @@ lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_
   p.b_wrap = L->Kpad / LQ_KSTAGE;
   p.k_stages = p.b_wrap * A->planes;
   p.branch_f16 = L->f16_branch ? 1 : 0;
-  p.branch_mx = L->r == 0 ? 0 : L->mxfp ? 1 : L->a8 ? 2 : 0;
+  p.branch_mx = L->r == 0 ? 0 : L->mxfp ? 1 : !L->a8 ? 0 : L->cfg.branch == LQ_BRANCH_MXINT4 ? 3 : 2;
   p.sft = A->d_sft; p.sfl2 = L->d_sfl2;
   p.branch_steps = L->r == 0 ? 0 : lq_ceil_div(L->r, L->f16_branch ? 16 : 32);   // a8: rank blocks of 32 (at most two)
   p.tiles_m = lq_ceil_div(A->M, LQ_BM);

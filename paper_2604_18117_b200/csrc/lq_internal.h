@@ -105,6 +105,8 @@ struct lq_act {
   int K, N, r, G, Kpad, Gpad, branch;
   bool mx, mxfp, a8;
   int planes;                  // 1, or 2 (a8): digit planes of the main codes; qx8 rows are planes * Kpad bytes
+  int tq_stride;               // bytes per row of d_tq: LQ_RCONT, or 2 LQ_RCONT when the intermediate's two digit planes get a
+                               // container each (a8 with MXINT4 factors: rank up to 128), d_sft then holds two chunks per row block
   uint8_t* d_sft;              // mxfp: E8M0 bytes of the rank-r intermediate's block scales, [Mpad/128][1][512]
   uint8_t* d_sfa;              // MX: E8M0 bytes of the activation scales, [Mpad/128][Kpad/128][512], same layout
   int M_max, Mpad, device, main_kind;

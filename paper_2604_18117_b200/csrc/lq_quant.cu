@@ -63,6 +63,7 @@ struct QuantParams {
   uint8_t* tq;          // [Mpad][LQ_RCONT]
   float* sT;            // [Mpad]
   int r, rpad;          // rank, rank rounded up to 8
+  int tq_stride;        // bytes per row of tq: LQ_RCONT, or 2 LQ_RCONT when each digit plane of the intermediate has a container
   int act6;             // MXFP: the activations (X and the rank-r intermediate) are MXFP6e2 instead of MXFP8e4
   float qm;             // largest branch activation code
   int32_t* status;
@@ -706,11 +707,14 @@ __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, NTR >= 8 ? 1 : 
               const int e = mxint8_exponent(warp_max(fabsf(v)));
               const float inv = e == -127 ? 0.f : __uint_as_float((uint32_t)(127 - e) << 23);
               const Code8 cd = mxint8_code(v, inv);
-              p.tq[(size_t)m * LQ_RCONT + j] = (uint8_t)(f32x2_to_e4m3x2(0.f, cd.hi) & 0xFF);
-              p.tq[(size_t)m * LQ_RCONT + 64 + j] = (uint8_t)(f32x2_to_e4m3x2(0.f, cd.lo) & 0xFF);
+              // one container for both planes (rank <= 64): lo digits 64 bytes after the hi digits, scale slots c and
+              // 2 + c of one chunk; a container per plane (rank <= 128): lo digits 128 bytes on, slot c of the next chunk
+              const bool split = p.tq_stride != LQ_RCONT;
+              p.tq[(size_t)m * p.tq_stride + j] = (uint8_t)(f32x2_to_e4m3x2(0.f, cd.hi) & 0xFF);
+              p.tq[(size_t)m * p.tq_stride + (split ? 128 : 64) + j] = (uint8_t)(f32x2_to_e4m3x2(0.f, cd.lo) & 0xFF);
               if (lane == 0) {
-                uint8_t* sf = p.sft + (size_t)(m >> 7) * 512 + 16 * (m & 31) + 4 * ((m & 127) >> 5);
-                sf[c] = (uint8_t)(e + 4 + 127); sf[2 + c] = (uint8_t)(e + 127);
+                uint8_t* sf = p.sft + (size_t)(m >> 7) * (split ? 1024 : 512) + 16 * (m & 31) + 4 * ((m & 127) >> 5);
+                sf[c] = (uint8_t)(e + 4 + 127); sf[(split ? 512 : 2) + c] = (uint8_t)(e + 127);
               }
             }
           }
@@ -820,7 +824,8 @@ cudaError_t dispatch_quant(int br, int ntr, const CUtensorMap& tm, QuantParams& 
   if constexpr (MAIN == MAIN_MXINT8) {
     if (ntr <= 2) return launch_quant<MAIN, BR_MXINT, 2>(tm, p, sms, st);
     if (ntr <= 4) return launch_quant<MAIN, BR_MXINT, 4>(tm, p, sms, st);
-    return launch_quant<MAIN, BR_MXINT, 8>(tm, p, sms, st);
+    if (ntr <= 8) return launch_quant<MAIN, BR_MXINT, 8>(tm, p, sms, st);
+    return launch_quant<MAIN, BR_MXINT, 16>(tm, p, sms, st);
   } else if constexpr (MAIN == MAIN_MXFP) {
     if (ntr <= 2) return launch_quant<MAIN, BR_MXFP, 2>(tm, p, sms, st);
     if (ntr <= 4) return launch_quant<MAIN, BR_MXFP, 4>(tm, p, sms, st);
@@ -864,6 +869,7 @@ lq_status lq_launch_quantize(const lq_layer* L, const void* X, int M, lq_act* A,
   p.sL1 = L->d_sL1; p.tq = A->d_tq; p.sT = A->d_sT;
   p.s1b = L->d_s1b; p.sft = A->d_sft;
   p.r = L->r; p.rpad = ntr * 8;
+  p.tq_stride = A->tq_stride;
   p.act6 = (L->mxfp && L->cfg.act_fmt == LQ_ACT_MXFP6) ? 1 : 0;
   p.qm = br == BR_INT ? (float)((1 << (abits - 1)) - 1) : 0.f;
   p.status = lq_device_status_ptr(A->device);

@@ -69,10 +69,11 @@ def _check(layer, X):
     assert rel_fro(Y16, ref["Y"]) <= (5e-3 if r else 1e-3)
 
 
-@pytest.mark.parametrize("branch,r", [("none", 0), ("mxint8", 64), ("mxint4", 64), ("mxint8", 32), ("mxint8", 40)])
+@pytest.mark.parametrize("branch,r", [("none", 0), ("mxint8", 64), ("mxint4", 64), ("mxint8", 32), ("mxint8", 40),
+                                      ("mxint4", 128), ("mxint4", 96), ("mxint4", 24)])
 def test_mxint8_forward_table_3_integer_rows(branch, r):
-    """MXINT4 weights x MXINT8 activations with MXINT8 factors of rank 64 (Table 3) and neighbours, on a PixArt-shaped
-    layer slice, several row tiles and a ragged tail."""
+    """MXINT4 weights x MXINT8 activations with MXINT8 factors of rank 64 or MXINT4 factors of rank 128 (Table 3's two
+    integer rows) and neighbours, on a PixArt-shaped layer slice, several row tiles and a ragged tail."""
     rng = np.random.default_rng(20 + r)
     M, K, N = 300, 1152, 384
     X = (rng.standard_normal((M, K))).astype(np.float16)
