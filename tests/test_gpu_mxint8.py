@@ -130,3 +130,42 @@ def test_mxint8_full_size_layer_sampled_rows():
     finally:
         B.lq_act_free(act)
         B.lq_layer_free(h)
+
+
+@pytest.mark.parametrize("branch,r", [("mxint8", 64), ("mxint4", 128)])
+def test_mxint8_host_entry_point_pipelines_row_chunks(branch, r):
+    """lq_linear_forward_host with 8-bit activation codes: the row-chunk views of the activation record (two code planes
+    per row, scale bytes per plane, the intermediate's one or two containers) must give the same bits as one call over
+    all rows, and the exported codes of all chunks must match the oracle."""
+    import torch
+    from paper_2604_18117_b200 import binding as B
+    from tests.helpers import import_oracle_mxint_layer
+    rng = np.random.default_rng(8)
+    M, K, N = 1300, 1152, 392                              # five chunks, the last one ragged; N not a multiple of 128
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    layer = _layer(rng, K, N, r, branch)
+    ref = I.forward(X, layer)
+    h, cfg = import_oracle_mxint_layer(layer)
+    B.lq_layer_to_device(h, 0)
+    act = B.lq_act_create(h, M, 0)
+    try:
+        st = torch.cuda.current_stream().cuda_stream
+        Xp = torch.from_numpy(X).pin_memory()
+        Yp = torch.full((M, N), float("nan"), dtype=torch.float16).pin_memory()
+        B.lq_linear_forward_host(h, act, Xp.data_ptr(), M, Yp.data_ptr(), B.OUT_F16, st)
+        assert B.lq_get_device_status(0)[0] == 0
+        Yh = Yp.numpy().copy()
+        ex = B.lq_act_export(act, M, cfg, st)
+        assert np.array_equal(ex["qx"].astype(np.int16), ref["xa"]) and np.array_equal(ex["sx"], ref["ex"])
+        Xd = torch.from_numpy(X).cuda()
+        Yd = torch.full((M, N), float("nan"), dtype=torch.float16, device="cuda")
+        B.lq_quantize_act(h, Xd.data_ptr(), M, act, st)
+        B.lq_linear_forward(h, act, Yd.data_ptr(), B.OUT_F16, st)
+        torch.cuda.synchronize()
+        ex2 = B.lq_act_export(act, M, cfg, st)
+        assert np.array_equal(ex["tq"], ex2["tq"]) and np.array_equal(ex["sT"], ex2["sT"])
+        assert np.array_equal(Yh, Yd.cpu().numpy())
+        assert rel_fro(Yh, ref["Y"]) <= 5e-3
+    finally:
+        B.lq_act_free(act)
+        B.lq_layer_free(h)
