@@ -116,3 +116,39 @@ def test_mxfp6_activations_table_4_rows(branch, r):
     layer = _layer(rng, K, N, r, branch)
     layer["act"] = "e2m3"
     _check(layer, X)
+
+
+def test_mxfp_host_entry_point_pipelines_row_chunks():
+    """lq_linear_forward_host with an MXFP layer: the row-chunk views of the activation record (element bytes, scale bytes
+    in chunks of 128 rows, the intermediate and its scale bytes) must give the same bits as one call over all rows."""
+    import torch
+    from tests.helpers import import_oracle_mxfp_layer
+    rng = np.random.default_rng(9)
+    M, K, N, r = 1300, 1152, 392, 64                       # five chunks, the last one ragged; N not a multiple of 128
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    layer = _layer(rng, K, N, r, "mxfp8")
+    ref = F.forward(X, layer)
+    h, cfg = import_oracle_mxfp_layer(layer)
+    B.lq_layer_to_device(h, 0)
+    act = B.lq_act_create(h, M, 0)
+    try:
+        st = torch.cuda.current_stream().cuda_stream
+        Xp = torch.from_numpy(X).pin_memory()
+        Yp = torch.full((M, N), float("nan"), dtype=torch.float16).pin_memory()
+        B.lq_linear_forward_host(h, act, Xp.data_ptr(), M, Yp.data_ptr(), B.OUT_F16, st)
+        assert B.lq_get_device_status(0)[0] == 0
+        Yh = Yp.numpy().copy()
+        ex = B.lq_act_export(act, M, cfg, st)
+        assert np.array_equal(B.e4m3_decode(ex["qx"]), ref["xa"]) and np.array_equal(ex["sx"], ref["ex"])
+        Xd = torch.from_numpy(X).cuda()
+        Yd = torch.full((M, N), float("nan"), dtype=torch.float16, device="cuda")
+        B.lq_quantize_act(h, Xd.data_ptr(), M, act, st)
+        B.lq_linear_forward(h, act, Yd.data_ptr(), B.OUT_F16, st)
+        torch.cuda.synchronize()
+        ex2 = B.lq_act_export(act, M, cfg, st)
+        assert np.array_equal(ex["tq"], ex2["tq"]) and np.array_equal(ex["sT"], ex2["sT"])
+        assert np.array_equal(Yh, Yd.cpu().numpy())
+        assert rel_fro(Yh, ref["Y"]) <= 5e-3
+    finally:
+        B.lq_act_free(act)
+        B.lq_layer_free(h)

@@ -169,3 +169,13 @@ def test_mxint8_host_entry_point_pipelines_row_chunks(branch, r):
     finally:
         B.lq_act_free(act)
         B.lq_layer_free(h)
+
+
+@pytest.mark.parametrize("M,K,N,r,branch", [(1, 32, 8, 0, "none"), (129, 96, 136, 8, "mxint8"), (257, 8192, 128, 128, "mxint4"),
+                                            (5, 160, 264, 33, "mxint8"), (1000, 40, 2000, 24, "mxint4"), (333, 5600, 24, 48, "mxint8")])
+def test_mxint8_edge_shapes(M, K, N, r, branch):
+    """One row, K below a block pair, the largest K and rank, ranks that end inside a block, N not a multiple of 128,
+    values from tiny to large."""
+    rng = np.random.default_rng(M + K)
+    X = (rng.standard_normal((M, K)) * rng.choice([0.01, 1.0, 30.0])).astype(np.float16)
+    _check(_layer(rng, K, N, r, branch, bias=(N % 16 == 0)), X)
