@@ -245,6 +245,10 @@ def workload_config(wl, args):
                    "L2 flushed (256 MiB write) before every timed step; layers inside a step run back to back"
                    if args.l2 == "flush" else
                    "no explicit flush: one step reads 132 MB of X and writes 170 MB of Y plus 66 MB of codes, the L2 holds 126 MB"),
+            "timing": ("`value` and `ms_per_step`: K steps with one CUDA-event pair around each step and nothing between the "
+                       "launches (launches overlap their set-up with the previous kernel's tail, as for a user); per-layer and "
+                       "per-kernel times (`layers`, `roofline`): the same K steps repeated with events around every launch, "
+                       "which serialises the launches - their step time is `ms_per_step_instrumented`"),
             "parallelism": f"rows sharded x{args.gpus}, no collective"}
 
 
@@ -329,7 +333,9 @@ def run_ours(args):
             B.lq_layer_free(L["h"])
 
     def measure(main, layers, steps, sample_clocks):
-        """Device-resident timing of `steps` steps; returns per-step and per-launch CUDA-event times."""
+        """Device-resident timing: `steps` steps with one event pair around each step (this is `value`: nothing sits between
+        the launches, so the library's overlapped launches work as they do for a user), then the same `steps` steps again
+        with events around every launch (per-layer and per-kernel times; their own step time is reported beside)."""
         r = STUDY[main][0] if main in STUDY else wl.rank
         def step(timed=None):
             if args.l2 == "flush" and not stack:
@@ -338,7 +344,7 @@ def run_ours(args):
                 timed["s"].record()
             for rep in range(repeats):
                 for i, L in enumerate(layers):
-                    ev = timed is not None and rep == 0
+                    ev = timed is not None and rep == 0 and "q0" in timed
                     if ev:
                         timed["q0"][i].record()
                     B.lq_quantize_act(L["h"], L["Xd"].data_ptr(), M, L["act"], st)
@@ -365,10 +371,14 @@ def run_ours(args):
         barrier()
         n_before = len(sampler.rows)
         t_timed = time.perf_counter()
-        for t in timers:
+        plain = [dict(s=ev(), e=ev()) for _ in range(steps)]
+        for t in plain:
             step(t)
         barrier()
         timed_wall = time.perf_counter() - t_timed
+        for t in timers:                          # the instrumented pass
+            step(t)
+        barrier()
         clocks = None
         if rank == 0 and sample_clocks:
             # The timed region of a short run is over before nvidia-smi (one line per 100 ms) reports: repeat the same
@@ -386,7 +396,8 @@ def run_ours(args):
         code, stage = B.lq_get_device_status(local)
         if code != 0:
             raise SystemExit(f"device status {code} (stage {stage}) after the timed region")
-        step_ms = [t["s"].elapsed_time(t["e"]) for t in timers]
+        step_ms = [t["s"].elapsed_time(t["e"]) for t in plain]
+        step_ms_instrumented = float(np.mean([t["s"].elapsed_time(t["e"]) for t in timers]))
         per_layer = []
         for i, L in enumerate(layers):
             q = float(np.mean([t["q0"][i].elapsed_time(t["g0"][i]) for t in timers]))
@@ -399,7 +410,8 @@ def run_ours(args):
                               "bounds_us": {k: round(v, 2) for k, v in bd.items() if k.endswith("_us")},
                               "k1_bytes": bd["k1_bytes"]})
         total_ms_max = D.max_over_ranks(float(sum(step_ms)), world, dev)
-        return {"total_ms": total_ms_max, "steps": steps, "layers": per_layer, "clocks": clocks}
+        return {"total_ms": total_ms_max, "steps": steps, "layers": per_layer, "clocks": clocks,
+                "ms_per_step_instrumented": step_ms_instrumented}
 
     def summarise(main, res):
         """value / roofline records of one measured format."""
@@ -436,6 +448,7 @@ def run_ours(args):
                  "frac": k1_bytes / (quant_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "avg_ms_sum": quant_ms}
         return {"value": D.job_throughput(ops_step, res["steps"], res["total_ms"], world) / 1e12,
                 "ms_per_step": res["total_ms"] / res["steps"],
+                "ms_per_step_instrumented": res["ms_per_step_instrumented"],
                 "tokens_per_s": D.job_throughput(M, res["steps"], res["total_ms"], world),
                 "roofline": roof, "roofline_quantizer": roofq}
 
@@ -478,7 +491,7 @@ def run_ours(args):
         mx_res = measure("mxint4", mx_layers, args.steps, True)
         mx_s = summarise("mxint4", mx_res)
         mx = {"what": "the same step with the MXINT4 main branch (blocks of 32, power-of-two scales, tcgen05 block-scaled MMA)",
-              "value": mx_s["value"], "unit": UNIT, "ms_per_step": mx_s["ms_per_step"], "tokens_per_s": mx_s["tokens_per_s"],
+              "value": mx_s["value"], "unit": UNIT, "ms_per_step": mx_s["ms_per_step"], "ms_per_step_instrumented": mx_s["ms_per_step_instrumented"], "tokens_per_s": mx_s["tokens_per_s"],
               "roofline": mx_s["roofline"], "roofline_quantizer": mx_s["roofline_quantizer"], "layers": mx_res["layers"],
               "clocks": mx_res["clocks"]}
         teardown(mx_layers)
@@ -490,7 +503,7 @@ def run_ours(args):
         fp_res = measure("mxfp4", fp_layers, args.steps, True)
         fp_s = summarise("mxfp4", fp_res)
         fp = {"what": f"the same layer shapes with MXFP4e2 residual weights, MXFP8e4 activations and a rank-{MXFP_RANK} {MXFP_BRANCH} branch",
-              "value": fp_s["value"], "unit": UNIT, "ms_per_step": fp_s["ms_per_step"], "tokens_per_s": fp_s["tokens_per_s"],
+              "value": fp_s["value"], "unit": UNIT, "ms_per_step": fp_s["ms_per_step"], "ms_per_step_instrumented": fp_s["ms_per_step_instrumented"], "tokens_per_s": fp_s["tokens_per_s"],
               "roofline": fp_s["roofline"], "roofline_quantizer": fp_s["roofline_quantizer"], "layers": fp_res["layers"],
               "clocks": fp_res["clocks"]}
         teardown(fp_layers)
@@ -502,7 +515,7 @@ def run_ours(args):
         i8_res = measure("mxint4a8", i8_layers, args.steps, True)
         i8_s = summarise("mxint4a8", i8_res)
         i8 = {"what": f"the same layer shapes with MXINT4 residual weights, MXINT8 activations and a rank-{MXINT_RANK} {MXINT_BRANCH} branch",
-              "value": i8_s["value"], "unit": UNIT, "ms_per_step": i8_s["ms_per_step"], "tokens_per_s": i8_s["tokens_per_s"],
+              "value": i8_s["value"], "unit": UNIT, "ms_per_step": i8_s["ms_per_step"], "ms_per_step_instrumented": i8_s["ms_per_step_instrumented"], "tokens_per_s": i8_s["tokens_per_s"],
               "roofline": i8_s["roofline"], "roofline_quantizer": i8_s["roofline_quantizer"], "layers": i8_res["layers"],
               "clocks": i8_res["clocks"]}
         teardown(i8_layers)
@@ -512,7 +525,8 @@ def run_ours(args):
         line = {
             "metric": METRIC, "value": summ["value"], "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": summ["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "ms_per_step": summ["ms_per_step"], "ms_per_step_instrumented": summ["ms_per_step_instrumented"],
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "e4m3 (exact int4 codes) / int8 operands, fp32 accumulate", "data": "synthetic",
             "config": workload_config(wl, args),
             "tokens_per_s": summ["tokens_per_s"],

@@ -273,6 +273,9 @@ lq_status lq_selftest_wait_timeout(int device, void* cuda_stream);
  *                  return them (parity tests); 0 (default): they stay on chip
  *   "gemm_ctas"    CTAs of the GEMM kernels; 0 (default) = one per SM
  *   "quant_ctas", "quant_warps"   residency and consumer warps of the quantizer kernel; 0 = chosen by the library
+ *   "overlap"      1 (default): kernels are launched with programmatic stream serialization - a kernel's CTAs may take
+ *                  their SMs and set up while the previous kernel on the stream drains, and wait (in the kernel) for
+ *                  that kernel's completion before touching global memory; 0: plain launches
  *   "main_kind"    byte format that carries the 4-bit codes into the tensor cores; only 1 (E4M3) exists
  * Returns INVALID_ARG for an unknown name or value. */
 lq_status lq_set_option(const char* name, int32_t value);

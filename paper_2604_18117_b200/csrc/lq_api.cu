@@ -13,6 +13,7 @@ int g_lq_gemm_ctas = 0;
 int g_lq_store_qb = 0;
 int g_lq_quant_warps = 0;
 int g_lq_quant_ctas = 0;
+int g_lq_overlap = 1;
 
 static thread_local cudaError_t t_last_cuda_error = cudaSuccess;
 
@@ -67,6 +68,11 @@ extern "C" lq_status lq_set_option(const char* name, int32_t value) {
   if (!strcmp(name, "quant_ctas")) {
     if (value < 0 || value > 4) return LQ_ERR_INVALID_ARG;
     g_lq_quant_ctas = value;
+    return LQ_OK;
+  }
+  if (!strcmp(name, "overlap")) {
+    if (value != 0 && value != 1) return LQ_ERR_INVALID_ARG;
+    g_lq_overlap = value;
     return LQ_OK;
   }
   if (!strcmp(name, "gemm_ctas")) {

@@ -97,6 +97,13 @@ __device__ __forceinline__ void mbar_settle(uint32_t bar, uint32_t parity, long 
   while (!mbar_try_wait(bar, parity) && clock64() - t0 < limit) { }
 }
 
+// Programmatic dependent launch: let the next kernel on the stream start its set-up, then wait until the previous
+// kernel on the stream has completed and its writes are visible (both are no-ops for a plain launch).
+__device__ __forceinline__ void grid_dependency_sync() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred;
   asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.b32 %0, 1, 0, P;\n\t}" : "=r"(pred));

@@ -165,6 +165,7 @@ lq_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 512);
   tc_fence_before();
   __syncthreads();
+  grid_dependency_sync();        // set-up done; from here on global memory written by earlier kernels is read
   tc_fence_after();
   const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
 
@@ -463,6 +464,6 @@ lq_status lq_launch_gemm(const lq_layer* L, const lq_act* A, void* Y, lq_out_dty
   int ctas = g_lq_gemm_ctas > 0 ? g_lq_gemm_ctas : sms;
   const long long units = (long long)p.tiles_m * p.units_n;
   if (ctas > units) ctas = (int)units;
-  lq_gemm_kernel<<<ctas, GEMM_THREADS, SMEM_BYTES, st>>>(A->tmA, L->tmB, A->tmT, L->tmL2, p);
-  return lq_note_cuda(cudaGetLastError()) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
+  const cudaError_t e = lq_launch(lq_gemm_kernel, ctas, GEMM_THREADS, SMEM_BYTES, st, A->tmA, L->tmB, A->tmT, L->tmL2, p);
+  return lq_note_cuda(e != cudaSuccess ? e : cudaGetLastError()) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
 }

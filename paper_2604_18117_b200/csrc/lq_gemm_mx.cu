@@ -188,6 +188,7 @@ lq_gemm_mx_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   }
   tc_fence_before();
   __syncthreads();
+  grid_dependency_sync();        // set-up done; from here on global memory written by earlier kernels is read
   tc_fence_after();
   const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
 
@@ -531,9 +532,10 @@ lq_status lq_launch_gemm_mx(const lq_layer* L, const lq_act* A, void* Y, lq_out_
   const long long tiles = (long long)p.tiles_m * ((p.units_n + 1) / 2);
   if (ctas > tiles) ctas = (int)tiles;
   p.by_units = (p.units_n & 1) && tiles < 4ll * ctas;
+  cudaError_t launched;
   if (p.branch_steps > 0 && !p.branch_f16 && !p.branch_mx)
-    lq_gemm_mx_kernel<true><<<ctas, GEMM_THREADS, SMEM_BYTES, st>>>(A->tmA, L->tmB, L->tmB2, A->tmT, L->tmL2, p);
+    launched = lq_launch(lq_gemm_mx_kernel<true>, ctas, GEMM_THREADS, SMEM_BYTES, st, A->tmA, L->tmB, L->tmB2, A->tmT, L->tmL2, p);
   else
-    lq_gemm_mx_kernel<false><<<ctas, GEMM_THREADS, SMEM_BYTES, st>>>(A->tmA, L->tmB, L->tmB2, A->tmT, L->tmL2, p);
-  return lq_note_cuda(cudaGetLastError()) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
+    launched = lq_launch(lq_gemm_mx_kernel<false>, ctas, GEMM_THREADS, SMEM_BYTES, st, A->tmA, L->tmB, L->tmB2, A->tmT, L->tmL2, p);
+  return lq_note_cuda(launched != cudaSuccess ? launched : cudaGetLastError()) == cudaSuccess ? LQ_OK : LQ_ERR_CUDA;
 }

@@ -159,4 +159,24 @@ static inline uint8_t lq_encode_code_host(int q, int kind) {
 extern int g_lq_main_kind;   // option "main_kind"
 extern int g_lq_gemm_ctas;   // option "gemm_ctas" (0 = one per SM)
 extern int g_lq_quant_warps, g_lq_quant_ctas;   // options "quant_warps", "quant_ctas": 0 = chosen by the launcher
+extern int g_lq_overlap;     // option "overlap": launch kernels with programmatic stream serialization
 extern int g_lq_store_qb;    // option "store_qb": also write the branch activation codes to HBM (parity export)
+
+#ifdef __CUDACC__
+// Launches `kernel` on `st`.  With the "overlap" option the launch carries programmatic stream serialization: the
+// kernel's CTAs may become resident and run their set-up (barriers, tensor memory) while the previous kernel on the
+// stream is still draining its last tiles; every kernel of this library executes griddepcontrol.wait after that set-up,
+// before it reads or writes global memory, and griddepcontrol.launch_dependents right before it, so that the chain
+// quantizer -> GEMM -> next quantizer overlaps its launch gaps and tails.  All kernels here are persistent (the whole
+// grid is resident at once), so a waiting successor never holds an SM that a predecessor CTA still needs.
+template <typename... KArgs, typename... Args>
+static inline cudaError_t lq_launch(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3((unsigned)grid); lc.blockDim = dim3((unsigned)block); lc.dynamicSmemBytes = smem; lc.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at; lc.numAttrs = g_lq_overlap ? 1 : 0;
+  return cudaLaunchKernelEx(&lc, kernel, std::forward<Args>(args)...);
+}
+#endif

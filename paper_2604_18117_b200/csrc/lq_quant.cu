@@ -326,6 +326,7 @@ __global__ void __launch_bounds__((MAX_CONSUMER_WARPS + 1) * 32, NTR >= 8 ? 1 : 
     if (threadIdx.x < 2 * TR) rowmax_s[threadIdx.x] = 0;
   }
   __syncthreads();
+  grid_dependency_sync();        // set-up done; from here on X is read and the activation record written
 
   const int passes = (BR == BR_INT && p.refetch) ? 2 : 1;   // how often the producer streams a tile
 
@@ -814,8 +815,8 @@ cudaError_t launch_quant(const CUtensorMap& tm, QuantParams& p, int sms, cudaStr
   p.depth = pl.depth; p.refetch = pl.refetch;
   int grid = sms * pl.ctas_per_sm;
   if (grid > p.ntiles) grid = p.ntiles;
-  lq_quant_kernel<MAIN, BR, NTR><<<grid, (pl.W + 1) * 32, pl.smem, st>>>(tm, p);
-  return cudaGetLastError();
+  const cudaError_t e = lq_launch(lq_quant_kernel<MAIN, BR, NTR>, grid, (pl.W + 1) * 32, pl.smem, st, tm, p);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 template <int MAIN>

@@ -243,3 +243,46 @@ def test_async_host_entry_point_on_two_streams():
         for j in jobs:
             B.lq_act_free(j["act"])
             B.lq_layer_free(j["h"])
+
+
+def test_overlapped_launches_keep_stream_order():
+    """The library launches its kernels so that a kernel may take its SMs and set up while the previous kernel on the
+    stream drains ("overlap" option, on by default); each kernel waits for that previous kernel before it touches global
+    memory.  Two layers are chained on one stream with no synchronisation in between - the second layer's input IS the
+    first layer's output - several times in a row; the result must be bit-identical with plain launches and agree with
+    the oracle run on the first layer's output."""
+    import torch
+    from tests.helpers import import_oracle_layer
+    rng = np.random.default_rng(21)
+    M, K, N1, N2, r = 2000, 1152, 1152, 384, 32
+    l1 = _random_layer(rng, K, N1, r, "w8a8")
+    l2 = _random_layer(rng, N1, N2, r, "w8a8")
+    X = (rng.standard_normal((M, K))).astype(np.float16)
+    h1, _ = import_oracle_layer(l1)
+    h2, _ = import_oracle_layer(l2)
+    for h in (h1, h2):
+        B.lq_layer_to_device(h, 0)
+    a1, a2 = B.lq_act_create(h1, M, 0), B.lq_act_create(h2, M, 0)
+    st = torch.cuda.current_stream().cuda_stream
+    Xd = torch.from_numpy(X).cuda()
+    out = {}
+    try:
+        for overlap in (1, 0):
+            B.lq_set_option("overlap", overlap)
+            Y1 = torch.zeros((M, N1), dtype=torch.float16, device="cuda")
+            Y2 = torch.zeros((M, N2), dtype=torch.float16, device="cuda")
+            for _ in range(3):                               # back to back: the next round's first kernel follows the last GEMM
+                B.lq_quantize_act(h1, Xd.data_ptr(), M, a1, st)
+                B.lq_linear_forward(h1, a1, Y1.data_ptr(), B.OUT_F16, st)
+                B.lq_quantize_act(h2, Y1.data_ptr(), M, a2, st)
+                B.lq_linear_forward(h2, a2, Y2.data_ptr(), B.OUT_F16, st)
+            torch.cuda.synchronize()
+            assert B.lq_get_device_status(0)[0] == 0
+            out[overlap] = (Y1.cpu().numpy(), Y2.cpu().numpy())
+        assert np.array_equal(out[1][0], out[0][0]) and np.array_equal(out[1][1], out[0][1])
+        assert rel_fro(out[1][0], O.forward(X, l1)["Y"]) <= TOL_F16
+        assert rel_fro(out[1][1], O.forward(out[1][0], l2)["Y"]) <= TOL_F16
+    finally:
+        B.lq_set_option("overlap", 1)
+        B.lq_act_free(a1); B.lq_act_free(a2)
+        B.lq_layer_free(h1); B.lq_layer_free(h2)
