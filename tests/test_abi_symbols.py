@@ -2,6 +2,7 @@
 import ctypes
 import os
 import re
+import pytest
 
 from paper_2604_18117_b200 import binding as B
 from paper_2604_18117_b200 import build as BUILD
@@ -40,3 +41,18 @@ def test_argument_errors_without_gpu():
                                ctypes.byref(out)) == 2
     assert lib.lq_quantize_act(None, None, 1, None, None) == 1
     assert lib.lq_set_option(b"no_such_option", 1) == 1
+
+
+def test_option_names_and_values_are_checked():
+    """lq_set_option knows its names and value ranges (no GPU needed: the switches are plain process-wide settings)."""
+    from paper_2604_18117_b200 import binding as B
+    for name, good, bad in (("overlap", (0, 1), (2, -1)), ("store_qb", (1, 0), ()), ("quant_ctas", (1, 0), (5,)),
+                            ("quant_warps", (9, 0), (10,)), ("gemm_ctas", (7, 0), (-1,))):
+        for v in good:
+            B.lq_set_option(name, v)
+        for v in bad:
+            with pytest.raises(B.LqError):
+                B.lq_set_option(name, v)
+    with pytest.raises(B.LqError):
+        B.lq_set_option("no_such_option", 1)
+    B.lq_set_option("overlap", 1)
